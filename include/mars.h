@@ -1,0 +1,204 @@
+/*
+ * mars.h -- C ABI of the B200 rollout-step library (libmars.so).
+ *
+ * The library computes what the paper's "Rollout module" (Section 3.3, agentic pipeline
+ * parallelism; Section 2.3, segment rollouts) computes for a ragged batch of live Solver /
+ * Verifier / Corrector trajectories: one forward pass of the shared policy model (a
+ * Qwen3-30B-A3B-shaped mixture-of-experts decoder, Section 4.1) over the new tokens of every
+ * sequence, attending over that sequence's paged key/value cache, then the sampled next token and
+ * its log-probability under the behaviour policy (the denominator of the importance ratio,
+ * Eq. 3).  All roles share one model and one set of sampling hyper-parameters (Section 4.1), so a
+ * step has no per-role branch.
+ *
+ * General rules
+ *   - Every byte of DEVICE memory is the caller's: weights, KV pools, workspace, metadata, inputs
+ *     and outputs.  The library borrows the pointers for the lifetime of the handle that received
+ *     them and owns only small host-side structures (pinned staging buffers included).
+ *   - All device pointers must be 256-byte aligned unless stated otherwise.
+ *   - Matrices are bf16, row-major [out_features, in_features]; norm gains are bf16 vectors.
+ *   - Calls that take a stream are asynchronous on it; outputs are valid once the stream has been
+ *     synchronised.  One call at a time per mars_model_t / mars_kv_t.
+ *   - Errors are reported by return value only; on error nothing has been launched and the
+ *     out-parameters and the cache bookkeeping are unchanged.  Token ids that are out of range on
+ *     the device and bounded device-side waits that gave up are reported by mars_poll_status().
+ *   - The library needs an sm_100a device; there is no CPU path.
+ */
+#ifndef MARS_H_
+#define MARS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MARS_API __attribute__((visibility("default")))
+
+typedef int32_t mars_status_t;
+enum {
+    MARS_OK = 0,
+    MARS_ERR_INVALID_ARG = 1,  /* NULL / out-of-range / misaligned argument                         */
+    MARS_ERR_UNSUPPORTED = 2,  /* a shape the kernels are not built for (see mars_model_load)       */
+    MARS_ERR_CUDA = 3,         /* a CUDA runtime call failed (mars_last_cuda_error gives the code)   */
+    MARS_ERR_KV_FULL = 4,      /* no free page / sequence already at max_pages_per_seq              */
+    MARS_ERR_TIMEOUT = 5,      /* a bounded device-side wait gave up (seen by mars_poll_status)     */
+    MARS_ERR_BAD_HANDLE = 6,   /* unknown sequence slot, double release, page already owned, ...    */
+    MARS_ERR_BAD_TOKEN = 7     /* a token id read on the device was outside [0, vocab)              */
+};
+
+/* Model shape.  max_pos bounds context_length + new tokens of any sequence. */
+typedef struct {
+    int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim;
+    int32_t n_experts, top_k, expert_inter, vocab;
+    int32_t qk_norm;   /* 1: RMS-normalise every query / key head (gain [head_dim]) before RoPE */
+    int32_t max_pos;
+    float rope_theta;  /* rotate-half pairing (i, i + head_dim/2), angle pos * theta^(-2i/head_dim) */
+    float rms_eps;     /* inside the square root */
+} mars_config_t;
+
+/* One decoder layer; device pointers, bf16. */
+typedef struct {
+    const void *attn_norm;  /* [hidden]                                                    */
+    const void *wqkv;       /* [(n_q + 2 n_kv) head_dim, hidden]: q rows, k rows, v rows   */
+    const void *q_norm;     /* [head_dim] (ignored when qk_norm == 0)                      */
+    const void *k_norm;     /* [head_dim]                                                  */
+    const void *wo;         /* [hidden, n_q head_dim]                                      */
+    const void *mlp_norm;   /* [hidden]                                                    */
+    const void *router;     /* [n_experts, hidden]                                         */
+    const void *w_gate_up;  /* [n_experts, 2 expert_inter, hidden]: gate rows, then up rows */
+    const void *w_down;     /* [n_experts, hidden, expert_inter]                           */
+} mars_layer_t;
+
+typedef struct {
+    const void *embed;          /* [vocab, hidden]                       */
+    const void *final_norm;     /* [hidden]                              */
+    const void *lm_head;        /* [vocab, hidden] (untied)              */
+    const mars_layer_t *layers; /* HOST array of n_layers entries (copied by mars_model_load) */
+} mars_weights_t;
+
+/* Sampling of the next token (Section 4.1: training T 0.85 / top_p 1.0; evaluation T 0.6 /
+ * top_p 0.95; top_k is always -1 in the paper and is not implemented).
+ *   greedy != 0: token = argmax of the logits (lowest id on ties), log-prob at temperature 1.
+ *   greedy == 0: pi = softmax(logits / temperature); nucleus = shortest prefix in (pi descending,
+ *     id ascending) order with mass >= top_p; the token is drawn from pi restricted to the nucleus
+ *     by inverting the cumulative distribution taken in ASCENDING TOKEN ID with one uniform per
+ *     (seed, step, sequence slot) from Philox4x32-10 (key = seed, counter = (step lo, step hi,
+ *     slot, 0), u = ((x0 >> 8) + 0.5) / 2^24).  The log-prob returned is log pi[token] over the
+ *     full vocabulary at that temperature (the behaviour-policy probability of Eq. 3 when
+ *     top_p = 1). */
+typedef struct {
+    float temperature, top_p;
+    int32_t greedy;
+    int32_t reserved;
+    uint64_t seed;
+    uint64_t step;
+} mars_sampling_t;
+
+/* Optional taps for tests (all device pointers, any may be NULL; NULL struct in timed runs).
+ * n = number of token rows of the call (decode: n_seqs; prefill: total chunk tokens), except
+ * logits, which has one row per emitted token (decode: n_seqs; prefill: requests with emit). */
+typedef struct {
+    float *logits;             /* [rows, vocab]                                                  */
+    float *hidden;             /* [n_layers + 1, n, hidden]: residual before layer 0 / after each */
+    float *router_w;           /* [n_layers, n, top_k]                                            */
+    int32_t *router_idx;       /* [n_layers, n, top_k], larger probability first                  */
+    const int32_t *forced_idx; /* [n_layers, n, top_k] or NULL: route to these experts instead    */
+    float *nucleus_mass;       /* [rows]: probability mass of the nucleus (1 when greedy)         */
+} mars_debug_t;
+
+typedef struct mars_model mars_model_t;
+typedef struct mars_kv mars_kv_t;
+
+/* Bytes of device workspace mars_model_load needs for steps of at most max_decode_seqs decode
+ * sequences and max_prefill_tokens prefill tokens per call.  0 on invalid arguments. */
+MARS_API size_t mars_workspace_bytes(const mars_config_t *cfg, int32_t max_decode_seqs, int32_t max_prefill_tokens);
+
+/* Validates the shape (MARS_ERR_UNSUPPORTED unless head_dim is 64 or 128, n_q_heads / n_kv_heads
+ * is an integer <= 8, hidden and expert_inter are multiples of 64, top_k <= n_experts <= 1024,
+ * top_k <= 32), records the borrowed weight pointers (no copy) and carves the workspace.  The
+ * workspace content is private to the library between calls. */
+MARS_API mars_status_t mars_model_load(const mars_config_t *cfg, const mars_weights_t *weights, void *workspace,
+                              size_t workspace_bytes, int32_t max_decode_seqs, int32_t max_prefill_tokens,
+                              mars_model_t **out);
+MARS_API mars_status_t mars_model_free(mars_model_t *model);
+
+/* ---- paged KV cache -------------------------------------------------------------------------
+ * Pool layout (K and V separate, bf16): [n_layers][n_pages][n_kv_heads][page_size][head_dim];
+ * a page id addresses the same page in every layer.  n_pages = pool_bytes_each / bytes of one
+ * layer-page / n_layers.  page_size is 16, 32, 64 or 128 tokens.  meta is device memory of
+ * mars_kv_meta_bytes() bytes holding the block table [max_seqs][max_pages_per_seq] (int32). */
+MARS_API size_t mars_kv_meta_bytes(int32_t max_seqs, int32_t max_pages_per_seq);
+MARS_API mars_status_t mars_kv_alloc(mars_model_t *model, void *k_pool, void *v_pool, size_t pool_bytes_each,
+                            int32_t page_size, int32_t max_seqs, int32_t max_pages_per_seq, void *meta,
+                            size_t meta_bytes, mars_kv_t **out);
+MARS_API mars_status_t mars_kv_free(mars_kv_t *kv);
+MARS_API int32_t mars_kv_num_pages(const mars_kv_t *kv);
+MARS_API int32_t mars_kv_free_pages(const mars_kv_t *kv);
+
+/* Sequence slots 0 .. max_seqs-1.  reserve: make room for n_tokens_total tokens (allocates the
+ * missing pages from the free list; MARS_ERR_KV_FULL leaves the slot unchanged).  adopt: hand the
+ * slot a list of specific free pages that the caller has filled, with ctx_len tokens valid
+ * (MARS_ERR_BAD_HANDLE if a page is owned already or the slot is not empty).  set_len: declare how
+ * many cached tokens are valid (<= reserved capacity).  release: return the slot's pages. */
+MARS_API mars_status_t mars_kv_seq_reserve(mars_kv_t *kv, int32_t seq, int32_t n_tokens_total);
+MARS_API mars_status_t mars_kv_seq_adopt(mars_kv_t *kv, int32_t seq, const int32_t *pages /*host*/, int32_t n_pages,
+                                int32_t ctx_len);
+MARS_API mars_status_t mars_kv_seq_set_len(mars_kv_t *kv, int32_t seq, int32_t ctx_len);
+MARS_API mars_status_t mars_kv_seq_release(mars_kv_t *kv, int32_t seq);
+MARS_API int32_t mars_kv_seq_len(const mars_kv_t *kv, int32_t seq); /* -1 if the slot is invalid */
+/* Copies the slot's page ids (host array, capacity cap) and their count. */
+MARS_API mars_status_t mars_kv_block_table(const mars_kv_t *kv, int32_t seq, int32_t *pages_out, int32_t cap, int32_t *n);
+
+/* ---- the step ---------------------------------------------------------------------------------
+ * mars_decode_step: for each listed sequence slot b (context length c_b), feed in_tokens[b] at
+ * position c_b, append its key/value to the cache (a new page is taken from the free list when
+ * c_b is a multiple of page_size; MARS_ERR_KV_FULL is returned before anything is launched),
+ * attend over positions 0..c_b, and write the sampled token and its log-prob.  c_b becomes
+ * c_b + 1.  seq_ids: host, distinct.  in_tokens / out_tokens / out_logprobs: device arrays of
+ * n_seqs entries; out_tokens may be passed as the next call's in_tokens.
+ *
+ * mars_prefill_chunk: for request r, feed chunk_lens[r] tokens (device array `tokens`, requests
+ * concatenated) at positions c_r .. c_r + len - 1 with causal attention over the cache and the
+ * chunk itself; c_r grows by len.  Where emit_last[r] != 0 a token is sampled from the last
+ * position of the chunk; out_tokens / out_logprobs receive one entry per emitting request, in
+ * request order (they may be NULL when no request emits). */
+MARS_API mars_status_t mars_decode_step(mars_model_t *model, mars_kv_t *kv, void *cuda_stream, int32_t n_seqs,
+                               const int32_t *seq_ids, const int32_t *in_tokens, const mars_sampling_t *sampling,
+                               int32_t *out_tokens, float *out_logprobs, const mars_debug_t *debug);
+MARS_API mars_status_t mars_prefill_chunk(mars_model_t *model, mars_kv_t *kv, void *cuda_stream, int32_t n_reqs,
+                                 const int32_t *seq_ids, const int32_t *chunk_lens, const int32_t *tokens,
+                                 const int32_t *emit_last, const mars_sampling_t *sampling, int32_t *out_tokens,
+                                 float *out_logprobs, const mars_debug_t *debug);
+
+/* Host-buffer convenience for callers that keep tokens on the host: copies in_tokens to the
+ * device, runs mars_decode_step, copies the results back and synchronises the stream. */
+MARS_API mars_status_t mars_decode_step_host(mars_model_t *model, mars_kv_t *kv, void *cuda_stream, int32_t n_seqs,
+                                    const int32_t *seq_ids, const int32_t *in_tokens_host,
+                                    const mars_sampling_t *sampling, int32_t *out_tokens_host,
+                                    float *out_logprobs_host);
+
+/* Synchronises the stream of the last call and reads the device status word: MARS_OK,
+ * MARS_ERR_BAD_TOKEN or MARS_ERR_TIMEOUT; the word is cleared. */
+MARS_API mars_status_t mars_poll_status(mars_model_t *model);
+
+/* Counters of the last step call: kernels launched by it, attention work items, cached tokens read. */
+typedef struct {
+    int64_t kernel_launches;
+    int64_t attn_items;
+    int64_t kv_tokens_read; /* sum over token rows of (position + 1) */
+} mars_step_info_t;
+MARS_API mars_status_t mars_last_step_info(const mars_model_t *model, mars_step_info_t *out);
+
+/* Device array [n_layers] (int32) inside the workspace that every step overwrites with the number
+ * of distinct experts selected per layer; valid after the step's stream is synchronised. */
+MARS_API const int32_t *mars_active_experts_device(const mars_model_t *model);
+
+MARS_API int32_t mars_last_cuda_error(void);
+MARS_API const char *mars_status_string(mars_status_t status);
+MARS_API const char *mars_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MARS_H_ */

@@ -1,0 +1,294 @@
+"""ctypes binding of libmars.so: the same entry points as ``include/mars.h``, argument marshalling
+only.  PyTorch appears here for device memory and streams; every step of the computation runs in
+the library's CUDA kernels.  There is no fallback: if the shared library is missing the import of
+any entry point raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_float, c_int32, c_int64, c_size_t, c_uint64, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmars.so")
+
+MARS_OK = 0
+STATUS_NAMES = {0: "MARS_OK", 1: "MARS_ERR_INVALID_ARG", 2: "MARS_ERR_UNSUPPORTED", 3: "MARS_ERR_CUDA",
+                4: "MARS_ERR_KV_FULL", 5: "MARS_ERR_TIMEOUT", 6: "MARS_ERR_BAD_HANDLE", 7: "MARS_ERR_BAD_TOKEN"}
+LAYER_FIELDS = ("attn_norm", "wqkv", "q_norm", "k_norm", "wo", "mlp_norm", "router", "w_gate_up", "w_down")
+
+
+class MarsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} "
+                         f"({lib().mars_status_string(status).decode()}; cuda={lib().mars_last_cuda_error()})")
+
+
+class mars_config_t(ctypes.Structure):
+    _fields_ = [(n, c_int32) for n in ("n_layers", "hidden", "n_q_heads", "n_kv_heads", "head_dim", "n_experts",
+                                       "top_k", "expert_inter", "vocab", "qk_norm", "max_pos")] + \
+               [("rope_theta", c_float), ("rms_eps", c_float)]
+
+
+class mars_layer_t(ctypes.Structure):
+    _fields_ = [(n, c_void_p) for n in LAYER_FIELDS]
+
+
+class mars_weights_t(ctypes.Structure):
+    _fields_ = [("embed", c_void_p), ("final_norm", c_void_p), ("lm_head", c_void_p), ("layers", POINTER(mars_layer_t))]
+
+
+class mars_sampling_t(ctypes.Structure):
+    _fields_ = [("temperature", c_float), ("top_p", c_float), ("greedy", c_int32), ("reserved", c_int32),
+                ("seed", c_uint64), ("step", c_uint64)]
+
+
+class mars_debug_t(ctypes.Structure):
+    _fields_ = [("logits", c_void_p), ("hidden", c_void_p), ("router_w", c_void_p), ("router_idx", c_void_p),
+                ("forced_idx", c_void_p), ("nucleus_mass", c_void_p)]
+
+
+class mars_step_info_t(ctypes.Structure):
+    _fields_ = [("kernel_launches", c_int64), ("attn_items", c_int64), ("kv_tokens_read", c_int64)]
+
+
+# name -> (restype, argtypes); mirrors include/mars.h one to one
+SIGNATURES = {
+    "mars_workspace_bytes": (c_size_t, [POINTER(mars_config_t), c_int32, c_int32]),
+    "mars_model_load": (c_int32, [POINTER(mars_config_t), POINTER(mars_weights_t), c_void_p, c_size_t, c_int32, c_int32,
+                                  POINTER(c_void_p)]),
+    "mars_model_free": (c_int32, [c_void_p]),
+    "mars_kv_meta_bytes": (c_size_t, [c_int32, c_int32]),
+    "mars_kv_alloc": (c_int32, [c_void_p, c_void_p, c_void_p, c_size_t, c_int32, c_int32, c_int32, c_void_p, c_size_t,
+                                POINTER(c_void_p)]),
+    "mars_kv_free": (c_int32, [c_void_p]),
+    "mars_kv_num_pages": (c_int32, [c_void_p]),
+    "mars_kv_free_pages": (c_int32, [c_void_p]),
+    "mars_kv_seq_reserve": (c_int32, [c_void_p, c_int32, c_int32]),
+    "mars_kv_seq_adopt": (c_int32, [c_void_p, c_int32, POINTER(c_int32), c_int32, c_int32]),
+    "mars_kv_seq_set_len": (c_int32, [c_void_p, c_int32, c_int32]),
+    "mars_kv_seq_release": (c_int32, [c_void_p, c_int32]),
+    "mars_kv_seq_len": (c_int32, [c_void_p, c_int32]),
+    "mars_kv_block_table": (c_int32, [c_void_p, c_int32, POINTER(c_int32), c_int32, POINTER(c_int32)]),
+    "mars_decode_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), c_void_p,
+                                   POINTER(mars_sampling_t), c_void_p, c_void_p, POINTER(mars_debug_t)]),
+    "mars_prefill_chunk": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), POINTER(c_int32), c_void_p,
+                                     POINTER(c_int32), POINTER(mars_sampling_t), c_void_p, c_void_p,
+                                     POINTER(mars_debug_t)]),
+    "mars_decode_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), c_void_p,
+                                        POINTER(mars_sampling_t), c_void_p, c_void_p]),
+    "mars_poll_status": (c_int32, [c_void_p]),
+    "mars_last_step_info": (c_int32, [c_void_p, POINTER(mars_step_info_t)]),
+    "mars_active_experts_device": (c_void_p, [c_void_p]),
+    "mars_last_cuda_error": (c_int32, []),
+    "mars_status_string": (c_char_p, [c_int32]),
+    "mars_version": (c_char_p, []),
+}
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libmars.so; raises if it has not been built (python -m paper_2511_11373_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} is missing: build it with `python -m paper_2511_11373_b200.build`")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != MARS_OK:
+        raise MarsError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _i32_array(values):
+    values = [int(v) for v in values]
+    return (c_int32 * len(values))(*values), len(values)
+
+
+def _stream_handle(stream) -> c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return c_void_p(stream.cuda_stream)
+
+
+def make_config(model: dict, max_pos: int) -> mars_config_t:
+    return mars_config_t(model["n_layers"], model["hidden"], model["n_q_heads"], model["n_kv_heads"],
+                         model["head_dim"], model["n_experts"], model["top_k"], model["expert_inter"], model["vocab"],
+                         model.get("qk_norm", 0), max_pos, model.get("rope_theta", 1e6), model.get("rms_eps", 1e-6))
+
+
+def make_sampling(greedy=True, temperature=1.0, top_p=1.0, seed=0, step=0) -> mars_sampling_t:
+    return mars_sampling_t(float(temperature), float(top_p), int(bool(greedy)), 0, int(seed), int(step))
+
+
+def make_debug(logits=None, hidden=None, router_w=None, router_idx=None, forced_idx=None, nucleus_mass=None):
+    d = mars_debug_t(*[t.data_ptr() if t is not None else None
+                       for t in (logits, hidden, router_w, router_idx, forced_idx, nucleus_mass)])
+    d._keep = (logits, hidden, router_w, router_idx, forced_idx, nucleus_mass)
+    return d
+
+
+class Model:
+    """mars_model_load / mars_model_free.  `weights` is the nested dict of CUDA bf16 tensors produced by
+    ``workloads.make_weights``; the tensors are borrowed, not copied, and are kept alive here."""
+
+    def __init__(self, model: dict, weights: dict, max_decode_seqs: int, max_prefill_tokens: int = 0,
+                 max_pos: int = 4096):
+        self.shape = dict(model)
+        self.cfg = make_config(model, max_pos)
+        self.weights = weights
+        self.max_decode_seqs, self.max_prefill_tokens = max_decode_seqs, max_prefill_tokens
+        nbytes = lib().mars_workspace_bytes(byref(self.cfg), max_decode_seqs, max_prefill_tokens)
+        if nbytes == 0:
+            raise MarsError(2, "mars_workspace_bytes")
+        dev = weights["embed"].device
+        self.device = dev
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        layers = (mars_layer_t * len(weights["layers"]))()
+        for i, layer in enumerate(weights["layers"]):
+            for f in LAYER_FIELDS:
+                t = layer[f]
+                assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+                setattr(layers[i], f, t.data_ptr())
+        w = mars_weights_t(weights["embed"].data_ptr(), weights["final_norm"].data_ptr(), weights["lm_head"].data_ptr(),
+                           layers)
+        self._layers = layers
+        handle = c_void_p()
+        with torch.cuda.device(dev):
+            _check(lib().mars_model_load(byref(self.cfg), byref(w), _ptr(self.workspace), nbytes, max_decode_seqs,
+                                         max_prefill_tokens, byref(handle)), "mars_model_load")
+        self.handle = handle
+
+    def poll_status(self) -> int:
+        return lib().mars_poll_status(self.handle)
+
+    def last_step_info(self) -> dict:
+        info = mars_step_info_t()
+        _check(lib().mars_last_step_info(self.handle, byref(info)), "mars_last_step_info")
+        return dict(kernel_launches=info.kernel_launches, attn_items=info.attn_items,
+                    kv_tokens_read=info.kv_tokens_read)
+
+    def active_experts(self) -> torch.Tensor:
+        """Distinct experts selected per layer in the last step (copied to the host; synchronises)."""
+        p = lib().mars_active_experts_device(self.handle)
+        out = torch.empty(self.shape["n_layers"], dtype=torch.int32, device=self.device)
+        n = self.shape["n_layers"] * 4
+        torch.cuda.synchronize(self.device)
+        # device-to-device view of the library's counter array, through the workspace tensor
+        off = p - self.workspace.data_ptr()
+        out.copy_(self.workspace[off:off + n].view(torch.int32))
+        return out.cpu()
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().mars_model_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class KvCache:
+    """mars_kv_alloc / mars_kv_free and the per-sequence calls.  The pools are caller tensors of shape
+    [n_layers, n_pages, n_kv_heads, page_size, head_dim] (bf16)."""
+
+    def __init__(self, model: Model, k_pool: torch.Tensor, v_pool: torch.Tensor, page_size: int, max_seqs: int,
+                 max_pages_per_seq: int):
+        assert k_pool.is_cuda and k_pool.dtype == torch.bfloat16 and k_pool.is_contiguous() and k_pool.shape == v_pool.shape
+        self.model, self.k_pool, self.v_pool = model, k_pool, v_pool
+        self.page_size, self.max_seqs, self.max_pages_per_seq = page_size, max_seqs, max_pages_per_seq
+        nmeta = lib().mars_kv_meta_bytes(max_seqs, max_pages_per_seq)
+        self.meta = torch.empty(nmeta, dtype=torch.uint8, device=k_pool.device)
+        handle = c_void_p()
+        with torch.cuda.device(k_pool.device):
+            _check(lib().mars_kv_alloc(model.handle, _ptr(k_pool), _ptr(v_pool), k_pool.numel() * 2, page_size, max_seqs,
+                                       max_pages_per_seq, _ptr(self.meta), nmeta, byref(handle)), "mars_kv_alloc")
+        self.handle = handle
+
+    @property
+    def num_pages(self) -> int:
+        return lib().mars_kv_num_pages(self.handle)
+
+    @property
+    def free_pages(self) -> int:
+        return lib().mars_kv_free_pages(self.handle)
+
+    def seq_reserve(self, seq: int, n_tokens_total: int):
+        _check(lib().mars_kv_seq_reserve(self.handle, seq, n_tokens_total), "mars_kv_seq_reserve")
+
+    def seq_adopt(self, seq: int, pages, ctx_len: int):
+        arr, n = _i32_array(pages)
+        _check(lib().mars_kv_seq_adopt(self.handle, seq, arr, n, ctx_len), "mars_kv_seq_adopt")
+
+    def seq_set_len(self, seq: int, ctx_len: int):
+        _check(lib().mars_kv_seq_set_len(self.handle, seq, ctx_len), "mars_kv_seq_set_len")
+
+    def seq_release(self, seq: int):
+        _check(lib().mars_kv_seq_release(self.handle, seq), "mars_kv_seq_release")
+
+    def seq_len(self, seq: int) -> int:
+        return lib().mars_kv_seq_len(self.handle, seq)
+
+    def block_table(self, seq: int):
+        arr = (c_int32 * self.max_pages_per_seq)()
+        n = c_int32()
+        _check(lib().mars_kv_block_table(self.handle, seq, arr, self.max_pages_per_seq, byref(n)), "mars_kv_block_table")
+        return list(arr[: n.value])
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().mars_kv_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def mars_decode_step(model: Model, kv: KvCache, seq_ids, in_tokens: torch.Tensor, sampling: mars_sampling_t,
+                     out_tokens: torch.Tensor, out_logprobs: torch.Tensor, debug: mars_debug_t | None = None,
+                     stream=None) -> int:
+    """Returns the status code (0 = ok) without raising, so that error paths can be tested."""
+    arr, n = _i32_array(seq_ids)
+    return lib().mars_decode_step(model.handle, kv.handle, _stream_handle(stream), n, arr, _ptr(in_tokens),
+                                  byref(sampling), _ptr(out_tokens), _ptr(out_logprobs),
+                                  byref(debug) if debug is not None else None)
+
+
+def mars_prefill_chunk(model: Model, kv: KvCache, seq_ids, chunk_lens, tokens: torch.Tensor, emit_last,
+                       sampling: mars_sampling_t, out_tokens, out_logprobs, debug: mars_debug_t | None = None,
+                       stream=None) -> int:
+    ids, n = _i32_array(seq_ids)
+    lens, _ = _i32_array(chunk_lens)
+    emit, _ = _i32_array(emit_last) if emit_last is not None else (None, 0)
+    return lib().mars_prefill_chunk(model.handle, kv.handle, _stream_handle(stream), n, ids, lens, _ptr(tokens), emit,
+                                    byref(sampling), _ptr(out_tokens), _ptr(out_logprobs),
+                                    byref(debug) if debug is not None else None)
+
+
+def mars_decode_step_host(model: Model, kv: KvCache, seq_ids, in_tokens_host: torch.Tensor, sampling: mars_sampling_t,
+                          out_tokens_host: torch.Tensor, out_logprobs_host: torch.Tensor, stream=None) -> int:
+    """Host-buffer variant: CPU int32 / fp32 tensors in and out, copies included, synchronous."""
+    arr, n = _i32_array(seq_ids)
+    assert not in_tokens_host.is_cuda and not out_tokens_host.is_cuda and not out_logprobs_host.is_cuda
+    return lib().mars_decode_step_host(model.handle, kv.handle, _stream_handle(stream), n, arr, _ptr(in_tokens_host),
+                                       byref(sampling), _ptr(out_tokens_host), _ptr(out_logprobs_host))

@@ -1,0 +1,54 @@
+// Launch wrappers of the rollout-step kernels (host side declarations).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "step.h"
+
+namespace mars {
+
+struct KvView {
+    __nv_bfloat16* k_pool;
+    __nv_bfloat16* v_pool;
+    int32_t* block_table;  // [max_seqs][max_pages_per_seq]
+    int n_pages, page_size, max_pages_per_seq;
+};
+
+struct LayerW {
+    const __nv_bfloat16 *attn_norm, *wqkv, *q_norm, *k_norm, *wo, *mlp_norm, *router, *w_gate_up, *w_down;
+};
+
+struct DebugTaps {
+    float* hidden;            // [L + 1, n_tok, H] or null
+    float* router_w;          // [L, n_tok, k] or null
+    int32_t* router_idx;      // [L, n_tok, k] or null
+    const int32_t* forced_idx;  // [L, n_tok, k] or null
+    float* nucleus_mass;      // [n_emit] or null
+};
+
+// Each wrapper enqueues its kernel(s) on `st` and returns the number of kernels it launched.
+int launch_prep(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, int n_tok, cudaStream_t st);
+int launch_embed(const Shape& s, const Buffers& b, const StepLayout& lay, const __nv_bfloat16* embed,
+                 const int32_t* tokens, const __nv_bfloat16* first_gain, float* hidden_tap, int n_tok, cudaStream_t st);
+int launch_qkv(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
+               int n_tok, cudaStream_t st);
+int launch_oproj(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
+int launch_lm_head(const Shape& s, const Buffers& b, const StepLayout& lay, const __nv_bfloat16* lm_head, int n_emit,
+                   cudaStream_t st);
+
+int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_k,
+                     const CUtensorMap& tm_v, int layer, int n_tok, int n_items, int sm_count, cudaStream_t st);
+
+int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,
+                  cudaStream_t st);
+int launch_experts(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
+int launch_combine(const Shape& s, const Buffers& b, const __nv_bfloat16* next_gain, float* hidden_tap, int n_tok,
+                   cudaStream_t st);
+
+int launch_sample(const Shape& s, const Buffers& b, const StepLayout& lay, int n_emit, int32_t* out_tokens,
+                  float* out_logprobs, float* nucleus_mass, cudaStream_t st);
+
+// Opt-in shared-memory attributes etc.; call once per device before the first launch.
+cudaError_t init_kernels();
+
+}  // namespace mars

@@ -1,0 +1,273 @@
+// Dense parts of the rollout step: step preparation, embedding, RMSNorm + QKV projection +
+// per-head norm + RoPE + cache append, output projection + residual, lm_head.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace mars {
+
+// ---------------------------------------------------------------------------------------------
+// Step preparation: write the block-table entries of pages taken for this step and tabulate
+// (cos, sin)(pos * theta_i) for every token row (fp64 angles: pos reaches 64k and beyond, where an
+// fp32 product pos * theta_0 is already off by milliradians).
+__global__ void prep_kernel(Buffers b, StepLayout lay, KvView kv, int half_d) {
+    const int32_t* hdr = b.step;
+    const int n_tok = hdr[H_NTOK];
+    if (blockIdx.x == 0) {
+        const int n_up = hdr[H_NUPDATES];
+        const int32_t* up = b.step + lay.updates;
+        for (int i = threadIdx.x; i < n_up; i += blockDim.x)
+            kv.block_table[(size_t)up[3 * i] * kv.max_pages_per_seq + up[3 * i + 1]] = up[3 * i + 2];
+    }
+    const int32_t* pos = b.step + lay.tok_pos;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_tok * half_d; i += gridDim.x * blockDim.x) {
+        const int t = i / half_d, f = i - t * half_d;
+        double sn, cs;
+        sincos((double)pos[t] * b.inv_freq[f], &sn, &cs);
+        b.rope[i] = make_float2((float)cs, (float)sn);
+    }
+}
+
+int launch_prep(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, int n_tok, cudaStream_t st) {
+    const int total = n_tok * (s.D / 2);
+    int grid = (total + 255) / 256;
+    if (grid < 1) grid = 1;
+    if (grid > 1024) grid = 1024;
+    prep_kernel<<<grid, 256, 0, st>>>(b, lay, kv, s.D / 2);
+    return 1;
+}
+
+// ---------------------------------------------------------------------------------------------
+// RMSNorm of one fp32 row held in registers/shared memory -> bf16 row (gain applied).
+// Called by every thread of the block; `vals` are this thread's elements c = tid + i * blockDim.
+template <int MAX_PER_THREAD>
+__device__ __forceinline__ void rms_to_bf16(const float (&vals)[MAX_PER_THREAD], int H, float eps,
+                                            const __nv_bfloat16* gain, __nv_bfloat16* out, float* scratch) {
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < MAX_PER_THREAD; ++i) {
+        const int c = threadIdx.x + i * blockDim.x;
+        if (c < H) ss += vals[i] * vals[i];
+    }
+    ss = block_sum(ss, scratch);
+    const float r = rsqrtf(ss / (float)H + eps);
+#pragma unroll
+    for (int i = 0; i < MAX_PER_THREAD; ++i) {
+        const int c = threadIdx.x + i * blockDim.x;
+        if (c < H) out[c] = __float2bfloat16_rn(vals[i] * r * __bfloat162float(gain[c]));
+    }
+}
+
+constexpr int kRowThreads = 256;
+constexpr int kRowMaxPer = 32;  // hidden <= 8192
+
+// Embedding gather: x = embed[token] (fp32), h = rms(x) * gain of the first layer's attention norm.
+__global__ void __launch_bounds__(kRowThreads) embed_kernel(Shape s, Buffers b, const __nv_bfloat16* embed,
+                                                            const int32_t* tokens, const __nv_bfloat16* gain,
+                                                            float* hidden_tap) {
+    __shared__ float scratch[32];
+    const int t = blockIdx.x;
+    int tok = tokens[t];
+    if (tok < 0 || tok >= s.V) {
+        if (threadIdx.x == 0) atomicOr(b.err, kErrBadToken);
+        tok = 0;
+    }
+    float v[kRowMaxPer];
+#pragma unroll
+    for (int i = 0; i < kRowMaxPer; ++i) {
+        const int c = threadIdx.x + i * kRowThreads;
+        v[i] = 0.f;
+        if (c < s.H) {
+            v[i] = __bfloat162float(embed[(size_t)tok * s.H + c]);
+            b.x[(size_t)t * s.H + c] = v[i];
+            if (hidden_tap) hidden_tap[(size_t)t * s.H + c] = v[i];
+        }
+    }
+    rms_to_bf16<kRowMaxPer>(v, s.H, s.eps, gain, b.h + (size_t)t * s.H, scratch);
+}
+
+int launch_embed(const Shape& s, const Buffers& b, const StepLayout&, const __nv_bfloat16* embed, const int32_t* tokens,
+                 const __nv_bfloat16* first_gain, float* hidden_tap, int n_tok, cudaStream_t st) {
+    embed_kernel<<<n_tok, kRowThreads, 0, st>>>(s, b, embed, tokens, first_gain, hidden_tap);
+    return 1;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Y^T = W X^T for up to 64 tokens per block column: weights streamed once from HBM, activations
+// staged through shared memory in K chunks (double buffered with cp.async).
+constexpr int kGemmWarps = 4;
+constexpr int kGemmTok = 64;
+constexpr int kGemmKC = 256;
+constexpr int kGemmXBytes = kGemmTok * x_row_bytes(kGemmKC);
+
+enum { EPI_STORE = 0, EPI_RESID = 1 };
+
+struct GemmParams {
+    const __nv_bfloat16* W;     // [rows, K]
+    const __nv_bfloat16* X;     // [*, K]
+    const int32_t* row_index;   // optional: X row of token t is row_index[t]
+    float* out;                 // [n_tok, rows]
+    int rows, K, n_tok;
+};
+
+template <int EPI>
+__global__ void __launch_bounds__(kGemmWarps * 32) dense_gemm_kernel(GemmParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, tig = lane & 3;
+    const int row_base = (blockIdx.x * kGemmWarps + warp) * 16;
+    const int tok0 = blockIdx.y * kGemmTok;
+    const int n_here = min(kGemmTok, p.n_tok - tok0);
+    constexpr int xrow = x_row_bytes(kGemmKC);
+
+    const int r0 = min(row_base + gid, p.rows - 1), r1 = min(row_base + gid + 8, p.rows - 1);
+    const __nv_bfloat16* wrow[1][2] = {{p.W + (size_t)r0 * p.K + tig * 8, p.W + (size_t)r1 * p.K + tig * 8}};
+
+    auto load_chunk = [&](int c, int buf) {
+        unsigned char* dst = smem + (size_t)buf * kGemmXBytes;
+        constexpr int pieces = kGemmKC * 2 / 16;  // 16-byte pieces per row
+        for (int i = threadIdx.x; i < kGemmTok * pieces; i += blockDim.x) {
+            const int t = i / pieces, pc = i - t * pieces;
+            unsigned char* d = dst + (size_t)t * xrow + pc * 16;
+            if (t < n_here) {
+                const int src_row = p.row_index ? p.row_index[tok0 + t] : tok0 + t;
+                cp_async16(d, p.X + (size_t)src_row * p.K + (size_t)c * kGemmKC + pc * 8);
+            } else {
+                *reinterpret_cast<uint4*>(d) = make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
+
+    float acc[1][8][4];
+#pragma unroll
+    for (int n = 0; n < 8; ++n)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[0][n][j] = 0.f;
+
+    const int n_chunks = p.K / kGemmKC;   // K is a multiple of kGemmKC (checked on the host)
+    load_chunk(0, 0);
+    cp_async_commit();
+    for (int c = 0; c < n_chunks; ++c) {
+        if (c + 1 < n_chunks) {
+            load_chunk(c + 1, (c + 1) & 1);
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const __nv_bfloat16* wr[1][2] = {{wrow[0][0] + (size_t)c * kGemmKC, wrow[0][1] + (size_t)c * kGemmKC}};
+        const unsigned char* xs = smem + (size_t)(c & 1) * kGemmXBytes + (size_t)gid * xrow + tig * 16;
+        stream_mma<1, 8, 4>(wr, kGemmKC / 32, xs, 8 * xrow, acc);
+        __syncthreads();
+    }
+
+#pragma unroll
+    for (int n = 0; n < 8; ++n)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int row = row_base + gid + ((j >> 1) << 3);
+            const int t = n * 8 + 2 * tig + (j & 1);
+            if (row < p.rows && t < n_here) {
+                float* dst = p.out + (size_t)(tok0 + t) * p.rows + row;
+                if (EPI == EPI_RESID) *dst += acc[0][n][j];
+                else *dst = acc[0][n][j];
+            }
+        }
+}
+
+template <int EPI>
+static int launch_gemm(const GemmParams& p, cudaStream_t st) {
+    dim3 grid((p.rows + kGemmWarps * 16 - 1) / (kGemmWarps * 16), (p.n_tok + kGemmTok - 1) / kGemmTok);
+    dense_gemm_kernel<EPI><<<grid, kGemmWarps * 32, 2 * kGemmXBytes, st>>>(p);
+    return 1;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Per-head RMS norm (optional), rotary embedding, cache append.  One block per token row, one
+// warp per head in turn; lane l owns the rotation pairs (l + 32 i, l + 32 i + D/2).
+template <int D>
+__global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepLayout lay, KvView kv,
+                                                       const __nv_bfloat16* q_gain, const __nv_bfloat16* k_gain,
+                                                       int layer) {
+    constexpr int HALF = D / 2, PER = HALF / 32;
+    const int t = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_heads = s.nq + 2 * s.nkv;
+    const int pos = b.step[lay.tok_pos + t], seq = b.step[lay.tok_seq + t];
+    const int page = kv.block_table[(size_t)seq * kv.max_pages_per_seq + pos / kv.page_size];
+    const int slot = pos % kv.page_size;
+    const float* raw = b.qkv + (size_t)t * n_heads * D;
+    for (int head = warp; head < n_heads; head += 4) {
+        const bool is_q = head < s.nq, is_k = !is_q && head < s.nq + s.nkv;
+        float lo[PER], hi[PER];
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            lo[i] = raw[head * D + lane + 32 * i];
+            hi[i] = raw[head * D + lane + 32 * i + HALF];
+            ss += lo[i] * lo[i] + hi[i] * hi[i];
+        }
+        if (!is_q && !is_k) {  // value head: stored as is
+            const int hk = head - s.nq - s.nkv;
+            __nv_bfloat16* dst = kv.v_pool +
+                ((((size_t)layer * kv.n_pages + page) * s.nkv + hk) * kv.page_size + slot) * D;
+#pragma unroll
+            for (int i = 0; i < PER; ++i) {
+                dst[lane + 32 * i] = __float2bfloat16_rn(lo[i]);
+                dst[lane + 32 * i + HALF] = __float2bfloat16_rn(hi[i]);
+            }
+            continue;
+        }
+        if (s.qk_norm) {
+            ss = warp_sum(ss);
+            const float r = rsqrtf(ss / (float)D + s.eps);
+            const __nv_bfloat16* g = is_q ? q_gain : k_gain;
+#pragma unroll
+            for (int i = 0; i < PER; ++i) {
+                lo[i] *= r * __bfloat162float(g[lane + 32 * i]);
+                hi[i] *= r * __bfloat162float(g[lane + 32 * i + HALF]);
+            }
+        }
+        __nv_bfloat16* dst;
+        if (is_q) {
+            dst = b.q + ((size_t)t * s.nq + head) * D;
+        } else {
+            const int hk = head - s.nq;
+            dst = kv.k_pool + ((((size_t)layer * kv.n_pages + page) * s.nkv + hk) * kv.page_size + slot) * D;
+        }
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const float2 cs = b.rope[(size_t)t * HALF + lane + 32 * i];
+            dst[lane + 32 * i] = __float2bfloat16_rn(lo[i] * cs.x - hi[i] * cs.y);
+            dst[lane + 32 * i + HALF] = __float2bfloat16_rn(hi[i] * cs.x + lo[i] * cs.y);
+        }
+    }
+}
+
+int launch_qkv(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
+               int n_tok, cudaStream_t st) {
+    GemmParams p{w.wqkv, b.h, nullptr, b.qkv, (s.nq + 2 * s.nkv) * s.D, s.H, n_tok};
+    int n = launch_gemm<EPI_STORE>(p, st);
+    if (s.D == 128) qkv_post_kernel<128><<<n_tok, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer);
+    else qkv_post_kernel<64><<<n_tok, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer);
+    return n + 1;
+}
+
+int launch_oproj(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st) {
+    GemmParams p{w.wo, b.o, nullptr, b.x, s.H, s.nq * s.D, n_tok};
+    return launch_gemm<EPI_RESID>(p, st);
+}
+
+int launch_lm_head(const Shape& s, const Buffers& b, const StepLayout& lay, const __nv_bfloat16* lm_head, int n_emit,
+                   cudaStream_t st) {
+    GemmParams p{lm_head, b.h, b.step + lay.emit_rows, b.logits, s.V, s.H, n_emit};
+    return launch_gemm<EPI_STORE>(p, st);
+}
+
+cudaError_t init_dense_kernels() {
+    cudaError_t e = cudaFuncSetAttribute(dense_gemm_kernel<EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         2 * kGemmXBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(dense_gemm_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                2 * kGemmXBytes);
+}
+
+}  // namespace mars

@@ -1,0 +1,708 @@
+// Host side of libmars: argument checking, paged-KV bookkeeping, per-step work lists, launch
+// sequence.  Every step of the computation runs in the kernels; nothing here touches tensor data.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/mars.h"
+#include "kernels.h"
+
+namespace mars {
+cudaError_t init_dense_kernels();
+cudaError_t init_attn_kernels();
+cudaError_t init_moe_kernels();
+}  // namespace mars
+
+using namespace mars;
+
+static thread_local int32_t g_last_cuda_error = 0;
+
+#define CUDA_TRY(expr)                                   \
+    do {                                                 \
+        cudaError_t _e = (expr);                         \
+        if (_e != cudaSuccess) {                         \
+            g_last_cuda_error = (int32_t)_e;             \
+            return MARS_ERR_CUDA;                        \
+        }                                                \
+    } while (0)
+
+namespace {
+
+constexpr int kSpanTokens = 512;    // cached tokens per attention work item at decode
+constexpr int kStagingSlots = 4;
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Caps {
+    int n_tok;     // token rows per call
+    int n_emit;    // sampled rows per call
+    int n_updates; // block-table writes per call
+    int n_items;   // attention work items per call
+};
+
+Caps make_caps(const mars_config_t& c, int max_decode, int max_prefill) {
+    Caps k;
+    k.n_tok = std::max(max_decode, max_prefill);
+    k.n_emit = std::max(max_decode, 1);
+    k.n_updates = k.n_tok + k.n_emit;
+    k.n_items = max_decode * (c.max_pos / kSpanTokens + 2) + max_prefill;
+    return k;
+}
+
+StepLayout make_layout(const Caps& k) {
+    StepLayout l;
+    int at = H_WORDS;
+    auto take = [&](int words) { int o = at; at += (words + 3) & ~3; return o; };
+    l.tok_seq = take(k.n_tok);
+    l.tok_pos = take(k.n_tok);
+    l.tok_item_off = take(k.n_tok + 1);
+    l.emit_rows = take(k.n_emit);
+    l.emit_slot = take(k.n_emit);
+    l.updates = take(3 * k.n_updates);
+    l.items = take(4 * k.n_items);
+    l.total_words = at;
+    return l;
+}
+
+bool shape_supported(const mars_config_t& c) {
+    if (c.n_layers < 1 || c.hidden < 256 || c.hidden > 8192 || c.hidden % 256) return false;
+    if (c.head_dim != 64 && c.head_dim != 128) return false;
+    if (c.n_kv_heads < 1 || c.n_q_heads % c.n_kv_heads || c.n_q_heads / c.n_kv_heads > 8) return false;
+    if ((c.n_q_heads * c.head_dim) % 256) return false;
+    if (c.n_experts < 1 || c.n_experts > 1024 || c.top_k < 1 || c.top_k > 32 || c.top_k > c.n_experts) return false;
+    if (c.expert_inter < 64 || c.expert_inter % 64) return false;
+    if (c.vocab < 2 || c.max_pos < 1) return false;
+    return true;
+}
+
+// Carves the workspace; with base == nullptr only sizes are computed.
+size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsigned char* base, Buffers* b,
+             int32_t** io_in, int32_t** io_out, float** io_lp) {
+    size_t at = 0;
+    auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes, 256); return base ? base + o : nullptr; };
+    const size_t n = k.n_tok, H = c.hidden, D = c.head_dim, nq = c.n_q_heads, nkv = c.n_kv_heads, kk = c.top_k;
+    Buffers t;
+    t.step = (int32_t*)take((size_t)lay.total_words * 4);
+    t.err = (int32_t*)take(256);
+    t.x = (float*)take(n * H * 4);
+    t.h = (__nv_bfloat16*)take(n * H * 2);
+    t.qkv = (float*)take(n * (nq + 2 * nkv) * D * 4);
+    t.q = (__nv_bfloat16*)take(n * nq * D * 2);
+    t.o = (__nv_bfloat16*)take(n * nq * D * 2);
+    t.rope = (float2*)take(n * (D / 2) * 8);
+    t.inv_freq = (double*)take((D / 2) * 8);
+    t.part_o = (float*)take((size_t)k.n_items * nq * D * 4);
+    t.part_ml = (float2*)take((size_t)k.n_items * nq * 8);
+    t.route_idx = (int32_t*)take(n * kk * 4);
+    t.route_w = (float*)take(n * kk * 4);
+    t.expert_off = (int32_t*)take(((size_t)c.n_experts + 1) * 4);
+    t.slot_token = (int32_t*)take(n * kk * 4);
+    t.slot_of = (int32_t*)take(n * kk * 4);
+    t.active = (int32_t*)take((size_t)c.n_layers * 4);
+    t.act = (__nv_bfloat16*)take(n * kk * c.expert_inter * 2);
+    t.y = (float*)take(n * kk * H * 4);
+    t.logits = (float*)take((size_t)k.n_emit * c.vocab * 4);
+    int32_t* a = (int32_t*)take((size_t)k.n_emit * 4);
+    int32_t* o = (int32_t*)take((size_t)k.n_emit * 4);
+    float* lp = (float*)take((size_t)k.n_emit * 4);
+    if (b) *b = t;
+    if (io_in) *io_in = a;
+    if (io_out) *io_out = o;
+    if (io_lp) *io_lp = lp;
+    return at;
+}
+
+}  // namespace
+
+struct mars_model {
+    mars_config_t cfg;
+    Shape shape;
+    Caps caps;
+    StepLayout lay;
+    Buffers buf;
+    std::vector<LayerW> layers;
+    const __nv_bfloat16 *embed, *final_norm, *lm_head;
+    int32_t *io_in, *io_out;
+    float* io_lp;
+    int device, sm_count;
+    int max_decode, max_prefill;
+    int32_t* staging[kStagingSlots];
+    cudaEvent_t staged[kStagingSlots];
+    int next_slot;
+    cudaStream_t last_stream;
+    mars_step_info_t info;
+};
+
+struct SeqState {
+    bool used = false;
+    int len = 0;
+    std::vector<int32_t> pages;
+};
+
+struct mars_kv {
+    mars_model* model;
+    KvView view;
+    CUtensorMap tm_k, tm_v;
+    int max_seqs;
+    std::vector<SeqState> seqs;
+    std::vector<int32_t> free_list;   // stack of free page ids
+    std::vector<uint8_t> owned;
+};
+
+extern "C" {
+
+const char* mars_version(void) { return "mars-rollout-b200 0.1"; }
+int32_t mars_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* mars_status_string(mars_status_t s) {
+    switch (s) {
+        case MARS_OK: return "ok";
+        case MARS_ERR_INVALID_ARG: return "invalid argument";
+        case MARS_ERR_UNSUPPORTED: return "unsupported shape";
+        case MARS_ERR_CUDA: return "CUDA runtime error";
+        case MARS_ERR_KV_FULL: return "KV cache full";
+        case MARS_ERR_TIMEOUT: return "bounded device wait gave up";
+        case MARS_ERR_BAD_HANDLE: return "bad handle or sequence slot";
+        case MARS_ERR_BAD_TOKEN: return "token id out of range";
+        default: return "unknown status";
+    }
+}
+
+size_t mars_workspace_bytes(const mars_config_t* cfg, int32_t max_decode_seqs, int32_t max_prefill_tokens) {
+    if (!cfg || max_decode_seqs < 0 || max_prefill_tokens < 0 || max_decode_seqs + max_prefill_tokens < 1) return 0;
+    if (!shape_supported(*cfg)) return 0;
+    const Caps k = make_caps(*cfg, max_decode_seqs, max_prefill_tokens);
+    const StepLayout lay = make_layout(k);
+    return carve(*cfg, k, lay, nullptr, nullptr, nullptr, nullptr, nullptr);
+}
+
+mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w, void* workspace, size_t workspace_bytes,
+                              int32_t max_decode_seqs, int32_t max_prefill_tokens, mars_model_t** out) {
+    if (!cfg || !w || !workspace || !out || !w->layers || !w->embed || !w->final_norm || !w->lm_head)
+        return MARS_ERR_INVALID_ARG;
+    if (max_decode_seqs < 0 || max_prefill_tokens < 0 || max_decode_seqs + max_prefill_tokens < 1)
+        return MARS_ERR_INVALID_ARG;
+    if (!shape_supported(*cfg)) return MARS_ERR_UNSUPPORTED;
+    if ((uintptr_t)workspace % 256) return MARS_ERR_INVALID_ARG;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        const mars_layer_t& s = w->layers[l];
+        if (!s.attn_norm || !s.wqkv || !s.wo || !s.mlp_norm || !s.router || !s.w_gate_up || !s.w_down)
+            return MARS_ERR_INVALID_ARG;
+        if (cfg->qk_norm && (!s.q_norm || !s.k_norm)) return MARS_ERR_INVALID_ARG;
+    }
+    const Caps k = make_caps(*cfg, max_decode_seqs, max_prefill_tokens);
+    const StepLayout lay = make_layout(k);
+    if (workspace_bytes < carve(*cfg, k, lay, nullptr, nullptr, nullptr, nullptr, nullptr)) return MARS_ERR_INVALID_ARG;
+
+    int dev = 0, major = 0, sms = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (major != 10) return MARS_ERR_UNSUPPORTED;
+    CUDA_TRY(init_dense_kernels());
+    CUDA_TRY(init_attn_kernels());
+    CUDA_TRY(init_moe_kernels());
+
+    mars_model* m = new (std::nothrow) mars_model();
+    if (!m) return MARS_ERR_INVALID_ARG;
+    m->cfg = *cfg;
+    m->shape = Shape{cfg->n_layers, cfg->hidden, cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim, cfg->n_experts,
+                     cfg->top_k, cfg->expert_inter, cfg->vocab, cfg->qk_norm, cfg->rms_eps};
+    m->caps = k;
+    m->lay = lay;
+    carve(*cfg, k, lay, (unsigned char*)workspace, &m->buf, &m->io_in, &m->io_out, &m->io_lp);
+    m->layers.resize(cfg->n_layers);
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        const mars_layer_t& s = w->layers[l];
+        m->layers[l] = LayerW{(const __nv_bfloat16*)s.attn_norm, (const __nv_bfloat16*)s.wqkv,
+                              (const __nv_bfloat16*)s.q_norm, (const __nv_bfloat16*)s.k_norm,
+                              (const __nv_bfloat16*)s.wo, (const __nv_bfloat16*)s.mlp_norm,
+                              (const __nv_bfloat16*)s.router, (const __nv_bfloat16*)s.w_gate_up,
+                              (const __nv_bfloat16*)s.w_down};
+    }
+    m->embed = (const __nv_bfloat16*)w->embed;
+    m->final_norm = (const __nv_bfloat16*)w->final_norm;
+    m->lm_head = (const __nv_bfloat16*)w->lm_head;
+    m->device = dev;
+    m->sm_count = sms;
+    m->max_decode = max_decode_seqs;
+    m->max_prefill = max_prefill_tokens;
+    m->next_slot = 0;
+    m->last_stream = nullptr;
+    std::memset(&m->info, 0, sizeof(m->info));
+    for (int i = 0; i < kStagingSlots; ++i) { m->staging[i] = nullptr; m->staged[i] = nullptr; }
+    auto fail = [&](cudaError_t e) {
+        g_last_cuda_error = (int32_t)e;
+        mars_model_free(m);
+        return MARS_ERR_CUDA;
+    };
+    for (int i = 0; i < kStagingSlots; ++i) {
+        cudaError_t e = cudaHostAlloc((void**)&m->staging[i], (size_t)lay.total_words * 4, cudaHostAllocDefault);
+        if (e != cudaSuccess) return fail(e);
+        e = cudaEventCreateWithFlags(&m->staged[i], cudaEventDisableTiming);
+        if (e != cudaSuccess) return fail(e);
+    }
+    // rotary frequencies theta^(-2i/D) in fp64, status word cleared
+    std::vector<double> inv((size_t)cfg->head_dim / 2);
+    for (int i = 0; i < cfg->head_dim / 2; ++i)
+        inv[i] = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)cfg->head_dim);
+    cudaError_t e = cudaMemcpy(m->buf.inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return fail(e);
+    e = cudaMemset(m->buf.err, 0, 256);
+    if (e != cudaSuccess) return fail(e);
+    e = cudaMemset(m->buf.active, 0, (size_t)cfg->n_layers * 4);
+    if (e != cudaSuccess) return fail(e);
+    *out = m;
+    return MARS_OK;
+}
+
+mars_status_t mars_model_free(mars_model_t* m) {
+    if (!m) return MARS_ERR_BAD_HANDLE;
+    for (int i = 0; i < kStagingSlots; ++i) {
+        if (m->staged[i]) cudaEventDestroy(m->staged[i]);
+        if (m->staging[i]) cudaFreeHost(m->staging[i]);
+    }
+    delete m;
+    return MARS_OK;
+}
+
+// ------------------------------------------------------------------------------- paged KV cache
+
+size_t mars_kv_meta_bytes(int32_t max_seqs, int32_t max_pages_per_seq) {
+    if (max_seqs < 1 || max_pages_per_seq < 1) return 0;
+    return align_up((size_t)max_seqs * max_pages_per_seq * 4, 256);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static mars_status_t make_pool_map(CUtensorMap* tm, void* pool, uint64_t rows, int D, int box_rows) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return MARS_ERR_UNSUPPORTED;
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = ((EncodeTiledFn)fn)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pool, dims, strides, box, estr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_last_cuda_error = (int32_t)r;
+        return MARS_ERR_CUDA;
+    }
+    return MARS_OK;
+}
+
+mars_status_t mars_kv_alloc(mars_model_t* m, void* k_pool, void* v_pool, size_t pool_bytes_each, int32_t page_size,
+                            int32_t max_seqs, int32_t max_pages_per_seq, void* meta, size_t meta_bytes, mars_kv_t** out) {
+    if (!m) return MARS_ERR_BAD_HANDLE;
+    if (!k_pool || !v_pool || !meta || !out || max_seqs < 1 || max_pages_per_seq < 1) return MARS_ERR_INVALID_ARG;
+    if (page_size != 16 && page_size != 32 && page_size != 64 && page_size != 128) return MARS_ERR_INVALID_ARG;
+    if ((uintptr_t)k_pool % 256 || (uintptr_t)v_pool % 256 || (uintptr_t)meta % 256) return MARS_ERR_INVALID_ARG;
+    if (meta_bytes < mars_kv_meta_bytes(max_seqs, max_pages_per_seq)) return MARS_ERR_INVALID_ARG;
+    const mars_config_t& c = m->cfg;
+    const size_t page_bytes = (size_t)c.n_kv_heads * page_size * c.head_dim * 2;
+    const size_t n_pages = pool_bytes_each / page_bytes / c.n_layers;
+    if (n_pages < 1 || n_pages > 0x3fffffff) return MARS_ERR_INVALID_ARG;
+    const uint64_t rows = (uint64_t)c.n_layers * n_pages * c.n_kv_heads * page_size;
+    if (rows > 0x7fffffffull) return MARS_ERR_UNSUPPORTED;
+    mars_kv* kv = new (std::nothrow) mars_kv();
+    if (!kv) return MARS_ERR_INVALID_ARG;
+    kv->model = m;
+    kv->view = KvView{(__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, (int32_t*)meta, (int)n_pages, page_size,
+                      max_pages_per_seq};
+    kv->max_seqs = max_seqs;
+    const int box_rows = std::min(page_size, 64);
+    mars_status_t st = make_pool_map(&kv->tm_k, k_pool, rows, c.head_dim, box_rows);
+    if (st == MARS_OK) st = make_pool_map(&kv->tm_v, v_pool, rows, c.head_dim, box_rows);
+    if (st != MARS_OK) { delete kv; return st; }
+    cudaError_t e = cudaMemset(meta, 0, mars_kv_meta_bytes(max_seqs, max_pages_per_seq));
+    if (e != cudaSuccess) { g_last_cuda_error = (int32_t)e; delete kv; return MARS_ERR_CUDA; }
+    kv->seqs.resize(max_seqs);
+    kv->owned.assign(n_pages, 0);
+    kv->free_list.resize(n_pages);
+    for (size_t i = 0; i < n_pages; ++i) kv->free_list[i] = (int32_t)(n_pages - 1 - i);   // page 0 is handed out first
+    *out = kv;
+    return MARS_OK;
+}
+
+mars_status_t mars_kv_free(mars_kv_t* kv) {
+    if (!kv) return MARS_ERR_BAD_HANDLE;
+    delete kv;
+    return MARS_OK;
+}
+
+int32_t mars_kv_num_pages(const mars_kv_t* kv) { return kv ? kv->view.n_pages : -1; }
+int32_t mars_kv_free_pages(const mars_kv_t* kv) { return kv ? (int32_t)kv->free_list.size() : -1; }
+
+static mars_status_t upload_row(mars_kv* kv, int seq, int first, int count) {
+    if (count <= 0) return MARS_OK;
+    CUDA_TRY(cudaMemcpy(kv->view.block_table + (size_t)seq * kv->view.max_pages_per_seq + first,
+                        kv->seqs[seq].pages.data() + first, (size_t)count * 4, cudaMemcpyHostToDevice));
+    return MARS_OK;
+}
+
+mars_status_t mars_kv_seq_reserve(mars_kv_t* kv, int32_t seq, int32_t n_tokens_total) {
+    if (!kv || seq < 0 || seq >= kv->max_seqs) return MARS_ERR_BAD_HANDLE;
+    if (n_tokens_total < 0 || n_tokens_total > kv->model->cfg.max_pos) return MARS_ERR_INVALID_ARG;
+    SeqState& s = kv->seqs[seq];
+    const int ps = kv->view.page_size;
+    const int need = (n_tokens_total + ps - 1) / ps;
+    const int have = (int)s.pages.size();
+    if (need > kv->view.max_pages_per_seq) return MARS_ERR_KV_FULL;
+    if (need - have > (int)kv->free_list.size()) return MARS_ERR_KV_FULL;
+    for (int i = have; i < need; ++i) {
+        const int32_t p = kv->free_list.back();
+        kv->free_list.pop_back();
+        kv->owned[p] = 1;
+        s.pages.push_back(p);
+    }
+    s.used = true;
+    return upload_row(kv, seq, have, need - have);
+}
+
+mars_status_t mars_kv_seq_adopt(mars_kv_t* kv, int32_t seq, const int32_t* pages, int32_t n_pages, int32_t ctx_len) {
+    if (!kv || seq < 0 || seq >= kv->max_seqs) return MARS_ERR_BAD_HANDLE;
+    if (!pages || n_pages < 0 || ctx_len < 0) return MARS_ERR_INVALID_ARG;
+    if (n_pages > kv->view.max_pages_per_seq || (int64_t)ctx_len > (int64_t)n_pages * kv->view.page_size)
+        return MARS_ERR_INVALID_ARG;
+    SeqState& s = kv->seqs[seq];
+    if (s.used) return MARS_ERR_BAD_HANDLE;
+    std::vector<int32_t> sorted(pages, pages + n_pages);
+    std::sort(sorted.begin(), sorted.end());
+    for (int i = 0; i < n_pages; ++i) {
+        if (sorted[i] < 0 || sorted[i] >= kv->view.n_pages) return MARS_ERR_INVALID_ARG;
+        if (kv->owned[sorted[i]] || (i > 0 && sorted[i] == sorted[i - 1])) return MARS_ERR_BAD_HANDLE;
+    }
+    for (int i = 0; i < n_pages; ++i) kv->owned[pages[i]] = 1;
+    kv->free_list.erase(std::remove_if(kv->free_list.begin(), kv->free_list.end(),
+                                       [&](int32_t p) { return std::binary_search(sorted.begin(), sorted.end(), p); }),
+                        kv->free_list.end());
+    s.pages.assign(pages, pages + n_pages);
+    s.len = ctx_len;
+    s.used = true;
+    return upload_row(kv, seq, 0, n_pages);
+}
+
+mars_status_t mars_kv_seq_set_len(mars_kv_t* kv, int32_t seq, int32_t ctx_len) {
+    if (!kv || seq < 0 || seq >= kv->max_seqs || !kv->seqs[seq].used) return MARS_ERR_BAD_HANDLE;
+    if (ctx_len < 0 || (int64_t)ctx_len > (int64_t)kv->seqs[seq].pages.size() * kv->view.page_size)
+        return MARS_ERR_INVALID_ARG;
+    kv->seqs[seq].len = ctx_len;
+    return MARS_OK;
+}
+
+mars_status_t mars_kv_seq_release(mars_kv_t* kv, int32_t seq) {
+    if (!kv || seq < 0 || seq >= kv->max_seqs || !kv->seqs[seq].used) return MARS_ERR_BAD_HANDLE;
+    SeqState& s = kv->seqs[seq];
+    for (auto it = s.pages.rbegin(); it != s.pages.rend(); ++it) {
+        kv->owned[*it] = 0;
+        kv->free_list.push_back(*it);
+    }
+    s = SeqState();
+    return MARS_OK;
+}
+
+int32_t mars_kv_seq_len(const mars_kv_t* kv, int32_t seq) {
+    if (!kv || seq < 0 || seq >= kv->max_seqs || !kv->seqs[seq].used) return -1;
+    return kv->seqs[seq].len;
+}
+
+mars_status_t mars_kv_block_table(const mars_kv_t* kv, int32_t seq, int32_t* pages_out, int32_t cap, int32_t* n) {
+    if (!kv || seq < 0 || seq >= kv->max_seqs || !kv->seqs[seq].used) return MARS_ERR_BAD_HANDLE;
+    if (!n || cap < 0 || (cap > 0 && !pages_out)) return MARS_ERR_INVALID_ARG;
+    const auto& p = kv->seqs[seq].pages;
+    *n = (int32_t)p.size();
+    for (int i = 0; i < std::min<int>(cap, (int)p.size()); ++i) pages_out[i] = p[i];
+    return MARS_OK;
+}
+
+// ------------------------------------------------------------------------------------- the step
+
+namespace {
+
+struct StepPlan {
+    std::vector<int32_t> tok_seq, tok_pos, emit_rows, emit_slot, updates;
+    const int32_t* tokens_dev;
+    int span;   // cached tokens per attention item
+};
+
+mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPlan& plan, const mars_sampling_t& smp,
+                       int32_t* out_tokens, float* out_logprobs, const mars_debug_t* dbg) {
+    const int n_tok = (int)plan.tok_seq.size();
+    const int n_emit = (int)plan.emit_rows.size();
+    const StepLayout& lay = m->lay;
+
+    // attention work items: spans of `span` cached tokens per token row (widened until they fit)
+    int span = plan.span;
+    int64_t n_items = 0;
+    for (;;) {
+        n_items = 0;
+        for (int t = 0; t < n_tok; ++t) n_items += ((int64_t)plan.tok_pos[t] + 1 + span - 1) / span;
+        if (n_items <= m->caps.n_items) break;
+        if (span > (1 << 28)) return MARS_ERR_INVALID_ARG;
+        span *= 2;
+    }
+
+    const int slot = m->next_slot;
+    m->next_slot = (slot + 1) % kStagingSlots;
+    CUDA_TRY(cudaEventSynchronize(m->staged[slot]));
+    int32_t* blk = m->staging[slot];
+    std::memset(blk, 0, H_WORDS * 4);
+    blk[H_NTOK] = n_tok;
+    blk[H_NITEMS] = (int32_t)n_items;
+    blk[H_NUPDATES] = (int32_t)(plan.updates.size() / 3);
+    blk[H_NEMIT] = n_emit;
+    blk[H_GREEDY] = smp.greedy ? 1 : 0;
+    std::memcpy(&blk[H_TEMPERATURE], &smp.temperature, 4);
+    std::memcpy(&blk[H_TOP_P], &smp.top_p, 4);
+    blk[H_SEED_LO] = (int32_t)(uint32_t)smp.seed;
+    blk[H_SEED_HI] = (int32_t)(uint32_t)(smp.seed >> 32);
+    blk[H_STEP_LO] = (int32_t)(uint32_t)smp.step;
+    blk[H_STEP_HI] = (int32_t)(uint32_t)(smp.step >> 32);
+    std::memcpy(blk + lay.tok_seq, plan.tok_seq.data(), (size_t)n_tok * 4);
+    std::memcpy(blk + lay.tok_pos, plan.tok_pos.data(), (size_t)n_tok * 4);
+    if (n_emit) {
+        std::memcpy(blk + lay.emit_rows, plan.emit_rows.data(), (size_t)n_emit * 4);
+        std::memcpy(blk + lay.emit_slot, plan.emit_slot.data(), (size_t)n_emit * 4);
+    }
+    if (!plan.updates.empty()) std::memcpy(blk + lay.updates, plan.updates.data(), plan.updates.size() * 4);
+    int64_t kv_tokens = 0;
+    {
+        int32_t* items = blk + lay.items;
+        int32_t* off = blk + lay.tok_item_off;
+        int at = 0;
+        for (int t = 0; t < n_tok; ++t) {
+            off[t] = at;
+            const int len = plan.tok_pos[t] + 1;
+            kv_tokens += len;
+            for (int s0 = 0; s0 < len; s0 += span) {
+                items[4 * at + 0] = t;
+                items[4 * at + 1] = s0;
+                items[4 * at + 2] = std::min(span, len - s0);
+                items[4 * at + 3] = 0;
+                ++at;
+            }
+        }
+        off[n_tok] = at;
+    }
+    // one copy uploads the whole block up to the last item
+    const size_t used_words = (size_t)lay.items + 4 * (size_t)n_items;
+    CUDA_TRY(cudaMemcpyAsync(m->buf.step, blk, used_words * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaEventRecord(m->staged[slot], st));
+
+    const Shape& s = m->shape;
+    const Buffers& b = m->buf;
+    DebugTaps taps{nullptr, nullptr, nullptr, nullptr, nullptr};
+    if (dbg) taps = DebugTaps{dbg->hidden, dbg->router_w, dbg->router_idx, dbg->forced_idx, dbg->nucleus_mass};
+    const size_t hid_stride = (size_t)n_tok * s.H;
+
+    int launches = 0;
+    launches += launch_prep(s, b, lay, kv->view, n_tok, st);
+    launches += launch_embed(s, b, lay, m->embed, plan.tokens_dev, m->layers[0].attn_norm, taps.hidden, n_tok, st);
+    for (int l = 0; l < s.L; ++l) {
+        const LayerW& w = m->layers[l];
+        launches += launch_qkv(s, b, lay, w, kv->view, l, n_tok, st);
+        launches += launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, n_tok, (int)n_items, m->sm_count, st);
+        launches += launch_oproj(s, b, w, n_tok, st);
+        launches += launch_router(s, b, w, taps, l, n_tok, st);
+        launches += launch_experts(s, b, w, n_tok, st);
+        const __nv_bfloat16* next_gain = l + 1 < s.L ? m->layers[l + 1].attn_norm : m->final_norm;
+        launches += launch_combine(s, b, next_gain, taps.hidden ? taps.hidden + (size_t)(l + 1) * hid_stride : nullptr,
+                                   n_tok, st);
+    }
+    if (n_emit) {
+        launches += launch_lm_head(s, b, lay, m->lm_head, n_emit, st);
+        if (dbg && dbg->logits)
+            CUDA_TRY(cudaMemcpyAsync(dbg->logits, b.logits, (size_t)n_emit * s.V * 4, cudaMemcpyDeviceToDevice, st));
+        launches += launch_sample(s, b, lay, n_emit, out_tokens, out_logprobs, taps.nucleus_mass, st);
+    }
+    CUDA_TRY(cudaGetLastError());
+    m->last_stream = st;
+    m->info.kernel_launches = launches;
+    m->info.attn_items = n_items;
+    m->info.kv_tokens_read = kv_tokens;
+    return MARS_OK;
+}
+
+}  // namespace
+
+mars_status_t mars_decode_step(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_seqs, const int32_t* seq_ids,
+                               const int32_t* in_tokens, const mars_sampling_t* sampling, int32_t* out_tokens,
+                               float* out_logprobs, const mars_debug_t* debug) {
+    if (!m || !kv || kv->model != m) return MARS_ERR_BAD_HANDLE;
+    if (!seq_ids || !in_tokens || !sampling || !out_tokens || !out_logprobs) return MARS_ERR_INVALID_ARG;
+    if (n_seqs < 1 || n_seqs > m->max_decode) return MARS_ERR_INVALID_ARG;
+    if (!sampling->greedy && (!(sampling->temperature > 0.f) || !(sampling->top_p > 0.f) || sampling->top_p > 1.f))
+        return MARS_ERR_INVALID_ARG;
+    const int ps = kv->view.page_size;
+    StepPlan plan;
+    plan.tokens_dev = in_tokens;
+    plan.span = kSpanTokens;
+    std::vector<uint8_t> seen(kv->max_seqs, 0);
+    int new_pages = 0;
+    for (int i = 0; i < n_seqs; ++i) {
+        const int sq = seq_ids[i];
+        if (sq < 0 || sq >= kv->max_seqs || !kv->seqs[sq].used || seen[sq]) return MARS_ERR_BAD_HANDLE;
+        seen[sq] = 1;
+        const SeqState& s = kv->seqs[sq];
+        if (s.len + 1 > m->cfg.max_pos) return MARS_ERR_INVALID_ARG;
+        if (s.len / ps >= (int)s.pages.size()) {
+            if ((int)s.pages.size() + 1 > kv->view.max_pages_per_seq) return MARS_ERR_KV_FULL;
+            ++new_pages;
+        }
+    }
+    if (new_pages > (int)kv->free_list.size()) return MARS_ERR_KV_FULL;
+    // nothing can fail on the host from here on except CUDA calls
+    std::vector<std::pair<int, int32_t>> taken;
+    for (int i = 0; i < n_seqs; ++i) {
+        const int sq = seq_ids[i];
+        SeqState& s = kv->seqs[sq];
+        if (s.len / ps >= (int)s.pages.size()) {
+            const int32_t p = kv->free_list.back();
+            kv->free_list.pop_back();
+            kv->owned[p] = 1;
+            plan.updates.push_back(sq);
+            plan.updates.push_back((int32_t)s.pages.size());
+            plan.updates.push_back(p);
+            s.pages.push_back(p);
+            taken.emplace_back(sq, p);
+        }
+        plan.tok_seq.push_back(sq);
+        plan.tok_pos.push_back(s.len);
+        plan.emit_rows.push_back(i);
+        plan.emit_slot.push_back(sq);
+    }
+    mars_status_t r = run_step(m, kv, (cudaStream_t)cuda_stream, plan, *sampling, out_tokens, out_logprobs, debug);
+    if (r != MARS_OK) {
+        for (auto it = taken.rbegin(); it != taken.rend(); ++it) {   // undo the page grabs
+            kv->seqs[it->first].pages.pop_back();
+            kv->owned[it->second] = 0;
+            kv->free_list.push_back(it->second);
+        }
+        return r;
+    }
+    for (int i = 0; i < n_seqs; ++i) kv->seqs[seq_ids[i]].len += 1;
+    return MARS_OK;
+}
+
+mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_reqs,
+                                 const int32_t* seq_ids, const int32_t* chunk_lens, const int32_t* tokens,
+                                 const int32_t* emit_last, const mars_sampling_t* sampling, int32_t* out_tokens,
+                                 float* out_logprobs, const mars_debug_t* debug) {
+    if (!m || !kv || kv->model != m) return MARS_ERR_BAD_HANDLE;
+    if (!seq_ids || !chunk_lens || !tokens || !sampling || n_reqs < 1) return MARS_ERR_INVALID_ARG;
+    if (!sampling->greedy && (!(sampling->temperature > 0.f) || !(sampling->top_p > 0.f) || sampling->top_p > 1.f))
+        return MARS_ERR_INVALID_ARG;
+    const int ps = kv->view.page_size;
+    int64_t total = 0, new_pages = 0;
+    int n_emit = 0;
+    std::vector<uint8_t> seen(kv->max_seqs, 0);
+    for (int r = 0; r < n_reqs; ++r) {
+        const int sq = seq_ids[r];
+        if (sq < 0 || sq >= kv->max_seqs || !kv->seqs[sq].used || seen[sq]) return MARS_ERR_BAD_HANDLE;
+        seen[sq] = 1;
+        if (chunk_lens[r] < 1) return MARS_ERR_INVALID_ARG;
+        const SeqState& s = kv->seqs[sq];
+        const int64_t end = (int64_t)s.len + chunk_lens[r];
+        if (end > m->cfg.max_pos) return MARS_ERR_INVALID_ARG;
+        const int64_t need = (end + ps - 1) / ps;
+        if (need > kv->view.max_pages_per_seq) return MARS_ERR_KV_FULL;
+        new_pages += std::max<int64_t>(0, need - (int64_t)s.pages.size());
+        total += chunk_lens[r];
+        if (emit_last && emit_last[r]) ++n_emit;
+    }
+    if (total > m->max_prefill) return MARS_ERR_INVALID_ARG;
+    if (n_emit > m->caps.n_emit) return MARS_ERR_INVALID_ARG;
+    if (n_emit && (!out_tokens || !out_logprobs)) return MARS_ERR_INVALID_ARG;
+    if (new_pages > (int64_t)kv->free_list.size()) return MARS_ERR_KV_FULL;
+
+    StepPlan plan;
+    plan.tokens_dev = tokens;
+    plan.span = 1 << 30;   // one work item per token row
+    std::vector<std::pair<int, int32_t>> taken;
+    int row = 0;
+    for (int r = 0; r < n_reqs; ++r) {
+        const int sq = seq_ids[r];
+        SeqState& s = kv->seqs[sq];
+        const int end = s.len + chunk_lens[r];
+        const int need = (end + ps - 1) / ps;
+        while ((int)s.pages.size() < need) {
+            const int32_t p = kv->free_list.back();
+            kv->free_list.pop_back();
+            kv->owned[p] = 1;
+            plan.updates.push_back(sq);
+            plan.updates.push_back((int32_t)s.pages.size());
+            plan.updates.push_back(p);
+            s.pages.push_back(p);
+            taken.emplace_back(sq, p);
+        }
+        for (int i = 0; i < chunk_lens[r]; ++i) {
+            plan.tok_seq.push_back(sq);
+            plan.tok_pos.push_back(s.len + i);
+        }
+        row += chunk_lens[r];
+        if (emit_last && emit_last[r]) {
+            plan.emit_rows.push_back(row - 1);
+            plan.emit_slot.push_back(sq);
+        }
+    }
+    mars_status_t st = run_step(m, kv, (cudaStream_t)cuda_stream, plan, *sampling, out_tokens, out_logprobs, debug);
+    if (st != MARS_OK) {
+        for (auto it = taken.rbegin(); it != taken.rend(); ++it) {
+            kv->seqs[it->first].pages.pop_back();
+            kv->owned[it->second] = 0;
+            kv->free_list.push_back(it->second);
+        }
+        return st;
+    }
+    for (int r = 0; r < n_reqs; ++r) kv->seqs[seq_ids[r]].len += chunk_lens[r];
+    return MARS_OK;
+}
+
+mars_status_t mars_decode_step_host(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_seqs,
+                                    const int32_t* seq_ids, const int32_t* in_tokens_host,
+                                    const mars_sampling_t* sampling, int32_t* out_tokens_host, float* out_logprobs_host) {
+    if (!m || !kv) return MARS_ERR_BAD_HANDLE;
+    if (!in_tokens_host || !out_tokens_host || !out_logprobs_host || n_seqs < 1 || n_seqs > m->max_decode)
+        return MARS_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CUDA_TRY(cudaMemcpyAsync(m->io_in, in_tokens_host, (size_t)n_seqs * 4, cudaMemcpyHostToDevice, st));
+    mars_status_t r = mars_decode_step(m, kv, cuda_stream, n_seqs, seq_ids, m->io_in, sampling, m->io_out, m->io_lp,
+                                       nullptr);
+    if (r != MARS_OK) return r;
+    CUDA_TRY(cudaMemcpyAsync(out_tokens_host, m->io_out, (size_t)n_seqs * 4, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaMemcpyAsync(out_logprobs_host, m->io_lp, (size_t)n_seqs * 4, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return MARS_OK;
+}
+
+mars_status_t mars_poll_status(mars_model_t* m) {
+    if (!m) return MARS_ERR_BAD_HANDLE;
+    CUDA_TRY(cudaStreamSynchronize(m->last_stream));
+    int32_t word = 0;
+    CUDA_TRY(cudaMemcpy(&word, m->buf.err, 4, cudaMemcpyDeviceToHost));
+    if (word) CUDA_TRY(cudaMemset(m->buf.err, 0, 4));
+    if (word & kErrTimeout) return MARS_ERR_TIMEOUT;
+    if (word & kErrBadToken) return MARS_ERR_BAD_TOKEN;
+    return MARS_OK;
+}
+
+mars_status_t mars_last_step_info(const mars_model_t* m, mars_step_info_t* out) {
+    if (!m) return MARS_ERR_BAD_HANDLE;
+    if (!out) return MARS_ERR_INVALID_ARG;
+    *out = m->info;
+    return MARS_OK;
+}
+
+const int32_t* mars_active_experts_device(const mars_model_t* m) { return m ? m->buf.active : nullptr; }
+
+}  // extern "C"

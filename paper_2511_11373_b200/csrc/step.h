@@ -1,0 +1,68 @@
+// Host/device description of one step: the model shape, the workspace carve-up and the per-step
+// metadata block that the host builds in pinned memory and uploads with a single copy.
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace mars {
+
+// Bits of the device status word (read and cleared by mars_poll_status).
+constexpr int kErrBadToken = 1;
+constexpr int kErrTimeout = 2;
+
+// Header words of the step block (int32 each).
+enum StepHdr {
+    H_NTOK = 0,       // token rows in this call
+    H_NITEMS = 1,     // attention work items
+    H_NUPDATES = 2,   // block-table entries to write before the step
+    H_NEMIT = 3,      // rows that sample a token
+    H_GREEDY = 4,
+    H_TEMPERATURE = 5,  // float bits
+    H_TOP_P = 6,        // float bits
+    H_SEED_LO = 7, H_SEED_HI = 8, H_STEP_LO = 9, H_STEP_HI = 10,
+    H_WORDS = 16
+};
+
+// Offsets (in int32 words) of the arrays inside the step block.
+struct StepLayout {
+    int tok_seq;       // [n_tok] sequence slot (block-table row) of every token row
+    int tok_pos;       // [n_tok] position of the token in its sequence
+    int tok_item_off;  // [n_tok + 1] first attention item of every token row
+    int emit_rows;     // [n_emit] token row whose hidden state is sampled
+    int emit_slot;     // [n_emit] sequence slot of that row (random-number counter)
+    int updates;       // [n_updates][3] (slot, page index, page id)
+    int items;         // [n_items][4] (token row, first cached token, number of tokens, 0)
+    int total_words;
+};
+
+struct Shape {
+    int L, H, nq, nkv, D, E, k, I, V, qk_norm;
+    float eps;
+};
+
+// Everything the kernels need to find their buffers.  All pointers are device pointers into the
+// caller's workspace unless noted.
+struct Buffers {
+    int32_t* step;          // the uploaded step block
+    int32_t* err;           // status word
+    float* x;               // [n_tok, H] residual stream (fp32)
+    __nv_bfloat16* h;       // [n_tok, H] normalised input of the next projection
+    float* qkv;             // [n_tok, (nq + 2 nkv) D] raw projection
+    __nv_bfloat16* q;       // [n_tok, nq D] rotated queries
+    __nv_bfloat16* o;       // [n_tok, nq D] attention output
+    float2* rope;           // [n_tok, D/2] (cos, sin) of pos * theta_i
+    double* inv_freq;       // [D/2] theta^(-2i/D)
+    float* part_o;          // [items, nq, D] unnormalised partial outputs
+    float2* part_ml;        // [items, nq] (running max in log2 units, sum)
+    int32_t* route_idx;     // [n_tok, k]
+    float* route_w;         // [n_tok, k]
+    int32_t* expert_off;    // [E + 1]
+    int32_t* slot_token;    // [n_tok k] token row served by every expert slot
+    int32_t* slot_of;       // [n_tok k] slot of (token, j)
+    int32_t* active;        // [L] distinct experts per layer
+    __nv_bfloat16* act;     // [n_tok k, I]
+    float* y;               // [n_tok k, H]
+    float* logits;          // [n_emit, V]
+};
+
+}  // namespace mars

@@ -1,0 +1,189 @@
+"""GPU-vs-oracle harness for the parity tests: builds one seeded case, runs the CUDA library through
+its C ABI, runs the CPU oracle on copies of the same bytes, and compares with the cascade rule.
+
+Tolerances (from the target this repository is built to):
+  routing indices exact wherever the oracle's fp32 gate margin (pi_k - pi_{k+1}) is >= 1e-3;
+  greedy tokens exact wherever the oracle's top-2 logit gap is >= 1e-2;
+  logits and log-probs within 2e-2 absolute; hidden states within 1e-2 relative L2 per token.
+"""
+from __future__ import annotations
+
+import torch
+
+import oracle
+from paper_2511_11373_b200 import binding, workloads as wl
+
+TOL_ROUTE_MARGIN = 1e-3
+TOL_LOGIT_GAP = 1e-2
+TOL_LOGIT_ABS = 2e-2
+TOL_HIDDEN_REL = 1e-2
+TOL_ROUTER_W = 2e-3
+
+
+class Case:
+    def __init__(self, model: dict, page_size: int, ctx, seed: int = 0, gains: str = "perturbed", headroom: int = 1,
+                 spare_pages: int = 3, poison: bool = True, max_prefill_tokens: int = 0, device: str = "cuda",
+                 max_decode: int | None = None, extra_seqs: int = 0):
+        self.model_shape, self.ps, self.ctx, self.seed = dict(model), page_size, list(ctx), seed
+        self.device = torch.device(device)
+        B = len(ctx)
+        self.B = B
+        cap = [c + headroom for c in ctx]
+        need = sum(wl.pages_needed(c, page_size) for c in cap)
+        self.n_pages = need + spare_pages
+        self.max_pages = max(wl.pages_needed(c, page_size) for c in cap) + 1
+        self.pages = wl.make_page_assignment(cap, page_size, self.n_pages, seed=seed)
+        self.weights = wl.make_weights(model, seed=seed, device=self.device, gains=gains)
+        self.k_pool, self.v_pool = wl.make_kv_pools(model, self.n_pages, page_size, seed=seed, device=self.device)
+        if poison:
+            self._poison_unused()
+        self.max_pos = max(cap) + max_prefill_tokens + 8
+        self.model = binding.Model(model, self.weights, max_decode_seqs=max_decode or B,
+                                   max_prefill_tokens=max_prefill_tokens, max_pos=self.max_pos)
+        self.kv = binding.KvCache(self.model, self.k_pool, self.v_pool, page_size, B + extra_seqs, self.max_pages)
+        for b in range(B):
+            self.kv.seq_adopt(b, self.pages[b], ctx[b])
+        # oracle side: CPU copies of the same bytes
+        self.w_cpu = wl.weights_to_cpu(self.weights)
+        self.k_cpu, self.v_cpu = self.k_pool.cpu(), self.v_pool.cpu()
+        self.bt = wl.block_table_tensor(self.pages, self.max_pages)
+        self.ocfg = oracle.Config(**model)
+        self.cur = list(ctx)
+
+    def _poison_unused(self):
+        """NaN in every cache slot that no sequence owns (beyond the context inside owned pages, and
+        every unowned page): a read past the end of a context shows up as NaN in the comparison."""
+        nan = float("nan")
+        owned = torch.zeros(self.n_pages, dtype=torch.bool)
+        for b, pg in enumerate(self.pages):
+            owned[torch.tensor(pg, dtype=torch.long)] = True
+            c = self.ctx[b]
+            last, used = c // self.ps, c % self.ps
+            for i, p in enumerate(pg):
+                if i > last:
+                    self.k_pool[:, p] = nan; self.v_pool[:, p] = nan
+                elif i == last:
+                    self.k_pool[:, p, :, used:] = nan; self.v_pool[:, p, :, used:] = nan
+        free = (~owned).nonzero().flatten().to(self.device)
+        if free.numel():
+            self.k_pool[:, free] = nan; self.v_pool[:, free] = nan
+
+    # ------------------------------------------------------------------ CUDA side
+    def gpu_decode(self, tokens: torch.Tensor, sampling: dict, forced_idx=None, seq_ids=None, step: int = 0,
+                   seed: int = 0):
+        m, dev = self.model_shape, self.device
+        ids = list(range(self.B)) if seq_ids is None else list(seq_ids)
+        n = len(ids)
+        L, H, k, V = m["n_layers"], m["hidden"], m["top_k"], m["vocab"]
+        out = dict(tokens=torch.empty(n, dtype=torch.int32, device=dev), logp=torch.empty(n, dtype=torch.float32, device=dev),
+                   logits=torch.empty(n, V, dtype=torch.float32, device=dev),
+                   hidden=torch.empty(L + 1, n, H, dtype=torch.float32, device=dev),
+                   router_w=torch.empty(L, n, k, dtype=torch.float32, device=dev),
+                   router_idx=torch.empty(L, n, k, dtype=torch.int32, device=dev),
+                   nucleus_mass=torch.empty(n, dtype=torch.float32, device=dev))
+        f = None if forced_idx is None else forced_idx.to(dev).contiguous()
+        dbg = binding.make_debug(out["logits"], out["hidden"], out["router_w"], out["router_idx"], f, out["nucleus_mass"])
+        smp = binding.make_sampling(seed=seed, step=step, **sampling)
+        st = binding.mars_decode_step(self.model, self.kv, ids, tokens.to(dev), smp, out["tokens"], out["logp"], dbg)
+        assert st == 0, binding.STATUS_NAMES.get(st, st)
+        assert self.model.poll_status() == 0
+        return {k_: v.cpu() for k_, v in out.items()}
+
+    # ------------------------------------------------------------------ oracle side
+    def oracle_decode(self, tokens: torch.Tensor, forced_idx=None, seq_ids=None):
+        ids = list(range(self.B)) if seq_ids is None else list(seq_ids)
+        seq = torch.tensor(ids, dtype=torch.int32)
+        pos = torch.tensor([self.cur[b] for b in ids], dtype=torch.int32)
+        res = oracle.forward(self.ocfg, self.w_cpu, tokens.to(torch.int32).cpu().contiguous(), seq, pos, self.k_cpu,
+                             self.v_cpu, self.bt, self.ps, forced_idx=forced_idx)
+        for b in ids:
+            self.cur[b] += 1
+        return res
+
+
+def topk_margin(probs: torch.Tensor, k: int) -> torch.Tensor:
+    """pi_k - pi_{k+1} of the sorted probabilities (inf when k == E)."""
+    s = torch.sort(probs.double(), dim=-1, descending=True).values
+    if s.shape[-1] == k:
+        return torch.full(s.shape[:-1], float("inf"), dtype=torch.float64)
+    return s[..., k - 1] - s[..., k]
+
+
+def compare_step(gpu: dict, orc: dict, k: int, greedy: bool, label: str = "") -> dict:
+    """`orc` is the oracle run with the GPU's routing forced (cascade rule): wherever the oracle's own
+    margin is >= 1e-3 its own top-k set must equal the GPU's; everything else is compared directly."""
+    stats = {}
+    probs = orc["router_probs"]                          # [L, n, E]
+    L, n, E = probs.shape
+    margin = topk_margin(probs, k)
+    own = torch.topk(probs.double(), k, dim=-1).indices
+    bad = 0
+    for l in range(L):
+        for t in range(n):
+            if margin[l, t] >= TOL_ROUTE_MARGIN:
+                if set(own[l, t].tolist()) != set(gpu["router_idx"][l, t].tolist()):
+                    bad += 1
+    stats["routing_checked"] = int((margin >= TOL_ROUTE_MARGIN).sum())
+    stats["routing_total"] = L * n
+    assert bad == 0, f"{label}: {bad} routing decisions differ where the oracle margin >= {TOL_ROUTE_MARGIN}"
+    # weights: compare per expert index (order of near-equal entries may differ)
+    gi, gw = gpu["router_idx"].long(), gpu["router_w"].double()
+    oi, ow = orc["router_idx"].long(), orc["router_w"].double()
+    dense_g = torch.zeros(L, n, E, dtype=torch.float64).scatter_(-1, gi, gw)
+    dense_o = torch.zeros(L, n, E, dtype=torch.float64).scatter_(-1, oi, ow)
+    stats["router_w_maxerr"] = float((dense_g - dense_o).abs().max())
+    assert stats["router_w_maxerr"] <= TOL_ROUTER_W, (label, stats)
+    assert torch.allclose(gw.sum(-1), torch.ones(L, n, dtype=torch.float64), atol=1e-5)
+    # hidden states, per token, relative L2
+    hg, ho = gpu["hidden"].double(), orc["hidden"].double()
+    assert torch.isfinite(hg).all(), f"{label}: non-finite hidden state (read past a context?)"
+    rel = (hg - ho).norm(dim=-1) / ho.norm(dim=-1).clamp_min(1e-30)
+    stats["hidden_rel_max"] = float(rel.max())
+    assert stats["hidden_rel_max"] <= TOL_HIDDEN_REL, (label, stats, rel.max(dim=-1).values.tolist())
+    # logits / log-probs
+    lg, lo = gpu["logits"].double(), orc["logits"].double()
+    stats["logit_maxerr"] = float((lg - lo).abs().max())
+    assert stats["logit_maxerr"] <= TOL_LOGIT_ABS, (label, stats)
+    if greedy:
+        top2 = torch.topk(lo, 2, dim=-1).values
+        gap = top2[:, 0] - top2[:, 1]
+        want = torch.argmax(lo, dim=-1)
+        sure = gap >= TOL_LOGIT_GAP
+        stats["greedy_checked"] = int(sure.sum())
+        assert torch.equal(gpu["tokens"].long()[sure], want[sure]), (label, "greedy tokens differ")
+        lse = torch.logsumexp(lo, -1)
+        lp_want = lo.gather(-1, gpu["tokens"].long()[:, None])[:, 0] - lse   # log-prob of the token the GPU chose
+        stats["logp_maxerr"] = float((gpu["logp"].double() - lp_want).abs().max())
+        assert stats["logp_maxerr"] <= TOL_LOGIT_ABS, (label, stats)
+    return stats
+
+
+def compare_sampled(gpu: dict, orc: dict, temperature: float, top_p: float, seed: int, step: int, slots, label=""):
+    """Nucleus sampling: the GPU's token must lie in the oracle's nucleus (or within the mass the
+    logit error can move the edge by) and the oracle's cumulative interval of that token (ascending
+    token id over the nucleus) must contain the uniform, within the shift that the measured logit
+    error allows (each probability moves by a factor of at most exp(2 max|dlogit| / T))."""
+    lg, lo = gpu["logits"].double(), orc["logits"].double()
+    err = float((lg - lo).abs().max())
+    tol = 2.0 * err / temperature * 2.0 + 1e-6
+    stats = dict(cdf_tol=tol, worst=0.0)
+    for i, slot in enumerate(slots):
+        u = oracle.uniform(seed, step, slot)
+        r = oracle.sample(orc["logits"][i].contiguous(), temperature, top_p, False, u, want_set=True)
+        pi = torch.softmax(lo[i] / temperature, 0)
+        S = r["in_nucleus"].bool()
+        t = int(gpu["tokens"][i])
+        if not S[t]:
+            # only acceptable right at the edge of the nucleus
+            edge = pi[S].min()
+            assert pi[t] >= edge * (1 - tol) - 1e-12, (label, i, "token outside the oracle nucleus")
+        cdf = torch.cumsum(torch.where(S, pi, torch.zeros_like(pi)), 0) / r["nucleus_mass"]
+        lo_t = float(cdf[t - 1]) if t > 0 else 0.0
+        hi_t = float(cdf[t]) if S[t] else lo_t
+        miss = max(lo_t - u, u - hi_t, 0.0)
+        stats["worst"] = max(stats["worst"], miss)
+        assert miss <= tol, (label, i, t, r["token"], lo_t, u, hi_t, tol)
+        lp_want = float(torch.log(pi[t]))
+        assert abs(float(gpu["logp"][i]) - lp_want) <= TOL_LOGIT_ABS, (label, i)
+        assert abs(float(gpu["nucleus_mass"][i]) - r["nucleus_mass"]) <= max(tol, 1e-4), (label, i)
+    return stats
