@@ -31,7 +31,12 @@ def check_cache_append(case: Case, ctx_before):
         for got, want in ((kg, case.k_cpu), (vg, case.v_cpu)):
             g, w = got[:, page, :, slot].float(), want[:, page, :, slot].float()
             assert torch.isfinite(g).all()
-            assert ((g - w).abs() <= 0.0079 * w.abs() + 1e-3).all(), (b, float((g - w).abs().max()))
+            # both sides round to bf16 values that differ by the projection's own error (activations
+            # are bf16 on the GPU): relative L2 per head row as for hidden states, plus an elementwise
+            # bound of one bf16 step and 2% of the row's RMS
+            rms = w.pow(2).mean(-1, keepdim=True).sqrt()
+            assert ((g - w).norm(dim=-1) <= 1e-2 * w.norm(dim=-1)).all(), (b, "row L2")
+            assert ((g - w).abs() <= 0.0079 * w.abs() + 0.02 * rms).all(), (b, float((g - w).abs().max()))
 
 
 # ------------------------------------------------------------------ config 1: tiny single layer
