@@ -18,6 +18,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&t);
 }
+// v ~= hi + lo with both parts bf16: about 16 mantissa bits survive.  Activations travel between
+// kernels as such pairs so that bf16 tensor-core contractions do not eat the error budget.
+__device__ __forceinline__ void split_bf16(float v, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(v);
+    lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
 __device__ __forceinline__ uint16_t to_bf16_bits(float v) {
     __nv_bfloat16 t = __float2bfloat16_rn(v);
     return *reinterpret_cast<uint16_t*>(&t);
@@ -85,11 +91,15 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // numbered as long as B uses the same numbering, so the B fragment of token column gid is the same
 // 16-byte slice of that token's activation row, read from shared memory.
 //
+// Activations are (hi, lo) bf16 pairs: token t occupies the two adjacent columns 2t (hi) and 2t+1
+// (lo), which land in the same thread's accumulator pair, so the epilogue adds d0 + d1 (rows gid)
+// and d2 + d3 (rows gid+8).  One 8-column tile therefore serves 4 tokens.
+//
 // MT: 16-row tiles per warp (each with its own pair of row pointers), NT: 8-token tiles, U: slices
 // whose loads are issued before the first MMA (memory-level parallelism).
 //   wrow[m][r]: pointer to W row (tile m, row gid + 8r), already offset by tig*8 elements
-//   xs: shared-memory address of activation row `gid` of token tile 0, offset by tig*16 bytes
-//   x_tile_stride: bytes between token tiles (8 rows), n_slices: K / 32
+//   xs: shared-memory address of activation row `gid` of column tile 0, offset by tig*16 bytes
+//   x_tile_stride: bytes between column tiles (8 rows), n_slices: K / 32
 template <int MT, int NT, int U>
 __device__ __forceinline__ void stream_mma(const __nv_bfloat16* const (&wrow)[MT][2], int n_slices,
                                            const unsigned char* xs, int x_tile_stride, float (&acc)[MT][NT][4]) {

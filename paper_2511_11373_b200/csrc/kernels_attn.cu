@@ -18,7 +18,7 @@ constexpr int kStageTok = 64;
 constexpr uint32_t kSpinLimit = 1u << 26;
 
 struct AttnParams {
-    const __nv_bfloat16* q;  // [n_tok, nq, D]
+    const __nv_bfloat16* q;  // [n_tok, 2, nq, D]: hi rows, lo rows
     float* part_o;           // [items, nq, D]
     float2* part_ml;         // [items, nq]
     const int32_t* step;
@@ -144,16 +144,20 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             for (int j = 0; j < pre; ++j) issue(j, gs + j);
         }
 
-        // Query fragments: head gid of the group on MMA row gid; rows >= g are zero.
-        uint32_t qa[KSTEPS][2];
+        // Query fragments.  The group has at most 8 heads, so MMA rows 0..7 carry the hi part of head
+        // gid and rows 8..15 its lo part: S = d0 + d2 (d1 + d3) costs no extra tensor work.
+        uint32_t qa[KSTEPS][4];
         {
-            const __nv_bfloat16* qrow = p.q + ((size_t)row * p.nq + hk * p.g + gid) * D;
+            const __nv_bfloat16* qhi = p.q + (size_t)row * 2 * p.nq * D + (size_t)(hk * p.g + gid) * D;
+            const __nv_bfloat16* qlo = qhi + (size_t)p.nq * D;
 #pragma unroll
             for (int ks = 0; ks < KSTEPS; ++ks) {
-                qa[ks][0] = qa[ks][1] = 0u;
+                qa[ks][0] = qa[ks][1] = qa[ks][2] = qa[ks][3] = 0u;
                 if (gid < p.g) {
-                    qa[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * tig);
-                    qa[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * tig);
+                    qa[ks][0] = *reinterpret_cast<const uint32_t*>(qhi + ks * 16 + 2 * tig);
+                    qa[ks][1] = *reinterpret_cast<const uint32_t*>(qlo + ks * 16 + 2 * tig);
+                    qa[ks][2] = *reinterpret_cast<const uint32_t*>(qhi + ks * 16 + 8 + 2 * tig);
+                    qa[ks][3] = *reinterpret_cast<const uint32_t*>(qlo + ks * 16 + 8 + 2 * tig);
                 }
             }
         }
@@ -204,8 +208,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     for (int kk = 0; kk < D / 32; ++kk) {
                         uint32_t kb[4];
                         ldmatrix_x4(kb, kbase + tile_off(kk >> 1, r, (kk & 1) * 4 + (lane >> 3)));
-                        mma_16816(sacc[nt], qa[2 * kk][0], 0u, qa[2 * kk][1], 0u, kb[0], kb[1]);
-                        mma_16816(sacc[nt], qa[2 * kk + 1][0], 0u, qa[2 * kk + 1][1], 0u, kb[2], kb[3]);
+                        mma_16816(sacc[nt], qa[2 * kk][0], qa[2 * kk][1], qa[2 * kk][2], qa[2 * kk][3], kb[0], kb[1]);
+                        mma_16816(sacc[nt], qa[2 * kk + 1][0], qa[2 * kk + 1][1], qa[2 * kk + 1][2], qa[2 * kk + 1][3],
+                                  kb[2], kb[3]);
                     }
                 }
                 // online softmax over the tokens of row gid (log2 domain)
@@ -214,7 +219,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int tl = w0 + (i >> 1) * 8 + 2 * tig + (i & 1);
-                    sv[i] = tl < n_valid ? sacc[i >> 1][i & 1] * p.scale_log2 : -INFINITY;
+                    sv[i] = tl < n_valid ? (sacc[i >> 1][i & 1] + sacc[i >> 1][2 + (i & 1)]) * p.scale_log2 : -INFINITY;
                     mx = fmaxf(mx, sv[i]);
                 }
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
@@ -226,19 +231,24 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 for (int i = 0; i < 4; ++i) pv[i] = exp2f(sv[i] - m_new);
                 l_run = l_run * alpha + (pv[0] + pv[1] + pv[2] + pv[3]);
                 m_run = m_new;
+                // P as (hi, lo) pairs: hi on rows 0..7, lo on rows 8..15 of the A operand
+                float pl[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) pl[i] = pv[i] - __bfloat162float(__float2bfloat16_rn(pv[i]));
                 const uint32_t pa0 = pack_bf16(pv[0], pv[1]), pa2 = pack_bf16(pv[2], pv[3]);
+                const uint32_t pa1 = pack_bf16(pl[0], pl[1]), pa3 = pack_bf16(pl[2], pl[3]);
                 // O = alpha O + P V
 #pragma unroll
                 for (int c = 0; c < NTILES; c += 2) {
-                    oacc[c][0] *= alpha; oacc[c][1] *= alpha;
-                    oacc[c + 1][0] *= alpha; oacc[c + 1][1] *= alpha;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { oacc[c][i] *= alpha; oacc[c + 1][i] *= alpha; }
                     const int mi = lane >> 3;
                     const int r = w0 + (mi & 1) * 8 + (lane & 7);
                     const int ch = c + (mi >> 1);
                     uint32_t vb[4];
                     ldmatrix_x4_trans(vb, vbase + tile_off(ch >> 3, r, ch & 7));
-                    mma_16816(oacc[c], pa0, 0u, pa2, 0u, vb[0], vb[1]);
-                    mma_16816(oacc[c + 1], pa0, 0u, pa2, 0u, vb[2], vb[3]);
+                    mma_16816(oacc[c], pa0, pa1, pa2, pa3, vb[0], vb[1]);
+                    mma_16816(oacc[c + 1], pa0, pa1, pa2, pa3, vb[2], vb[3]);
                 }
             }
             __syncthreads();
@@ -253,8 +263,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         float* ml = mm + kAttnWarps * 8;                            // [warps][8]
 #pragma unroll
         for (int c = 0; c < NTILES; ++c) {
-            mo[(warp * 8 + gid) * D + c * 8 + 2 * tig] = oacc[c][0];
-            mo[(warp * 8 + gid) * D + c * 8 + 2 * tig + 1] = oacc[c][1];
+            mo[(warp * 8 + gid) * D + c * 8 + 2 * tig] = oacc[c][0] + oacc[c][2];       // hi rows + lo rows
+            mo[(warp * 8 + gid) * D + c * 8 + 2 * tig + 1] = oacc[c][1] + oacc[c][3];
         }
         if (tig == 0) { mm[warp * 8 + gid] = m_run; ml[warp * 8 + gid] = l_run; }
         __syncthreads();
@@ -294,7 +304,9 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(Buffers b, StepLayout l
         den += ml.y * sc;
         o += b.part_o[((size_t)i * nq + j) * D + d] * sc;
     }
-    b.o[((size_t)t * nq + j) * D + d] = __float2bfloat16_rn(o / den);
+    // (hi, lo) rows of the token: b.o is [n_tok][2][nq D]
+    __nv_bfloat16* dst = b.o + (size_t)t * 2 * nq * D + (size_t)j * D + d;
+    split_bf16(o / den, dst[0], dst[(size_t)nq * D]);
 }
 
 template <int D>

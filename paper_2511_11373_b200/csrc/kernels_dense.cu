@@ -37,10 +37,11 @@ int launch_prep(const Shape& s, const Buffers& b, const StepLayout& lay, const K
 }
 
 // ---------------------------------------------------------------------------------------------
-// RMSNorm of one fp32 row held in registers/shared memory -> bf16 row (gain applied).
-// Called by every thread of the block; `vals` are this thread's elements c = tid + i * blockDim.
+// RMSNorm of one fp32 row held in registers -> (hi, lo) bf16 rows (gain applied).  Called by every
+// thread of the block; `vals` are this thread's elements c = tid + i * blockDim.  `out` points at
+// the token's hi row; the lo row follows it.
 template <int MAX_PER_THREAD>
-__device__ __forceinline__ void rms_to_bf16(const float (&vals)[MAX_PER_THREAD], int H, float eps,
+__device__ __forceinline__ void rms_to_pair(const float (&vals)[MAX_PER_THREAD], int H, float eps,
                                             const __nv_bfloat16* gain, __nv_bfloat16* out, float* scratch) {
     float ss = 0.f;
 #pragma unroll
@@ -53,7 +54,7 @@ __device__ __forceinline__ void rms_to_bf16(const float (&vals)[MAX_PER_THREAD],
 #pragma unroll
     for (int i = 0; i < MAX_PER_THREAD; ++i) {
         const int c = threadIdx.x + i * blockDim.x;
-        if (c < H) out[c] = __float2bfloat16_rn(vals[i] * r * __bfloat162float(gain[c]));
+        if (c < H) split_bf16(vals[i] * r * __bfloat162float(gain[c]), out[c], out[H + c]);
     }
 }
 
@@ -82,7 +83,7 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(Shape s, Buffers b, 
             if (hidden_tap) hidden_tap[(size_t)t * s.H + c] = v[i];
         }
     }
-    rms_to_bf16<kRowMaxPer>(v, s.H, s.eps, gain, b.h + (size_t)t * s.H, scratch);
+    rms_to_pair<kRowMaxPer>(v, s.H, s.eps, gain, b.h + (size_t)t * 2 * s.H, scratch);
 }
 
 int launch_embed(const Shape& s, const Buffers& b, const StepLayout&, const __nv_bfloat16* embed, const int32_t* tokens,
@@ -93,18 +94,20 @@ int launch_embed(const Shape& s, const Buffers& b, const StepLayout&, const __nv
 
 // ---------------------------------------------------------------------------------------------
 // Y^T = W X^T for up to 64 tokens per block column: weights streamed once from HBM, activations
-// staged through shared memory in K chunks (double buffered with cp.async).
+// (hi/lo pairs = 128 columns) staged through shared memory in K chunks (double buffered, cp.async).
 constexpr int kGemmWarps = 4;
 constexpr int kGemmTok = 64;
+constexpr int kGemmCols = 2 * kGemmTok;
+constexpr int kGemmNT = kGemmCols / 8;
 constexpr int kGemmKC = 256;
-constexpr int kGemmXBytes = kGemmTok * x_row_bytes(kGemmKC);
+constexpr int kGemmXBytes = kGemmCols * x_row_bytes(kGemmKC);
 
 enum { EPI_STORE = 0, EPI_RESID = 1 };
 
 struct GemmParams {
     const __nv_bfloat16* W;     // [rows, K]
-    const __nv_bfloat16* X;     // [*, K]
-    const int32_t* row_index;   // optional: X row of token t is row_index[t]
+    const __nv_bfloat16* X;     // [*, 2, K] (hi row, lo row per token)
+    const int32_t* row_index;   // optional: X token of output token t is row_index[t]
     float* out;                 // [n_tok, rows]
     int rows, K, n_tok;
 };
@@ -124,21 +127,22 @@ __global__ void __launch_bounds__(kGemmWarps * 32) dense_gemm_kernel(GemmParams 
     auto load_chunk = [&](int c, int buf) {
         unsigned char* dst = smem + (size_t)buf * kGemmXBytes;
         constexpr int pieces = kGemmKC * 2 / 16;  // 16-byte pieces per row
-        for (int i = threadIdx.x; i < kGemmTok * pieces; i += blockDim.x) {
-            const int t = i / pieces, pc = i - t * pieces;
-            unsigned char* d = dst + (size_t)t * xrow + pc * 16;
+        for (int i = threadIdx.x; i < kGemmCols * pieces; i += blockDim.x) {
+            const int v = i / pieces, pc = i - v * pieces;     // v: column = 2 * token + plane
+            unsigned char* d = dst + (size_t)v * xrow + pc * 16;
+            const int t = v >> 1;
             if (t < n_here) {
-                const int src_row = p.row_index ? p.row_index[tok0 + t] : tok0 + t;
-                cp_async16(d, p.X + (size_t)src_row * p.K + (size_t)c * kGemmKC + pc * 8);
+                const int src_tok = p.row_index ? p.row_index[tok0 + t] : tok0 + t;
+                cp_async16(d, p.X + ((size_t)src_tok * 2 + (v & 1)) * p.K + (size_t)c * kGemmKC + pc * 8);
             } else {
                 *reinterpret_cast<uint4*>(d) = make_uint4(0, 0, 0, 0);
             }
         }
     };
 
-    float acc[1][8][4];
+    float acc[1][kGemmNT][4];
 #pragma unroll
-    for (int n = 0; n < 8; ++n)
+    for (int n = 0; n < kGemmNT; ++n)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[0][n][j] = 0.f;
 
@@ -156,20 +160,21 @@ __global__ void __launch_bounds__(kGemmWarps * 32) dense_gemm_kernel(GemmParams 
         __syncthreads();
         const __nv_bfloat16* wr[1][2] = {{wrow[0][0] + (size_t)c * kGemmKC, wrow[0][1] + (size_t)c * kGemmKC}};
         const unsigned char* xs = smem + (size_t)(c & 1) * kGemmXBytes + (size_t)gid * xrow + tig * 16;
-        stream_mma<1, 8, 4>(wr, kGemmKC / 32, xs, 8 * xrow, acc);
+        stream_mma<1, kGemmNT, 4>(wr, kGemmKC / 32, xs, 8 * xrow, acc);
         __syncthreads();
     }
 
 #pragma unroll
-    for (int n = 0; n < 8; ++n)
+    for (int n = 0; n < kGemmNT; ++n)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int row = row_base + gid + ((j >> 1) << 3);
-            const int t = n * 8 + 2 * tig + (j & 1);
+        for (int hf = 0; hf < 2; ++hf) {
+            const int row = row_base + gid + hf * 8;
+            const int t = n * 4 + tig;
             if (row < p.rows && t < n_here) {
+                const float v = acc[0][n][2 * hf] + acc[0][n][2 * hf + 1];   // hi column + lo column
                 float* dst = p.out + (size_t)(tok0 + t) * p.rows + row;
-                if (EPI == EPI_RESID) *dst += acc[0][n][j];
-                else *dst = acc[0][n][j];
+                if (EPI == EPI_RESID) *dst += v;
+                else *dst = v;
             }
         }
 }
@@ -183,7 +188,8 @@ static int launch_gemm(const GemmParams& p, cudaStream_t st) {
 
 // ---------------------------------------------------------------------------------------------
 // Per-head RMS norm (optional), rotary embedding, cache append.  One block per token row, one
-// warp per head in turn; lane l owns the rotation pairs (l + 32 i, l + 32 i + D/2).
+// warp per head in turn; lane l owns the rotation pairs (l + 32 i, l + 32 i + D/2).  Queries leave
+// as (hi, lo) pairs: b.q is [n_tok][2][nq D]; keys and values are rounded to bf16 by the cache format.
 template <int D>
 __global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepLayout lay, KvView kv,
                                                        const __nv_bfloat16* q_gain, const __nv_bfloat16* k_gain,
@@ -226,18 +232,21 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepL
                 hi[i] *= r * __bfloat162float(g[lane + 32 * i + HALF]);
             }
         }
-        __nv_bfloat16* dst;
-        if (is_q) {
-            dst = b.q + ((size_t)t * s.nq + head) * D;
-        } else {
-            const int hk = head - s.nq;
-            dst = kv.k_pool + ((((size_t)layer * kv.n_pages + page) * s.nkv + hk) * kv.page_size + slot) * D;
-        }
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const float2 cs = b.rope[(size_t)t * HALF + lane + 32 * i];
-            dst[lane + 32 * i] = __float2bfloat16_rn(lo[i] * cs.x - hi[i] * cs.y);
-            dst[lane + 32 * i + HALF] = __float2bfloat16_rn(hi[i] * cs.x + lo[i] * cs.y);
+            const float a = lo[i] * cs.x - hi[i] * cs.y, c = hi[i] * cs.x + lo[i] * cs.y;
+            if (is_q) {
+                __nv_bfloat16* dq = b.q + (size_t)t * 2 * s.nq * D + head * D;
+                split_bf16(a, dq[lane + 32 * i], dq[s.nq * D + lane + 32 * i]);
+                split_bf16(c, dq[lane + 32 * i + HALF], dq[s.nq * D + lane + 32 * i + HALF]);
+            } else {
+                const int hk = head - s.nq;
+                __nv_bfloat16* dk = kv.k_pool +
+                    ((((size_t)layer * kv.n_pages + page) * s.nkv + hk) * kv.page_size + slot) * D;
+                dk[lane + 32 * i] = __float2bfloat16_rn(a);
+                dk[lane + 32 * i + HALF] = __float2bfloat16_rn(c);
+            }
         }
     }
 }

@@ -12,8 +12,8 @@ constexpr int kMaxExperts = 1024;
 constexpr int kMaxTopK = 32;
 
 // ---------------------------------------------------------------------------------------------
-// One block per token row.  h2 = rms(x) * g (kept in fp32 for the gate, stored as bf16 for the
-// experts); z_e = <W_r[e], h2> accumulated in fp32 in a fixed order; pi = softmax(z); the k largest
+// One block per token row.  h2 = rms(x) * g (kept in fp32 for the gate, stored as a (hi, lo) bf16
+// pair for the experts); z_e = <W_r[e], h2> accumulated in fp32 in a fixed order; pi = softmax(z); the k largest
 // pi (ties: lower index) and their renormalised weights.
 __global__ void __launch_bounds__(kRouterThreads) router_kernel(Shape s, Buffers b, const __nv_bfloat16* gain,
                                                                 const __nv_bfloat16* Wr, DebugTaps dbg, int layer,
@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(kRouterThreads) router_kernel(Shape s, Buffers
     for (int c = tid; c < H; c += kRouterThreads) {
         const float v = hs[c] * r * __bfloat162float(gain[c]);
         hs[c] = v;
-        b.h[(size_t)t * H + c] = __float2bfloat16_rn(v);
+        split_bf16(v, b.h[(size_t)t * 2 * H + c], b.h[(size_t)t * 2 * H + H + c]);
     }
     __syncthreads();
 
@@ -143,12 +143,13 @@ __global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int l
 // Grouped SwiGLU, first half: act[slot, i] = silu(<W_gate[e, i], h>) * <W_up[e, i], h> for the
 // tokens of expert e.  grid = (row blocks, experts); a warp owns 16 gate rows and the matching 16
 // up rows and streams them once over the full K; the expert's activation rows sit in shared memory.
-constexpr int kExpWarps = 4;
+constexpr int kExpMaxWarps = 12;
 
 template <int NT>
 __device__ __forceinline__ void gate_up_tile(const __nv_bfloat16* Wg, const __nv_bfloat16* Wu, int H, int I,
                                              int row_base, const unsigned char* xs_base, int xrow, int m_here,
-                                             __nv_bfloat16* act_out /* slot t0 of this expert */, int lane) {
+                                             __nv_bfloat16* act_out /* slot t0 of this expert, [slot][2][I] */,
+                                             int lane) {
     const int gid = lane >> 2, tig = lane & 3;
     const __nv_bfloat16* wrow[2][2] = {
         {Wg + (size_t)(row_base + gid) * H + tig * 8, Wg + (size_t)(row_base + gid + 8) * H + tig * 8},
@@ -162,17 +163,19 @@ __device__ __forceinline__ void gate_up_tile(const __nv_bfloat16* Wg, const __nv
 #pragma unroll
     for (int n = 0; n < NT; ++n)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int row = row_base + gid + ((j >> 1) << 3);
-            const int t = n * 8 + 2 * tig + (j & 1);
+        for (int hf = 0; hf < 2; ++hf) {
+            const int row = row_base + gid + hf * 8;
+            const int t = n * 4 + tig;                 // columns 2t (hi) and 2t+1 (lo) of token t
             if (t < m_here) {
-                const float gte = acc[0][n][j], up = acc[1][n][j];
-                act_out[(size_t)t * I + row] = __float2bfloat16_rn(gte / (1.f + expf(-gte)) * up);
+                const float gte = acc[0][n][2 * hf] + acc[0][n][2 * hf + 1];
+                const float up = acc[1][n][2 * hf] + acc[1][n][2 * hf + 1];
+                __nv_bfloat16* dst = act_out + (size_t)t * 2 * I + row;
+                split_bf16(gte / (1.f + expf(-gte)) * up, dst[0], dst[I]);
             }
         }
 }
 
-__global__ void __launch_bounds__(kExpWarps * 32) expert_gate_up_kernel(Shape s, Buffers b, const __nv_bfloat16* Wgu,
+__global__ void __launch_bounds__(kExpMaxWarps * 32) expert_gate_up_kernel(Shape s, Buffers b, const __nv_bfloat16* Wgu,
                                                                         int tok_cap) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int e = blockIdx.y;
@@ -180,7 +183,7 @@ __global__ void __launch_bounds__(kExpWarps * 32) expert_gate_up_kernel(Shape s,
     if (m == 0) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int H = s.H, I = s.I;
-    const int row_base = (blockIdx.x * kExpWarps + warp) * 16;
+    const int row_base = (blockIdx.x * (blockDim.x >> 5) + warp) * 16;
     const bool row_ok = row_base < I;       // I is a multiple of 16
     const int xrow = x_row_bytes(H);
     const __nv_bfloat16* Wg = Wgu + (size_t)e * 2 * I * H;
@@ -188,19 +191,20 @@ __global__ void __launch_bounds__(kExpWarps * 32) expert_gate_up_kernel(Shape s,
     const int pieces = H / 8;
     for (int t0 = 0; t0 < m; t0 += tok_cap) {
         const int m_here = min(tok_cap, m - t0);
-        const int rows_ld = (m_here + 7) & ~7;
-        for (int i = threadIdx.x; i < rows_ld * pieces; i += blockDim.x) {
-            const int t = i / pieces, pc = i - t * pieces;
-            unsigned char* d = smem + (size_t)t * xrow + pc * 16;
-            if (t < m_here) cp_async16(d, b.h + (size_t)b.slot_token[o0 + t0 + t] * H + pc * 8);
+        const int cols_ld = (2 * m_here + 7) & ~7;      // column v = 2 * token + plane
+        for (int i = threadIdx.x; i < cols_ld * pieces; i += blockDim.x) {
+            const int v = i / pieces, pc = i - v * pieces;
+            unsigned char* d = smem + (size_t)v * xrow + pc * 16;
+            if ((v >> 1) < m_here)
+                cp_async16(d, b.h + ((size_t)b.slot_token[o0 + t0 + (v >> 1)] * 2 + (v & 1)) * H + pc * 8);
             else *reinterpret_cast<uint4*>(d) = make_uint4(0, 0, 0, 0);
         }
         cp_async_commit();
         cp_async_wait<0>();
         __syncthreads();
         if (row_ok) {
-            __nv_bfloat16* out = b.act + (size_t)(o0 + t0) * I;
-            const int nt = (m_here + 7) >> 3;
+            __nv_bfloat16* out = b.act + (size_t)(o0 + t0) * 2 * I;
+            const int nt = (m_here + 3) >> 2;
             if (nt == 1) gate_up_tile<1>(Wg, Wu, H, I, row_base, smem, xrow, m_here, out, lane);
             else if (nt == 2) gate_up_tile<2>(Wg, Wu, H, I, row_base, smem, xrow, m_here, out, lane);
             else gate_up_tile<4>(Wg, Wu, H, I, row_base, smem, xrow, m_here, out, lane);
@@ -228,14 +232,14 @@ __device__ __forceinline__ void down_tile(const __nv_bfloat16* Wd, int H, int I,
 #pragma unroll
         for (int n = 0; n < NT; ++n)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int row = row_base + mt * 16 + gid + ((j >> 1) << 3);
-                const int t = n * 8 + 2 * tig + (j & 1);
-                if (t < m_here) y_out[(size_t)t * H + row] = acc[mt][n][j];
+            for (int hf = 0; hf < 2; ++hf) {
+                const int row = row_base + mt * 16 + gid + hf * 8;
+                const int t = n * 4 + tig;
+                if (t < m_here) y_out[(size_t)t * H + row] = acc[mt][n][2 * hf] + acc[mt][n][2 * hf + 1];
             }
 }
 
-__global__ void __launch_bounds__(kExpWarps * 32) expert_down_kernel(Shape s, Buffers b, const __nv_bfloat16* Wdn,
+__global__ void __launch_bounds__(kExpMaxWarps * 32) expert_down_kernel(Shape s, Buffers b, const __nv_bfloat16* Wdn,
                                                                      int tok_cap) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int e = blockIdx.y;
@@ -243,18 +247,18 @@ __global__ void __launch_bounds__(kExpWarps * 32) expert_down_kernel(Shape s, Bu
     if (m == 0) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int H = s.H, I = s.I;
-    const int row_base = (blockIdx.x * kExpWarps + warp) * 32;
+    const int row_base = (blockIdx.x * (blockDim.x >> 5) + warp) * 32;
     const bool row_ok = row_base < H;       // H is a multiple of 32
     const int xrow = x_row_bytes(I);
     const __nv_bfloat16* Wd = Wdn + (size_t)e * H * I;
     const int pieces = I / 8;
     for (int t0 = 0; t0 < m; t0 += tok_cap) {
         const int m_here = min(tok_cap, m - t0);
-        const int rows_ld = (m_here + 7) & ~7;
-        for (int i = threadIdx.x; i < rows_ld * pieces; i += blockDim.x) {
-            const int t = i / pieces, pc = i - t * pieces;
-            unsigned char* d = smem + (size_t)t * xrow + pc * 16;
-            if (t < m_here) cp_async16(d, b.act + (size_t)(o0 + t0 + t) * I + pc * 8);
+        const int cols_ld = (2 * m_here + 7) & ~7;      // act rows are already (hi, lo) interleaved
+        for (int i = threadIdx.x; i < cols_ld * pieces; i += blockDim.x) {
+            const int v = i / pieces, pc = i - v * pieces;
+            unsigned char* d = smem + (size_t)v * xrow + pc * 16;
+            if ((v >> 1) < m_here) cp_async16(d, b.act + ((size_t)(o0 + t0) * 2 + v) * I + pc * 8);
             else *reinterpret_cast<uint4*>(d) = make_uint4(0, 0, 0, 0);
         }
         cp_async_commit();
@@ -262,7 +266,7 @@ __global__ void __launch_bounds__(kExpWarps * 32) expert_down_kernel(Shape s, Bu
         __syncthreads();
         if (row_ok) {
             float* out = b.y + (size_t)(o0 + t0) * H;
-            const int nt = (m_here + 7) >> 3;
+            const int nt = (m_here + 3) >> 2;
             if (nt == 1) down_tile<1>(Wd, H, I, row_base, smem, xrow, m_here, out, lane);
             else if (nt == 2) down_tile<2>(Wd, H, I, row_base, smem, xrow, m_here, out, lane);
             else down_tile<4>(Wd, H, I, row_base, smem, xrow, m_here, out, lane);
@@ -302,7 +306,9 @@ __global__ void __launch_bounds__(kRouterThreads) combine_kernel(Shape s, Buffer
 #pragma unroll
     for (int i = 0; i < kRowMaxPer; ++i) {
         const int c = tid + i * kRouterThreads;
-        if (c < H) b.h[(size_t)t * H + c] = __float2bfloat16_rn(v[i] * r * __bfloat162float(next_gain[c]));
+        if (c < H)
+            split_bf16(v[i] * r * __bfloat162float(next_gain[c]), b.h[(size_t)t * 2 * H + c],
+                       b.h[(size_t)t * 2 * H + H + c]);
     }
 }
 
@@ -314,18 +320,24 @@ int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const Debug
     return 2;
 }
 
-static int expert_tok_cap(const Shape& s, int n_tok) {
-    // average tokens per expert decides how many 8-token tiles a pass holds (the tail loops)
+// Tokens held in shared memory per pass (4 per column tile); experts with more tokens loop and
+// stream their weights again.  Small groups keep the footprint low enough for three CTAs of four
+// warps per SM; larger ones use one wide CTA per SM so that enough loads stay in flight.
+static void expert_plan(const Shape& s, int n_tok, int* cap, int* warps) {
     const double avg = (double)n_tok * s.k / s.E;
-    return avg <= 2.0 ? 8 : (avg <= 6.0 ? 16 : 32);
+    *cap = avg <= 5.0 ? 8 : 16;
+    *warps = *cap == 8 ? 4 : kExpMaxWarps;
+    while ((size_t)*cap * 2 * x_row_bytes(s.H) > 200u * 1024u && *cap > 4) *cap /= 2;
 }
 
 int launch_experts(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st) {
-    const int cap = expert_tok_cap(s, n_tok);
-    dim3 g1((s.I / 16 + kExpWarps - 1) / kExpWarps, s.E);
-    expert_gate_up_kernel<<<g1, kExpWarps * 32, (size_t)cap * x_row_bytes(s.H), st>>>(s, b, w.w_gate_up, cap);
-    dim3 g2((s.H / 32 + kExpWarps - 1) / kExpWarps, s.E);
-    expert_down_kernel<<<g2, kExpWarps * 32, (size_t)cap * x_row_bytes(s.I), st>>>(s, b, w.w_down, cap);
+    int cap, warps;
+    expert_plan(s, n_tok, &cap, &warps);
+    dim3 g1((s.I / 16 + warps - 1) / warps, s.E);
+    expert_gate_up_kernel<<<g1, warps * 32, (size_t)cap * 2 * x_row_bytes(s.H), st>>>(s, b, w.w_gate_up, cap);
+    const int w2 = warps == kExpMaxWarps ? 8 : warps;
+    dim3 g2((s.H / 32 + w2 - 1) / w2, s.E);
+    expert_down_kernel<<<g2, w2 * 32, (size_t)cap * 2 * x_row_bytes(s.I), st>>>(s, b, w.w_down, cap);
     return 2;
 }
 

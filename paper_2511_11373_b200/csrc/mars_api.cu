@@ -90,10 +90,10 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
     t.step = (int32_t*)take((size_t)lay.total_words * 4);
     t.err = (int32_t*)take(256);
     t.x = (float*)take(n * H * 4);
-    t.h = (__nv_bfloat16*)take(n * H * 2);
+    t.h = (__nv_bfloat16*)take(n * 2 * H * 2);
     t.qkv = (float*)take(n * (nq + 2 * nkv) * D * 4);
-    t.q = (__nv_bfloat16*)take(n * nq * D * 2);
-    t.o = (__nv_bfloat16*)take(n * nq * D * 2);
+    t.q = (__nv_bfloat16*)take(n * 2 * nq * D * 2);
+    t.o = (__nv_bfloat16*)take(n * 2 * nq * D * 2);
     t.rope = (float2*)take(n * (D / 2) * 8);
     t.inv_freq = (double*)take((D / 2) * 8);
     t.part_o = (float*)take((size_t)k.n_items * nq * D * 4);
@@ -104,7 +104,7 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
     t.slot_token = (int32_t*)take(n * kk * 4);
     t.slot_of = (int32_t*)take(n * kk * 4);
     t.active = (int32_t*)take((size_t)c.n_layers * 4);
-    t.act = (__nv_bfloat16*)take(n * kk * c.expert_inter * 2);
+    t.act = (__nv_bfloat16*)take(n * kk * 2 * c.expert_inter * 2);
     t.y = (float*)take(n * kk * H * 4);
     t.logits = (float*)take((size_t)k.n_emit * c.vocab * 4);
     int32_t* a = (int32_t*)take((size_t)k.n_emit * 4);

@@ -46,10 +46,10 @@ struct Buffers {
     int32_t* step;          // the uploaded step block
     int32_t* err;           // status word
     float* x;               // [n_tok, H] residual stream (fp32)
-    __nv_bfloat16* h;       // [n_tok, H] normalised input of the next projection
+    __nv_bfloat16* h;       // [n_tok, 2, H] normalised input of the next projection, (hi, lo) rows
     float* qkv;             // [n_tok, (nq + 2 nkv) D] raw projection
-    __nv_bfloat16* q;       // [n_tok, nq D] rotated queries
-    __nv_bfloat16* o;       // [n_tok, nq D] attention output
+    __nv_bfloat16* q;       // [n_tok, 2, nq D] rotated queries, (hi, lo) rows
+    __nv_bfloat16* o;       // [n_tok, 2, nq D] attention output, (hi, lo) rows
     float2* rope;           // [n_tok, D/2] (cos, sin) of pos * theta_i
     double* inv_freq;       // [D/2] theta^(-2i/D)
     float* part_o;          // [items, nq, D] unnormalised partial outputs
@@ -60,7 +60,7 @@ struct Buffers {
     int32_t* slot_token;    // [n_tok k] token row served by every expert slot
     int32_t* slot_of;       // [n_tok k] slot of (token, j)
     int32_t* active;        // [L] distinct experts per layer
-    __nv_bfloat16* act;     // [n_tok k, I]
+    __nv_bfloat16* act;     // [n_tok k, 2, I] SwiGLU activations, (hi, lo) rows
     float* y;               // [n_tok k, H]
     float* logits;          // [n_emit, V]
 };

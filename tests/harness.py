@@ -117,12 +117,14 @@ def compare_step(gpu: dict, orc: dict, k: int, greedy: bool, label: str = "") ->
     L, n, E = probs.shape
     margin = topk_margin(probs, k)
     own = torch.topk(probs.double(), k, dim=-1).indices
-    bad = 0
+    bad, equal = 0, 0
     for l in range(L):
         for t in range(n):
-            if margin[l, t] >= TOL_ROUTE_MARGIN:
-                if set(own[l, t].tolist()) != set(gpu["router_idx"][l, t].tolist()):
-                    bad += 1
+            same = set(own[l, t].tolist()) == set(gpu["router_idx"][l, t].tolist())
+            equal += same
+            if margin[l, t] >= TOL_ROUTE_MARGIN and not same:
+                bad += 1
+    stats["routing_equal"] = equal
     stats["routing_checked"] = int((margin >= TOL_ROUTE_MARGIN).sum())
     stats["routing_total"] = L * n
     assert bad == 0, f"{label}: {bad} routing decisions differ where the oracle margin >= {TOL_ROUTE_MARGIN}"
