@@ -1,0 +1,378 @@
+"""Benchmark of the rollout step: decode tokens/s on a Qwen3-30B-A3B-shaped MoE and the fraction of
+the HBM roofline it reaches.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 2|3|5] [--impl reference]
+
+One "step" is one pass of the whole hot path (embedding, 48 x {QKV+RoPE+append, paged attention,
+output projection, router, experts, combine}, lm_head, sampling) over the batch.  Inputs are
+synthetic and seeded (random-init bf16 weights, N(0,1) cache, uniform tokens); every step streams far
+more than the L2 holds (tens of GB), so no L2 flush is needed between timed steps.
+
+With N > 1 (torchrun) every rank runs an independent replica of the same workload on its own GPU:
+sequences are independent, there is no collective on the data path, and the reported value is the
+sum over replicas divided by the slowest rank's time ("replicas only", weak scaling).
+
+`--impl reference` times the CPU oracle (test infrastructure, plain C, as it stands) on a bounded
+sample of the same workload on the host cores; it is a deliberately slow baseline.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2511_11373_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode_tokens_per_sec"
+UNIT = "tokens/s"
+PEAKS_FALLBACK = dict(hbm_gbs=6650.0, source="fallback")
+
+
+def load_peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), source="measured")
+    return dict(PEAKS_FALLBACK)
+
+
+# ----------------------------------------------------------------------------------- clocks sampler
+CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+class ClockSampler:
+    def __init__(self, gpu_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={CLOCK_QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"], stdout=self.tmp,
+                                         stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = [l.strip().split(", ") for l in open(self.tmp.name) if l.strip()]
+        os.unlink(self.tmp.name)
+        clocks, reasons, smax = [], set(), None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                clocks.append(float(r[1])); smax = float(r[2])
+            except ValueError:
+                continue
+            for name, val in zip(names, r[5:9]):
+                if val.strip().lower() == "active":
+                    reasons.add(name)
+        if clocks:
+            out.update(sm_mhz=statistics.median(clocks), sm_max_mhz=smax, reasons=sorted(reasons), samples=len(clocks))
+        return out
+
+
+# ----------------------------------------------------------------------------------- workload set-up
+def algorithmic_bytes(model: dict, kv_tokens: int, active_per_layer, n_lm_rows: int = 1) -> dict:
+    """Bytes one decode step must move: attention + router weights, the weights of the experts that
+    were actually selected, the cached keys/values read, and the lm_head (all bf16)."""
+    H, nq, nkv, D = model["hidden"], model["n_q_heads"], model["n_kv_heads"], model["head_dim"]
+    E, I, V, L = model["n_experts"], model["expert_inter"], model["vocab"], model["n_layers"]
+    w_attn = (H * (nq + 2 * nkv) * D + nq * D * H) * 2
+    w_router = E * H * 2
+    w_expert = 3 * H * I * 2
+    kv = 2 * nkv * D * 2 * kv_tokens * L
+    experts = sum(int(a) for a in active_per_layer) * w_expert
+    lm = V * H * 2
+    return dict(attn_router=L * (w_attn + w_router), experts=experts, kv=kv, lm_head=lm,
+                total=L * (w_attn + w_router) + experts + kv + lm, w_expert=w_expert)
+
+
+class DecodeWorkload:
+    """Builds a config (weights, cache, page tables) on one GPU and steps it through the C ABI."""
+
+    def __init__(self, cfg: dict, total_steps: int, device: torch.device, seed: int = 0):
+        from paper_2511_11373_b200 import binding
+        self.binding = binding
+        self.cfg, self.device = cfg, device
+        model, ps = cfg["model"], cfg["page_size"]
+        self.model_shape = model
+        self.ctx, self.stages = wl.make_context_lengths(cfg, seed=seed)
+        B = len(self.ctx)
+        self.B = B
+        cap = [c + total_steps + 1 for c in self.ctx]
+        n_pages = sum(wl.pages_needed(c, ps) for c in cap) + 8
+        max_pages = max(wl.pages_needed(c, ps) for c in cap) + 1
+        free, _ = torch.cuda.mem_get_info(device)
+        t0 = time.time()
+        self.weights = wl.make_weights(model, seed=seed, device=device, gains="ones")
+        self.k_pool, self.v_pool = wl.make_kv_pools(model, n_pages, ps, seed=seed, device=device)
+        torch.cuda.synchronize(device)
+        self.setup_s = time.time() - t0
+        self.pages = wl.make_page_assignment(cap, ps, n_pages, seed=seed)
+        self.model = binding.Model(model, self.weights, max_decode_seqs=B, max_prefill_tokens=0, max_pos=max(cap) + 8)
+        self.kv = binding.KvCache(self.model, self.k_pool, self.v_pool, ps, B, max_pages)
+        for b in range(B):
+            self.kv.seq_adopt(b, self.pages[b], self.ctx[b])
+        self.tok_a = wl.make_tokens(B, model["vocab"], seed=seed).to(device)
+        self.tok_b = torch.empty_like(self.tok_a)
+        self.logp = torch.empty(B, dtype=torch.float32, device=device)
+        self.step_no = 0
+        s = cfg["sampling"]
+        self.sampling = dict(greedy=s["greedy"], temperature=s["temperature"], top_p=s["top_p"])
+        self.ids = list(range(B))
+        self.mem_free_before = free
+
+    def step(self):
+        b = self.binding
+        smp = b.make_sampling(seed=2025, step=self.step_no, **self.sampling)
+        st = b.mars_decode_step(self.model, self.kv, self.ids, self.tok_a, smp, self.tok_b, self.logp)
+        if st != 0:
+            raise b.MarsError(st, "mars_decode_step")
+        self.tok_a, self.tok_b = self.tok_b, self.tok_a      # the sampled tokens feed the next step
+        self.step_no += 1
+
+    def step_host(self, in_host, out_tok_host, out_lp_host):
+        b = self.binding
+        smp = b.make_sampling(seed=2025, step=self.step_no, **self.sampling)
+        st = b.mars_decode_step_host(self.model, self.kv, self.ids, in_host, smp, out_tok_host, out_lp_host)
+        if st != 0:
+            raise b.MarsError(st, "mars_decode_step_host")
+        self.step_no += 1
+
+    def kv_tokens_now(self) -> int:
+        return sum(self.kv.seq_len(b) for b in range(self.B))
+
+
+# ----------------------------------------------------------------------------------- CPU baseline
+class OracleSample:
+    """The CPU oracle, as it stands, on a bounded sample of the workload: ONE decoder layer plus the
+    lm_head and sampling over the first n_seq sequences (own CPU-generated weights and cache of the
+    same shapes and distributions); a full step is the layer time scaled by the number of layers."""
+
+    def __init__(self, cfg: dict, n_seq: int, seed: int = 0):
+        import oracle
+        self.oracle, self.cfg = oracle, cfg
+        self.model = dict(cfg["model"])
+        one = dict(self.model, n_layers=1)
+        ctx_all, _ = wl.make_context_lengths(cfg, seed=seed)
+        self.n_all = len(ctx_all)
+        self.n_seq = min(n_seq, self.n_all)
+        ctx = ctx_all[: self.n_seq]
+        self.ps = cfg["page_size"]
+        cap = [c + 1 for c in ctx]
+        n_pages = sum(wl.pages_needed(c, self.ps) for c in cap)
+        pages = wl.make_page_assignment(cap, self.ps, n_pages, seed=seed, shuffle=False)
+        self.w = wl.make_weights(one, seed=seed, device="cpu", gains="ones")
+        self.kp, self.vp = wl.make_kv_pools(one, n_pages, self.ps, seed=seed, device="cpu")
+        self.bt = wl.block_table_tensor(pages, max(len(p) for p in pages))
+        self.ocfg = oracle.Config(**one)
+        self.toks = wl.make_tokens(self.n_seq, self.model["vocab"], seed=seed)
+        self.seq = torch.arange(self.n_seq, dtype=torch.int32)
+        self.pos = torch.tensor(ctx, dtype=torch.int32)
+
+    def run(self) -> dict:
+        o = self.oracle
+        x = o.embed(self.w["embed"], self.toks)
+        t0 = time.perf_counter()
+        o.layer_forward(self.ocfg, self.w["layers"][0], x, self.seq, self.pos, self.kp[0], self.vp[0], self.bt, self.ps)
+        t_layer = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        logits = o.lm_head(self.ocfg, self.w["final_norm"], self.w["lm_head"], x)
+        s = self.cfg["sampling"]
+        for i in range(self.n_seq):
+            o.sample(logits[i].contiguous(), s["temperature"], s["top_p"], bool(s["greedy"]), o.uniform(1, 0, i))
+        t_head = time.perf_counter() - t0
+        total = t_layer * self.model["n_layers"] + t_head
+        return dict(value=self.n_seq / total, unit=UNIT, cores=os.cpu_count(), kind="oracle",
+                    sample=f"{self.n_seq} of {self.n_all} sequences; one decoder layer timed ({t_layer:.2f} s) and "
+                           f"scaled by {self.model['n_layers']} layers, plus lm_head+sampling ({t_head:.2f} s)",
+                    seconds=t_layer + t_head)
+
+
+# ----------------------------------------------------------------------------------- distributed glue
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    """Max of a scalar over ranks (NCCL on GPUs, gloo on CPU); identity for one rank."""
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# ----------------------------------------------------------------------------------- main arms
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    cfg = wl.CONFIGS[args.workload]
+    sample = OracleSample(cfg, 4)
+    for _ in range(args.warmup):
+        sample.run()
+    t0 = time.perf_counter()
+    rates = [sample.run() for _ in range(args.steps)]
+    wall = time.perf_counter() - t0
+    value = statistics.mean(r["value"] for r in rates)
+    base = rates[-1]
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=1000.0 * wall / max(args.steps, 1), higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=cfg["name"], note="CPU oracle on a bounded sample per step, extrapolated to a full step"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=base["cores"], kind="oracle", sample=base["sample"]),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+def run_cuda(args):
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    cfg = wl.CONFIGS[args.workload]
+    e2e_steps = min(args.steps, 16)
+    prof_steps = min(args.steps, 8)
+    total = args.warmup + args.steps + e2e_steps + prof_steps + 4
+    w = DecodeWorkload(cfg, total, device)
+    model = cfg["model"]
+    stream = torch.cuda.current_stream()
+
+    for _ in range(args.warmup):
+        w.step()
+    torch.cuda.synchronize()
+    barrier(world)
+    kv_tokens_start = w.kv_tokens_now()
+    sampler = ClockSampler(local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(args.steps):
+        w.step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    clocks = sampler.stop()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, device)
+    assert w.model.poll_status() == 0
+    info = w.model.last_step_info()
+    ms_per_step = ms / args.steps
+    value = world * w.B * args.steps / (ms / 1000.0)
+
+    # end to end through the host-buffer entry point (pinned host tokens in, tokens + log-probs out)
+    in_host = w.tok_a.cpu().pin_memory()
+    out_tok = torch.empty(w.B, dtype=torch.int32).pin_memory()
+    out_lp = torch.empty(w.B, dtype=torch.float32).pin_memory()
+    torch.cuda.synchronize()
+    barrier(world)
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        w.step_host(in_host, out_tok, out_lp)
+        in_host.copy_(out_tok)
+    torch.cuda.synchronize()
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1000.0, world, device)
+    e2e = dict(value=world * w.B * e2e_steps / (e2e_ms / 1000.0), unit=UNIT, h2d_bytes_per_step=w.B * 4,
+               d2h_bytes_per_step=w.B * 8, steps=e2e_steps)
+
+    # per-kernel-class device time over a few more steps (event pairs around every launch)
+    w.tok_a.copy_(out_tok.to(device))
+    w.model.profile_enable(True)
+    kv_tokens_prof = w.kv_tokens_now()
+    for _ in range(prof_steps):
+        w.step()
+    prof = w.model.profile_read()
+    w.model.profile_enable(False)
+    active = w.model.active_experts().tolist()
+
+    peaks = load_peaks()
+    kv_mid = kv_tokens_start + w.B * (args.steps + 1) // 2          # cached tokens read by the average timed step
+    bytes_step = algorithmic_bytes(model, kv_mid, active)
+    step_gbs = bytes_step["total"] / (ms_per_step * 1e-3) / 1e9
+    # dominant kernel: algorithmic bytes per launch / mean launch time
+    kv_prof = kv_tokens_prof + w.B * (prof_steps + 1) // 2
+    per_launch = {
+        "attn": 2 * model["n_kv_heads"] * model["head_dim"] * 2 * kv_prof,
+        "gate_up": (sum(active) / len(active)) * 2 * model["hidden"] * model["expert_inter"] * 2,
+        "down": (sum(active) / len(active)) * model["hidden"] * model["expert_inter"] * 2,
+    }
+    kernels = {}
+    for name, (kms, n) in prof.items():
+        if n:
+            kernels[name] = dict(ms_per_step=kms / prof_steps, launches_per_step=n / prof_steps,
+                                 us_per_launch=1000.0 * kms / n)
+            if name in per_launch:
+                kernels[name]["achieved_gbs"] = per_launch[name] / (kms / n * 1e-3) / 1e9
+    top = max(per_launch, key=lambda k: kernels.get(k, {}).get("ms_per_step", 0.0))
+    roofline = dict(bound="hbm", kernel=top, achieved=kernels[top]["achieved_gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=kernels[top]["achieved_gbs"] / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"],
+                    bytes_per_launch=per_launch[top], us_per_launch=kernels[top]["us_per_launch"])
+
+    if rank != 0:
+        return
+    cpu = OracleSample(cfg, 8).run()
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic",
+                config=dict(workload=cfg["name"], batch=w.B, n_layers=model["n_layers"], page_size=cfg["page_size"],
+                            context_tokens=kv_tokens_start, sampling=cfg["sampling"], l2="inputs larger than L2",
+                            replicas=world, setup_s=round(w.setup_s, 1)),
+                clocks=clocks, e2e=e2e, gpu_launches=int(info["kernel_launches"]) * args.steps,
+                roofline=roofline,
+                step_roofline=dict(bytes_per_step=bytes_step["total"], experts=bytes_step["experts"], kv=bytes_step["kv"],
+                                   attn_router=bytes_step["attn_router"], lm_head=bytes_step["lm_head"],
+                                   achieved_gbs=step_gbs, frac_of_measured_hbm=step_gbs / peaks["hbm_gbs"],
+                                   frac_of_nominal_8tbs=step_gbs / 8000.0,
+                                   active_experts_mean=sum(active) / len(active)),
+                kernels=kernels, cpu_baseline={k: v for k, v in cpu.items() if k != "seconds"})
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", type=int, default=3, choices=[2, 3, 5])
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

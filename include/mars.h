@@ -190,6 +190,28 @@ typedef struct {
 } mars_step_info_t;
 MARS_API mars_status_t mars_last_step_info(const mars_model_t *model, mars_step_info_t *out);
 
+/* Per-kernel-class timing for benchmarks.  While enabled, every step brackets each launch of the
+ * classes below with a CUDA event pair on the step's stream (the events are host objects owned by
+ * the library).  mars_profile_read synchronises the stream, adds the elapsed milliseconds and the
+ * launch counts recorded since the last read into the two arrays of MARS_K_COUNT entries, and
+ * recycles the events. */
+enum {
+    MARS_K_QKV = 0,      /* QKV projection + per-head norm + RoPE + cache append */
+    MARS_K_ATTN,         /* split-K paged attention                              */
+    MARS_K_ATTN_MERGE,   /* merge of the spans                                   */
+    MARS_K_OPROJ,        /* output projection + residual                         */
+    MARS_K_ROUTER,       /* router + permutation                                 */
+    MARS_K_GATE_UP,      /* expert gate/up contraction + SwiGLU                  */
+    MARS_K_DOWN,         /* expert down contraction                              */
+    MARS_K_COMBINE,      /* weighted combine + residual + next norm              */
+    MARS_K_LM_HEAD,      /* lm_head contraction                                  */
+    MARS_K_SAMPLE,       /* log-softmax + sampling                               */
+    MARS_K_OTHER,        /* step preparation, embedding                          */
+    MARS_K_COUNT
+};
+MARS_API mars_status_t mars_profile_enable(mars_model_t *model, int32_t enable);
+MARS_API mars_status_t mars_profile_read(mars_model_t *model, double *ms_per_class, int64_t *launches_per_class);
+
 /* Device array [n_layers] (int32) inside the workspace that every step overwrites with the number
  * of distinct experts selected per layer; valid after the step's stream is synchronised. */
 MARS_API const int32_t *mars_active_experts_device(const mars_model_t *model);

@@ -20,6 +20,10 @@ STATUS_NAMES = {0: "MARS_OK", 1: "MARS_ERR_INVALID_ARG", 2: "MARS_ERR_UNSUPPORTE
 LAYER_FIELDS = ("attn_norm", "wqkv", "q_norm", "k_norm", "wo", "mlp_norm", "router", "w_gate_up", "w_down")
 
 
+KERNEL_CLASSES = ("qkv", "attn", "attn_merge", "oproj", "router", "gate_up", "down", "combine", "lm_head", "sample",
+                  "other")
+
+
 class MarsError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -81,6 +85,8 @@ SIGNATURES = {
     "mars_decode_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), c_void_p,
                                         POINTER(mars_sampling_t), c_void_p, c_void_p]),
     "mars_poll_status": (c_int32, [c_void_p]),
+    "mars_profile_enable": (c_int32, [c_void_p, c_int32]),
+    "mars_profile_read": (c_int32, [c_void_p, POINTER(ctypes.c_double), POINTER(c_int64)]),
     "mars_last_step_info": (c_int32, [c_void_p, POINTER(mars_step_info_t)]),
     "mars_active_experts_device": (c_void_p, [c_void_p]),
     "mars_last_cuda_error": (c_int32, []),
@@ -181,6 +187,16 @@ class Model:
         _check(lib().mars_last_step_info(self.handle, byref(info)), "mars_last_step_info")
         return dict(kernel_launches=info.kernel_launches, attn_items=info.attn_items,
                     kv_tokens_read=info.kv_tokens_read)
+
+    def profile_enable(self, on: bool = True):
+        _check(lib().mars_profile_enable(self.handle, int(on)), "mars_profile_enable")
+
+    def profile_read(self) -> dict:
+        """{class name: (milliseconds, launches)} accumulated since the last read."""
+        ms = (ctypes.c_double * len(KERNEL_CLASSES))()
+        n = (c_int64 * len(KERNEL_CLASSES))()
+        _check(lib().mars_profile_read(self.handle, ms, n), "mars_profile_read")
+        return {name: (ms[i], n[i]) for i, name in enumerate(KERNEL_CLASSES)}
 
     def active_experts(self) -> torch.Tensor:
         """Distinct experts selected per layer in the last step (copied to the host; synchronises)."""

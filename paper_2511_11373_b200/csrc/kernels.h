@@ -37,11 +37,13 @@ int launch_lm_head(const Shape& s, const Buffers& b, const StepLayout& lay, cons
                    cudaStream_t st);
 
 int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_k,
-                     const CUtensorMap& tm_v, int layer, int n_tok, int n_items, int sm_count, cudaStream_t st);
+                     const CUtensorMap& tm_v, int layer, int sm_count, cudaStream_t st);
+int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st);
 
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,
                   cudaStream_t st);
-int launch_experts(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
+int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
+int launch_down(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
 int launch_combine(const Shape& s, const Buffers& b, const __nv_bfloat16* next_gain, float* hidden_tap, int n_tok,
                    cudaStream_t st);
 

@@ -313,7 +313,7 @@ template <int D>
 static size_t attn_smem_bytes() { return (size_t)kAttnStages * 2 * kStageTok * D * 2 + 1024; }
 
 int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_k,
-                     const CUtensorMap& tm_v, int layer, int n_tok, int n_items, int sm_count, cudaStream_t st) {
+                     const CUtensorMap& tm_v, int layer, int sm_count, cudaStream_t st) {
     AttnParams p;
     p.q = b.q; p.part_o = b.part_o; p.part_ml = b.part_ml; p.step = b.step; p.lay = lay;
     p.block_table = kv.block_table; p.err = b.err;
@@ -322,15 +322,15 @@ int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, co
     p.nkv = s.nkv; p.nq = s.nq; p.g = s.nq / s.nkv; p.layer = layer;
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
     const int grid = sm_count * 2;
-    (void)n_items;
-    if (s.D == 128) {
-        attn_decode_kernel<128><<<grid, kAttnWarps * 32, attn_smem_bytes<128>(), st>>>(tm_k, tm_v, p);
-        attn_combine_kernel<128><<<dim3(n_tok, s.nq), 128, 0, st>>>(b, lay, s.nq);
-    } else {
-        attn_decode_kernel<64><<<grid, kAttnWarps * 32, attn_smem_bytes<64>(), st>>>(tm_k, tm_v, p);
-        attn_combine_kernel<64><<<dim3(n_tok, s.nq), 64, 0, st>>>(b, lay, s.nq);
-    }
-    return 2;
+    if (s.D == 128) attn_decode_kernel<128><<<grid, kAttnWarps * 32, attn_smem_bytes<128>(), st>>>(tm_k, tm_v, p);
+    else attn_decode_kernel<64><<<grid, kAttnWarps * 32, attn_smem_bytes<64>(), st>>>(tm_k, tm_v, p);
+    return 1;
+}
+
+int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st) {
+    if (s.D == 128) attn_combine_kernel<128><<<dim3(n_tok, s.nq), 128, 0, st>>>(b, lay, s.nq);
+    else attn_combine_kernel<64><<<dim3(n_tok, s.nq), 64, 0, st>>>(b, lay, s.nq);
+    return 1;
 }
 
 cudaError_t init_attn_kernels() {

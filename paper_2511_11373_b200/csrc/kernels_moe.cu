@@ -330,15 +330,21 @@ static void expert_plan(const Shape& s, int n_tok, int* cap, int* warps) {
     while ((size_t)*cap * 2 * x_row_bytes(s.H) > 200u * 1024u && *cap > 4) *cap /= 2;
 }
 
-int launch_experts(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st) {
+int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st) {
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
     dim3 g1((s.I / 16 + warps - 1) / warps, s.E);
     expert_gate_up_kernel<<<g1, warps * 32, (size_t)cap * 2 * x_row_bytes(s.H), st>>>(s, b, w.w_gate_up, cap);
+    return 1;
+}
+
+int launch_down(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st) {
+    int cap, warps;
+    expert_plan(s, n_tok, &cap, &warps);
     const int w2 = warps == kExpMaxWarps ? 8 : warps;
     dim3 g2((s.H / 32 + w2 - 1) / w2, s.E);
     expert_down_kernel<<<g2, w2 * 32, (size_t)cap * 2 * x_row_bytes(s.I), st>>>(s, b, w.w_down, cap);
-    return 2;
+    return 1;
 }
 
 int launch_combine(const Shape& s, const Buffers& b, const __nv_bfloat16* next_gain, float* hidden_tap, int n_tok,

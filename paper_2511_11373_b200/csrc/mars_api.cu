@@ -136,6 +136,11 @@ struct mars_model {
     int next_slot;
     cudaStream_t last_stream;
     mars_step_info_t info;
+    // per-kernel-class timing (mars_profile_enable)
+    bool profiling;
+    std::vector<cudaEvent_t> ev_pool;          // all events ever created
+    size_t ev_used;                            // events handed out since the last read
+    std::vector<int> ev_class;                 // class of every (start, stop) pair handed out
 };
 
 struct SeqState {
@@ -234,6 +239,8 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
     m->max_prefill = max_prefill_tokens;
     m->next_slot = 0;
     m->last_stream = nullptr;
+    m->profiling = false;
+    m->ev_used = 0;
     std::memset(&m->info, 0, sizeof(m->info));
     for (int i = 0; i < kStagingSlots; ++i) { m->staging[i] = nullptr; m->staged[i] = nullptr; }
     auto fail = [&](cudaError_t e) {
@@ -263,6 +270,7 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
 
 mars_status_t mars_model_free(mars_model_t* m) {
     if (!m) return MARS_ERR_BAD_HANDLE;
+    for (cudaEvent_t e : m->ev_pool) cudaEventDestroy(e);
     for (int i = 0; i < kStagingSlots; ++i) {
         if (m->staged[i]) cudaEventDestroy(m->staged[i]);
         if (m->staging[i]) cudaFreeHost(m->staging[i]);
@@ -506,25 +514,53 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     const size_t hid_stride = (size_t)n_tok * s.H;
 
     int launches = 0;
-    launches += launch_prep(s, b, lay, kv->view, n_tok, st);
-    launches += launch_embed(s, b, lay, m->embed, plan.tokens_dev, m->layers[0].attn_norm, taps.hidden, n_tok, st);
+    cudaError_t ev_err = cudaSuccess;
+    // runs one launch wrapper, bracketed by an event pair when profiling is on
+    auto run = [&](int cls, auto&& fn) {
+        cudaEvent_t e0 = nullptr, e1 = nullptr;
+        if (m->profiling && ev_err == cudaSuccess) {
+            while (m->ev_pool.size() < m->ev_used + 2 && ev_err == cudaSuccess) {
+                cudaEvent_t e;
+                ev_err = cudaEventCreate(&e);
+                if (ev_err == cudaSuccess) m->ev_pool.push_back(e);
+            }
+            if (ev_err == cudaSuccess) {
+                e0 = m->ev_pool[m->ev_used];
+                e1 = m->ev_pool[m->ev_used + 1];
+                m->ev_used += 2;
+                m->ev_class.push_back(cls);
+                ev_err = cudaEventRecord(e0, st);
+            }
+        }
+        launches += fn();
+        if (e1 && ev_err == cudaSuccess) ev_err = cudaEventRecord(e1, st);
+    };
+    run(MARS_K_OTHER, [&] { return launch_prep(s, b, lay, kv->view, n_tok, st); });
+    run(MARS_K_OTHER, [&] {
+        return launch_embed(s, b, lay, m->embed, plan.tokens_dev, m->layers[0].attn_norm, taps.hidden, n_tok, st);
+    });
     for (int l = 0; l < s.L; ++l) {
         const LayerW& w = m->layers[l];
-        launches += launch_qkv(s, b, lay, w, kv->view, l, n_tok, st);
-        launches += launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, n_tok, (int)n_items, m->sm_count, st);
-        launches += launch_oproj(s, b, w, n_tok, st);
-        launches += launch_router(s, b, w, taps, l, n_tok, st);
-        launches += launch_experts(s, b, w, n_tok, st);
+        run(MARS_K_QKV, [&] { return launch_qkv(s, b, lay, w, kv->view, l, n_tok, st); });
+        run(MARS_K_ATTN, [&] { return launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st); });
+        run(MARS_K_ATTN_MERGE, [&] { return launch_attn_merge(s, b, lay, n_tok, st); });
+        run(MARS_K_OPROJ, [&] { return launch_oproj(s, b, w, n_tok, st); });
+        run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, st); });
+        run(MARS_K_GATE_UP, [&] { return launch_gate_up(s, b, w, n_tok, st); });
+        run(MARS_K_DOWN, [&] { return launch_down(s, b, w, n_tok, st); });
         const __nv_bfloat16* next_gain = l + 1 < s.L ? m->layers[l + 1].attn_norm : m->final_norm;
-        launches += launch_combine(s, b, next_gain, taps.hidden ? taps.hidden + (size_t)(l + 1) * hid_stride : nullptr,
-                                   n_tok, st);
+        float* tap = taps.hidden ? taps.hidden + (size_t)(l + 1) * hid_stride : nullptr;
+        run(MARS_K_COMBINE, [&] { return launch_combine(s, b, next_gain, tap, n_tok, st); });
     }
     if (n_emit) {
-        launches += launch_lm_head(s, b, lay, m->lm_head, n_emit, st);
+        run(MARS_K_LM_HEAD, [&] { return launch_lm_head(s, b, lay, m->lm_head, n_emit, st); });
         if (dbg && dbg->logits)
             CUDA_TRY(cudaMemcpyAsync(dbg->logits, b.logits, (size_t)n_emit * s.V * 4, cudaMemcpyDeviceToDevice, st));
-        launches += launch_sample(s, b, lay, n_emit, out_tokens, out_logprobs, taps.nucleus_mass, st);
+        run(MARS_K_SAMPLE, [&] {
+            return launch_sample(s, b, lay, n_emit, out_tokens, out_logprobs, taps.nucleus_mass, st);
+        });
     }
+    CUDA_TRY(ev_err);
     CUDA_TRY(cudaGetLastError());
     m->last_stream = st;
     m->info.kernel_launches = launches;
@@ -693,6 +729,27 @@ mars_status_t mars_poll_status(mars_model_t* m) {
     if (word) CUDA_TRY(cudaMemset(m->buf.err, 0, 4));
     if (word & kErrTimeout) return MARS_ERR_TIMEOUT;
     if (word & kErrBadToken) return MARS_ERR_BAD_TOKEN;
+    return MARS_OK;
+}
+
+mars_status_t mars_profile_enable(mars_model_t* m, int32_t enable) {
+    if (!m) return MARS_ERR_BAD_HANDLE;
+    m->profiling = enable != 0;
+    return MARS_OK;
+}
+
+mars_status_t mars_profile_read(mars_model_t* m, double* ms_per_class, int64_t* launches_per_class) {
+    if (!m) return MARS_ERR_BAD_HANDLE;
+    if (!ms_per_class || !launches_per_class) return MARS_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(m->last_stream));
+    for (size_t i = 0; i < m->ev_class.size(); ++i) {
+        float ms = 0.f;
+        CUDA_TRY(cudaEventElapsedTime(&ms, m->ev_pool[2 * i], m->ev_pool[2 * i + 1]));
+        ms_per_class[m->ev_class[i]] += (double)ms;
+        launches_per_class[m->ev_class[i]] += 1;
+    }
+    m->ev_class.clear();
+    m->ev_used = 0;
     return MARS_OK;
 }
 
