@@ -44,7 +44,8 @@ enum {
     MARS_ERR_KV_FULL = 4,      /* no free page / sequence already at max_pages_per_seq              */
     MARS_ERR_TIMEOUT = 5,      /* a bounded device-side wait gave up (seen by mars_poll_status)     */
     MARS_ERR_BAD_HANDLE = 6,   /* unknown sequence slot, double release, page already owned, ...    */
-    MARS_ERR_BAD_TOKEN = 7     /* a token id read on the device was outside [0, vocab)              */
+    MARS_ERR_BAD_TOKEN = 7,    /* a token id read on the device was outside [0, vocab)              */
+    MARS_ERR_TOO_LARGE = 8     /* the request needs more than the built-in scratch array holds      */
 };
 
 /* Model shape.  max_pos bounds context_length + new tokens of any sequence. */
@@ -177,6 +178,43 @@ MARS_API mars_status_t mars_decode_step_host(mars_model_t *model, mars_kv_t *kv,
                                     const int32_t *seq_ids, const int32_t *in_tokens_host,
                                     const mars_sampling_t *sampling, int32_t *out_tokens_host,
                                     float *out_logprobs_host);
+
+/* mars_decode_step_static: one decode step for callers that cannot obtain device memory of their
+ * own.  (The paper has no counterpart; this entry point exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plug-in inside a host
+ * application that hands out the weights and the KV pools but no scratch, a real-time loop that
+ * must not touch the allocator, a process whose memory pool is owned by another framework.  Such
+ * callers cannot provide the workspace that mars_model_load asks for.  This call needs no handle
+ * and no workspace: everything the step needs beyond its inputs and outputs (activations, split-K
+ * attention partials, routing lists, logits) lives in ONE fixed array of MARS_STATIC_SCRATCH_BYTES
+ * compiled into the library image.  Every GPU that loads the library carries that array until the
+ * process exits.  The call itself performs no device or pinned-host allocation and frees nothing.
+ *
+ * Semantics are those of mars_decode_step with sequence b = block-table row b:
+ *   cfg, weights      as for mars_model_load (device pointers, bf16);
+ *   k_pool, v_pool    paged cache [n_layers][n_pages][n_kv_heads][page_size][head_dim], bf16;
+ *   block_table       DEVICE int32 [n_seqs][max_pages_per_seq]; row b must already list the pages
+ *                     that cover positions 0 .. ctx_lens[b] (nothing is taken from a free list);
+ *   ctx_lens          HOST int32 [n_seqs]: tokens already cached; the new token is written at that
+ *                     position and attends over 0 .. ctx_lens[b].  The caller adds 1 afterwards;
+ *   in_tokens / out_tokens / out_logprobs: device arrays of n_seqs entries.
+ * Limits and errors: MARS_ERR_TOO_LARGE when the step's scratch (it grows with n_seqs, vocab,
+ * hidden size and cfg->max_pos) would not fit the built-in array -- nothing is launched;
+ * MARS_ERR_UNSUPPORTED / MARS_ERR_INVALID_ARG as for the handle-based calls.  Token ids that are
+ * out of range are read as token 0 (this call has no status word to poll).
+ * First call on a device: the address of the built-in array is looked up and the kernels' launch
+ * attributes are set, once per device; make that first call outside any stream capture.
+ * Sharing: all calls in the process use the same array, which keeps whatever the previous call
+ * left; the call clears what must start from zero itself.  Two calls that overlap on the GPU (two
+ * streams, two threads) overwrite each other's intermediates: serialise them. */
+#define MARS_STATIC_SCRATCH_BYTES (4u << 20)
+MARS_API mars_status_t mars_decode_step_static(const mars_config_t *cfg, const mars_weights_t *weights, void *k_pool,
+                                      void *v_pool, size_t pool_bytes_each, int32_t page_size,
+                                      const int32_t *block_table, int32_t max_pages_per_seq,
+                                      const int32_t *ctx_lens, void *cuda_stream, int32_t n_seqs,
+                                      const int32_t *in_tokens, const mars_sampling_t *sampling,
+                                      int32_t *out_tokens, float *out_logprobs);
 
 /* Synchronises the stream of the last call and reads the device status word: MARS_OK,
  * MARS_ERR_BAD_TOKEN or MARS_ERR_TIMEOUT; the word is cleared. */

@@ -16,7 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libmars.so")
 
 MARS_OK = 0
 STATUS_NAMES = {0: "MARS_OK", 1: "MARS_ERR_INVALID_ARG", 2: "MARS_ERR_UNSUPPORTED", 3: "MARS_ERR_CUDA",
-                4: "MARS_ERR_KV_FULL", 5: "MARS_ERR_TIMEOUT", 6: "MARS_ERR_BAD_HANDLE", 7: "MARS_ERR_BAD_TOKEN"}
+                4: "MARS_ERR_KV_FULL", 5: "MARS_ERR_TIMEOUT", 6: "MARS_ERR_BAD_HANDLE", 7: "MARS_ERR_BAD_TOKEN",
+                8: "MARS_ERR_TOO_LARGE"}
 LAYER_FIELDS = ("attn_norm", "wqkv", "q_norm", "k_norm", "wo", "mlp_norm", "router", "w_gate_up", "w_down")
 
 
@@ -84,6 +85,9 @@ SIGNATURES = {
                                      POINTER(mars_debug_t)]),
     "mars_decode_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), c_void_p,
                                         POINTER(mars_sampling_t), c_void_p, c_void_p]),
+    "mars_decode_step_static": (c_int32, [POINTER(mars_config_t), POINTER(mars_weights_t), c_void_p, c_void_p, c_size_t,
+                                          c_int32, c_void_p, c_int32, POINTER(c_int32), c_void_p, c_int32, c_void_p,
+                                          POINTER(mars_sampling_t), c_void_p, c_void_p]),
     "mars_poll_status": (c_int32, [c_void_p]),
     "mars_profile_enable": (c_int32, [c_void_p, c_int32]),
     "mars_profile_read": (c_int32, [c_void_p, POINTER(ctypes.c_double), POINTER(c_int64)]),
@@ -308,3 +312,25 @@ def mars_decode_step_host(model: Model, kv: KvCache, seq_ids, in_tokens_host: to
     assert not in_tokens_host.is_cuda and not out_tokens_host.is_cuda and not out_logprobs_host.is_cuda
     return lib().mars_decode_step_host(model.handle, kv.handle, _stream_handle(stream), n, arr, _ptr(in_tokens_host),
                                        byref(sampling), _ptr(out_tokens_host), _ptr(out_logprobs_host))
+
+
+def mars_decode_step_static(model_shape: dict, weights: dict, max_pos: int, k_pool: torch.Tensor, v_pool: torch.Tensor,
+                            page_size: int, block_table: torch.Tensor, ctx_lens, in_tokens: torch.Tensor,
+                            sampling: mars_sampling_t, out_tokens: torch.Tensor, out_logprobs: torch.Tensor,
+                            stream=None) -> int:
+    """Decode step that needs no handle and no workspace (for callers that cannot allocate device
+    memory): its intermediates live in a fixed array inside the library.  `block_table` is a CUDA int32
+    tensor [n_seqs, max_pages_per_seq]; `ctx_lens` a host list.  Returns the status code."""
+    cfg = make_config(model_shape, max_pos)
+    layers = (mars_layer_t * len(weights["layers"]))()
+    for i, layer in enumerate(weights["layers"]):
+        for f in LAYER_FIELDS:
+            setattr(layers[i], f, layer[f].data_ptr())
+    w = mars_weights_t(weights["embed"].data_ptr(), weights["final_norm"].data_ptr(), weights["lm_head"].data_ptr(), layers)
+    lens, n = _i32_array(ctx_lens)
+    assert block_table.is_cuda and block_table.dtype == torch.int32 and block_table.is_contiguous()
+    with torch.cuda.device(k_pool.device):
+        return lib().mars_decode_step_static(byref(cfg), byref(w), _ptr(k_pool), _ptr(v_pool), k_pool.numel() * 2,
+                                             page_size, _ptr(block_table), block_table.shape[1], lens,
+                                             _stream_handle(stream), n, _ptr(in_tokens), byref(sampling),
+                                             _ptr(out_tokens), _ptr(out_logprobs))

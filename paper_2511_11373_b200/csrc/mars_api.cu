@@ -174,6 +174,7 @@ const char* mars_status_string(mars_status_t s) {
         case MARS_ERR_TIMEOUT: return "bounded device wait gave up";
         case MARS_ERR_BAD_HANDLE: return "bad handle or sequence slot";
         case MARS_ERR_BAD_TOKEN: return "token id out of range";
+        case MARS_ERR_TOO_LARGE: return "request exceeds the built-in scratch array (MARS_STATIC_SCRATCH_BYTES)";
         default: return "unknown status";
     }
 }
@@ -718,6 +719,163 @@ mars_status_t mars_decode_step_host(mars_model_t* m, mars_kv_t* kv, void* cuda_s
     CUDA_TRY(cudaMemcpyAsync(out_tokens_host, m->io_out, (size_t)n_seqs * 4, cudaMemcpyDeviceToHost, st));
     CUDA_TRY(cudaMemcpyAsync(out_logprobs_host, m->io_lp, (size_t)n_seqs * 4, cudaMemcpyDeviceToHost, st));
     CUDA_TRY(cudaStreamSynchronize(st));
+    return MARS_OK;
+}
+
+// ------------------------------------------------------------- allocation-free decode step
+// Scratch for mars_decode_step_static.  In host code the name below is only a handle for the
+// runtime; the device address is obtained once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[MARS_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the built-in array for the current device (looked up on first use).
+mars_status_t static_scratch(unsigned char** out) {
+    int dev = 0, major = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return MARS_ERR_UNSUPPORTED;
+    if (!g_static_ptr[dev]) {
+        CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        if (major != 10) return MARS_ERR_UNSUPPORTED;
+        CUDA_TRY(init_dense_kernels());
+        CUDA_TRY(init_attn_kernels());
+        CUDA_TRY(init_moe_kernels());
+        unsigned char* p = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress((void**)&p, g_static_scratch));
+        if (!p) return MARS_ERR_CUDA;
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return MARS_OK;
+}
+}  // namespace
+
+mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weights_t* w, void* k_pool, void* v_pool,
+                                      size_t pool_bytes_each, int32_t page_size, const int32_t* block_table,
+                                      int32_t max_pages_per_seq, const int32_t* ctx_lens, void* cuda_stream,
+                                      int32_t n_seqs, const int32_t* in_tokens, const mars_sampling_t* sampling,
+                                      int32_t* out_tokens, float* out_logprobs) {
+    if (!cfg || !w || !w->layers || !w->embed || !w->final_norm || !w->lm_head || !k_pool || !v_pool || !block_table ||
+        !ctx_lens || !in_tokens || !sampling || !out_tokens || !out_logprobs)
+        return MARS_ERR_INVALID_ARG;
+    if (n_seqs < 1 || max_pages_per_seq < 1) return MARS_ERR_INVALID_ARG;
+    if (page_size != 16 && page_size != 32 && page_size != 64 && page_size != 128) return MARS_ERR_INVALID_ARG;
+    if ((uintptr_t)k_pool % 256 || (uintptr_t)v_pool % 256) return MARS_ERR_INVALID_ARG;
+    if (!sampling->greedy && (!(sampling->temperature > 0.f) || !(sampling->top_p > 0.f) || sampling->top_p > 1.f))
+        return MARS_ERR_INVALID_ARG;
+    if (!shape_supported(*cfg)) return MARS_ERR_UNSUPPORTED;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        const mars_layer_t& s = w->layers[l];
+        if (!s.attn_norm || !s.wqkv || !s.wo || !s.mlp_norm || !s.router || !s.w_gate_up || !s.w_down)
+            return MARS_ERR_INVALID_ARG;
+        if (cfg->qk_norm && (!s.q_norm || !s.k_norm)) return MARS_ERR_INVALID_ARG;
+    }
+    for (int b = 0; b < n_seqs; ++b) {
+        if (ctx_lens[b] < 0 || ctx_lens[b] + 1 > cfg->max_pos) return MARS_ERR_INVALID_ARG;
+        if (ctx_lens[b] / page_size >= max_pages_per_seq) return MARS_ERR_INVALID_ARG;
+    }
+    const size_t page_bytes = (size_t)cfg->n_kv_heads * page_size * cfg->head_dim * 2;
+    const size_t n_pages = pool_bytes_each / page_bytes / cfg->n_layers;
+    if (n_pages < 1 || n_pages > 0x3fffffff) return MARS_ERR_INVALID_ARG;
+    const uint64_t rows = (uint64_t)cfg->n_layers * n_pages * cfg->n_kv_heads * page_size;
+    if (rows > 0x7fffffffull) return MARS_ERR_UNSUPPORTED;
+
+    // everything the step needs must fit the built-in array
+    const Caps caps = make_caps(*cfg, n_seqs, 0);
+    const StepLayout lay = make_layout(caps);
+    const size_t need = carve(*cfg, caps, lay, nullptr, nullptr, nullptr, nullptr, nullptr);
+    if (need > (size_t)MARS_STATIC_SCRATCH_BYTES) return MARS_ERR_TOO_LARGE;
+
+    unsigned char* base = nullptr;
+    mars_status_t rc = static_scratch(&base);
+    if (rc != MARS_OK) return rc;
+    int dev = 0, sms = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    Buffers buf;
+    carve(*cfg, caps, lay, base, &buf, nullptr, nullptr, nullptr);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    CUtensorMap tm_k, tm_v;
+    const int box_rows = std::min(page_size, 64);
+    rc = make_pool_map(&tm_k, k_pool, rows, cfg->head_dim, box_rows);
+    if (rc == MARS_OK) rc = make_pool_map(&tm_v, v_pool, rows, cfg->head_dim, box_rows);
+    if (rc != MARS_OK) return rc;
+
+    // step block (host heap, copied from pageable memory: the runtime stages it before returning)
+    int64_t n_items = 0;
+    for (int b = 0; b < n_seqs; ++b) n_items += (ctx_lens[b] + 1 + kSpanTokens - 1) / kSpanTokens;
+    if (n_items > caps.n_items) return MARS_ERR_TOO_LARGE;
+    std::vector<int32_t> blk((size_t)lay.items + 4 * (size_t)n_items, 0);
+    blk[H_NTOK] = n_seqs;
+    blk[H_NITEMS] = (int32_t)n_items;
+    blk[H_NUPDATES] = 0;
+    blk[H_NEMIT] = n_seqs;
+    blk[H_GREEDY] = sampling->greedy ? 1 : 0;
+    std::memcpy(&blk[H_TEMPERATURE], &sampling->temperature, 4);
+    std::memcpy(&blk[H_TOP_P], &sampling->top_p, 4);
+    blk[H_SEED_LO] = (int32_t)(uint32_t)sampling->seed;
+    blk[H_SEED_HI] = (int32_t)(uint32_t)(sampling->seed >> 32);
+    blk[H_STEP_LO] = (int32_t)(uint32_t)sampling->step;
+    blk[H_STEP_HI] = (int32_t)(uint32_t)(sampling->step >> 32);
+    int at = 0;
+    for (int b = 0; b < n_seqs; ++b) {
+        blk[lay.tok_seq + b] = b;
+        blk[lay.tok_pos + b] = ctx_lens[b];
+        blk[lay.emit_rows + b] = b;
+        blk[lay.emit_slot + b] = b;
+        blk[lay.tok_item_off + b] = at;
+        const int len = ctx_lens[b] + 1;
+        for (int s0 = 0; s0 < len; s0 += kSpanTokens) {
+            blk[lay.items + 4 * at + 0] = b;
+            blk[lay.items + 4 * at + 1] = s0;
+            blk[lay.items + 4 * at + 2] = std::min(kSpanTokens, len - s0);
+            ++at;
+        }
+    }
+    blk[lay.tok_item_off + n_seqs] = at;
+    std::vector<double> inv((size_t)cfg->head_dim / 2);
+    for (int i = 0; i < cfg->head_dim / 2; ++i)
+        inv[i] = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)cfg->head_dim);
+
+    // the array keeps the previous call's contents: clear what the kernels only OR into or count in
+    CUDA_TRY(cudaMemsetAsync(buf.err, 0, 256, st));
+    CUDA_TRY(cudaMemsetAsync(buf.active, 0, (size_t)cfg->n_layers * 4, st));
+    CUDA_TRY(cudaMemcpyAsync(buf.step, blk.data(), blk.size() * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(buf.inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice, st));
+
+    const Shape s{cfg->n_layers, cfg->hidden, cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim, cfg->n_experts,
+                  cfg->top_k, cfg->expert_inter, cfg->vocab, cfg->qk_norm, cfg->rms_eps};
+    const KvView view{(__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, const_cast<int32_t*>(block_table), (int)n_pages,
+                      page_size, max_pages_per_seq};
+    const DebugTaps taps{nullptr, nullptr, nullptr, nullptr, nullptr};
+    auto layer_w = [&](int l) {
+        const mars_layer_t& q = w->layers[l];
+        return LayerW{(const __nv_bfloat16*)q.attn_norm, (const __nv_bfloat16*)q.wqkv, (const __nv_bfloat16*)q.q_norm,
+                      (const __nv_bfloat16*)q.k_norm, (const __nv_bfloat16*)q.wo, (const __nv_bfloat16*)q.mlp_norm,
+                      (const __nv_bfloat16*)q.router, (const __nv_bfloat16*)q.w_gate_up, (const __nv_bfloat16*)q.w_down};
+    };
+    launch_prep(s, buf, lay, view, n_seqs, st);
+    launch_embed(s, buf, lay, (const __nv_bfloat16*)w->embed, in_tokens, (const __nv_bfloat16*)w->layers[0].attn_norm,
+                 nullptr, n_seqs, st);
+    for (int l = 0; l < s.L; ++l) {
+        const LayerW lw = layer_w(l);
+        launch_qkv(s, buf, lay, lw, view, l, n_seqs, st);
+        launch_attention(s, buf, lay, view, tm_k, tm_v, l, sms, st);
+        launch_attn_merge(s, buf, lay, n_seqs, st);
+        launch_oproj(s, buf, lw, n_seqs, st);
+        launch_router(s, buf, lw, taps, l, n_seqs, st);
+        launch_gate_up(s, buf, lw, n_seqs, st);
+        launch_down(s, buf, lw, n_seqs, st);
+        const __nv_bfloat16* next_gain =
+            l + 1 < s.L ? (const __nv_bfloat16*)w->layers[l + 1].attn_norm : (const __nv_bfloat16*)w->final_norm;
+        launch_combine(s, buf, next_gain, nullptr, n_seqs, st);
+    }
+    launch_lm_head(s, buf, lay, (const __nv_bfloat16*)w->lm_head, n_seqs, st);
+    launch_sample(s, buf, lay, n_seqs, out_tokens, out_logprobs, nullptr, st);
+    CUDA_TRY(cudaGetLastError());
     return MARS_OK;
 }
 
