@@ -143,6 +143,40 @@ __device__ __forceinline__ void stream_mma(const __nv_bfloat16* const (&wrow)[MT
     }
 }
 
+// ----- weight stream through a per-warp shared-memory ring ----------------------------------------
+// The same contraction with the A operand staged by cp.async: every thread copies the two 16-byte
+// pieces it will need for a K slice (its row of MMA rows 0..7 and its row of MMA rows 8..15) into a
+// slot of its warp's ring and reads the same two pieces back kRing slices later.  The bytes in
+// flight then live in shared memory instead of registers (a register-staged stream tops out near
+// 8 KB per warp), no other thread ever touches a slot, and consecutive lanes own consecutive 16-byte
+// pieces, so the read-back is free of bank conflicts.  One commit group per slice; a slot is
+// refilled only after the MMAs that consumed it have been issued.
+constexpr int kRing = 8;
+constexpr int kRingStageBytes = 1024;                      // per warp and slice: 2 pieces x 32 lanes x 16 B
+constexpr int kRingWarpBytes = kRing * kRingStageBytes;
+
+__device__ __forceinline__ void ring_issue(unsigned char* warp_ring, int stage, int lane, const __nv_bfloat16* p0,
+                                           const __nv_bfloat16* p1) {
+    unsigned char* d = warp_ring + stage * kRingStageBytes + lane * 16;
+    cp_async16(d, p0);
+    cp_async16(d + 512, p1);
+}
+
+// acc[n] += A(slice) * B(slice, column tile n); xs points at this thread's 16 bytes of column tile 0.
+template <int NT>
+__device__ __forceinline__ void ring_consume(const unsigned char* warp_ring, int stage, int lane, const unsigned char* xs,
+                                             int x_tile_stride, float (&acc)[NT][4]) {
+    const unsigned char* s = warp_ring + stage * kRingStageBytes + lane * 16;
+    const uint4 w0 = *reinterpret_cast<const uint4*>(s);
+    const uint4 w1 = *reinterpret_cast<const uint4*>(s + 512);
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+        const uint4 x = *reinterpret_cast<const uint4*>(xs + (size_t)n * x_tile_stride);
+        mma_16816(acc[n], w0.x, w1.x, w0.y, w1.y, x.x, x.y);
+        mma_16816(acc[n], w0.z, w1.z, w0.w, w1.w, x.z, x.w);
+    }
+}
+
 // Activation rows in shared memory are padded by 64 bytes so that the 16-byte B-fragment reads of
 // a quarter warp (rows gid, gid+1; four 16-byte pieces each) fall into 32 distinct banks.
 __host__ __device__ constexpr int x_row_bytes(int k_elems) { return k_elems * 2 + 64; }

@@ -32,6 +32,8 @@ int launch_embed(const Shape& s, const Buffers& b, const StepLayout& lay, const 
                  const int32_t* tokens, const __nv_bfloat16* first_gain, float* hidden_tap, int n_tok, cudaStream_t st);
 int launch_qkv(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
                int n_tok, cudaStream_t st);
+// K elements per phase, number of K splits (partials) and phases per CTA of the streaming GEMM.
+void gemm_plan(int K, int n_tok, bool many_rows, int* ks, int* ksplit, int* phases);
 int launch_oproj(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
 int launch_lm_head(const Shape& s, const Buffers& b, const StepLayout& lay, const __nv_bfloat16* lm_head, int n_emit,
                    cudaStream_t st);
@@ -42,7 +44,7 @@ int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, i
 
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,
                   cudaStream_t st);
-int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
+int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st);
 int launch_down(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
 int launch_combine(const Shape& s, const Buffers& b, const __nv_bfloat16* next_gain, float* hidden_tap, int n_tok,
                    cudaStream_t st);

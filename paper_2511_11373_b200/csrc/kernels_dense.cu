@@ -93,96 +93,110 @@ int launch_embed(const Shape& s, const Buffers& b, const StepLayout&, const __nv
 }
 
 // ---------------------------------------------------------------------------------------------
-// Y^T = W X^T for up to 64 tokens per block column: weights streamed once from HBM, activations
-// (hi/lo pairs = 128 columns) staged through shared memory in K chunks (double buffered, cp.async).
-constexpr int kGemmWarps = 4;
+// Y^T = W X^T for up to 64 tokens per block: a CTA owns 128 weight rows (8 warps x 16) and a range
+// of K.  The activations of that K range (hi/lo pairs = 128 columns) sit in shared memory, one
+// phase of at most 512 elements at a time; the weights stream once from HBM through the per-warp
+// cp.async rings and keep streaming while a phase's activations are swapped.  With split-K
+// (gridDim.y > 1) every K range writes its own fp32 partial [ksplit][tokens][rows]; the consumer
+// kernel adds the partials in a fixed order, so results do not depend on scheduling.
+constexpr int kGemmWarps = 8;
 constexpr int kGemmTok = 64;
 constexpr int kGemmCols = 2 * kGemmTok;
 constexpr int kGemmNT = kGemmCols / 8;
-constexpr int kGemmKC = 256;
-constexpr int kGemmXBytes = kGemmCols * x_row_bytes(kGemmKC);
-
-enum { EPI_STORE = 0, EPI_RESID = 1 };
+constexpr int kGemmMaxKS = 512;
 
 struct GemmParams {
     const __nv_bfloat16* W;     // [rows, K]
     const __nv_bfloat16* X;     // [*, 2, K] (hi row, lo row per token)
     const int32_t* row_index;   // optional: X token of output token t is row_index[t]
-    float* out;                 // [n_tok, rows]
+    float* out;                 // [ksplit, n_tok, rows]
     int rows, K, n_tok;
+    int ks;                     // K elements per phase (multiple of 64, <= 512)
+    int phases;                 // phases per CTA; gridDim.y * phases * ks == K
 };
 
-template <int EPI>
-__global__ void __launch_bounds__(kGemmWarps * 32) dense_gemm_kernel(GemmParams p) {
+static size_t gemm_smem_bytes(int ks) { return (size_t)kGemmCols * x_row_bytes(ks) + (size_t)kGemmWarps * kRingWarpBytes; }
+
+__global__ void __launch_bounds__(kGemmWarps * 32, 1) stream_gemm_kernel(GemmParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, tig = lane & 3;
+    const int xrow = x_row_bytes(p.ks);
+    unsigned char* xt = smem;
+    unsigned char* ring = smem + (size_t)kGemmCols * xrow + (size_t)warp * kRingWarpBytes;
     const int row_base = (blockIdx.x * kGemmWarps + warp) * 16;
-    const int tok0 = blockIdx.y * kGemmTok;
+    const int tok0 = blockIdx.z * kGemmTok;
     const int n_here = min(kGemmTok, p.n_tok - tok0);
-    constexpr int xrow = x_row_bytes(kGemmKC);
+    const int k_begin = blockIdx.y * p.phases * p.ks;
+    const int slices_per_phase = p.ks / 32;
+    const int total_slices = p.phases * slices_per_phase;
 
     const int r0 = min(row_base + gid, p.rows - 1), r1 = min(row_base + gid + 8, p.rows - 1);
-    const __nv_bfloat16* wrow[1][2] = {{p.W + (size_t)r0 * p.K + tig * 8, p.W + (size_t)r1 * p.K + tig * 8}};
+    const __nv_bfloat16* w0 = p.W + (size_t)r0 * p.K + k_begin + tig * 8;
+    const __nv_bfloat16* w1 = p.W + (size_t)r1 * p.K + k_begin + tig * 8;
 
-    auto load_chunk = [&](int c, int buf) {
-        unsigned char* dst = smem + (size_t)buf * kGemmXBytes;
-        constexpr int pieces = kGemmKC * 2 / 16;  // 16-byte pieces per row
-        for (int i = threadIdx.x; i < kGemmCols * pieces; i += blockDim.x) {
-            const int v = i / pieces, pc = i - v * pieces;     // v: column = 2 * token + plane
-            unsigned char* d = dst + (size_t)v * xrow + pc * 16;
-            const int t = v >> 1;
-            if (t < n_here) {
-                const int src_tok = p.row_index ? p.row_index[tok0 + t] : tok0 + t;
-                cp_async16(d, p.X + ((size_t)src_tok * 2 + (v & 1)) * p.K + (size_t)c * kGemmKC + pc * 8);
-            } else {
-                *reinterpret_cast<uint4*>(d) = make_uint4(0, 0, 0, 0);
-            }
-        }
-    };
-
-    float acc[1][kGemmNT][4];
+    // prime the ring: slices 0 .. kRing-1 (one commit group each, empty past the end)
 #pragma unroll
-    for (int n = 0; n < kGemmNT; ++n)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[0][n][j] = 0.f;
-
-    const int n_chunks = p.K / kGemmKC;   // K is a multiple of kGemmKC (checked on the host)
-    load_chunk(0, 0);
-    cp_async_commit();
-    for (int c = 0; c < n_chunks; ++c) {
-        if (c + 1 < n_chunks) {
-            load_chunk(c + 1, (c + 1) & 1);
-            cp_async_commit();
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
-        __syncthreads();
-        const __nv_bfloat16* wr[1][2] = {{wrow[0][0] + (size_t)c * kGemmKC, wrow[0][1] + (size_t)c * kGemmKC}};
-        const unsigned char* xs = smem + (size_t)(c & 1) * kGemmXBytes + (size_t)gid * xrow + tig * 16;
-        stream_mma<1, kGemmNT, 4>(wr, kGemmKC / 32, xs, 8 * xrow, acc);
-        __syncthreads();
+    for (int i = 0; i < kRing; ++i) {
+        if (i < total_slices) ring_issue(ring, i, lane, w0 + (size_t)i * 32, w1 + (size_t)i * 32);
+        cp_async_commit();
     }
 
+    float acc[kGemmNT][4];
+#pragma unroll
+    for (int n = 0; n < kGemmNT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+
+    const int pieces = p.ks / 8;   // 16-byte pieces per activation row
+    for (int ph = 0; ph < p.phases; ++ph) {
+        if (ph > 0) __syncthreads();             // every warp is done with the previous phase's activations
+        for (int i = threadIdx.x; i < kGemmCols * pieces; i += blockDim.x) {
+            const int v = i / pieces, pc = i - v * pieces;     // v: column = 2 * token + plane
+            const int t = v >> 1;
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if (t < n_here) {
+                const int src_tok = p.row_index ? p.row_index[tok0 + t] : tok0 + t;
+                val = *reinterpret_cast<const uint4*>(p.X + ((size_t)src_tok * 2 + (v & 1)) * p.K + k_begin +
+                                                      (size_t)ph * p.ks + pc * 8);
+            }
+            *reinterpret_cast<uint4*>(xt + (size_t)v * xrow + pc * 16) = val;
+        }
+        __syncthreads();
+        const unsigned char* xs = xt + (size_t)gid * xrow + tig * 16;
+        for (int sl = 0; sl < slices_per_phase; ++sl) {
+            const int s = ph * slices_per_phase + sl;
+            cp_async_wait<kRing - 1>();
+            ring_consume<kGemmNT>(ring, s % kRing, lane, xs + (size_t)sl * 64, 8 * xrow, acc);
+            const int nx = s + kRing;
+            if (nx < total_slices) ring_issue(ring, s % kRing, lane, w0 + (size_t)nx * 32, w1 + (size_t)nx * 32);
+            cp_async_commit();
+        }
+    }
+
+    float* out = p.out + (size_t)blockIdx.y * p.n_tok * p.rows;
 #pragma unroll
     for (int n = 0; n < kGemmNT; ++n)
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
             const int row = row_base + gid + hf * 8;
             const int t = n * 4 + tig;
-            if (row < p.rows && t < n_here) {
-                const float v = acc[0][n][2 * hf] + acc[0][n][2 * hf + 1];   // hi column + lo column
-                float* dst = p.out + (size_t)(tok0 + t) * p.rows + row;
-                if (EPI == EPI_RESID) *dst += v;
-                else *dst = v;
-            }
+            if (row < p.rows && t < n_here)
+                out[(size_t)(tok0 + t) * p.rows + row] = acc[n][2 * hf] + acc[n][2 * hf + 1];   // hi + lo column
         }
 }
 
-template <int EPI>
-static int launch_gemm(const GemmParams& p, cudaStream_t st) {
-    dim3 grid((p.rows + kGemmWarps * 16 - 1) / (kGemmWarps * 16), (p.n_tok + kGemmTok - 1) / kGemmTok);
-    dense_gemm_kernel<EPI><<<grid, kGemmWarps * 32, 2 * kGemmXBytes, st>>>(p);
+// K range per phase and the number of K splits: split-K only pays (and only fits its partial
+// buffer) for decode-sized token counts and matrices with few rows.
+void gemm_plan(int K, int n_tok, bool many_rows, int* ks, int* ksplit, int* phases) {
+    *ks = (K % kGemmMaxKS == 0) ? kGemmMaxKS : 256;      // K is a multiple of 256
+    const int n_ph = K / *ks;
+    if (n_tok <= kGemmTok && !many_rows) { *ksplit = n_ph; *phases = 1; }
+    else { *ksplit = 1; *phases = n_ph; }
+}
+
+static int launch_gemm(GemmParams p, bool many_rows, cudaStream_t st) {
+    int ksplit;
+    gemm_plan(p.K, p.n_tok, many_rows, &p.ks, &ksplit, &p.phases);
+    dim3 grid((p.rows + kGemmWarps * 16 - 1) / (kGemmWarps * 16), ksplit, (p.n_tok + kGemmTok - 1) / kGemmTok);
+    stream_gemm_kernel<<<grid, kGemmWarps * 32, gemm_smem_bytes(p.ks), st>>>(p);
     return 1;
 }
 
@@ -193,7 +207,7 @@ static int launch_gemm(const GemmParams& p, cudaStream_t st) {
 template <int D>
 __global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepLayout lay, KvView kv,
                                                        const __nv_bfloat16* q_gain, const __nv_bfloat16* k_gain,
-                                                       int layer) {
+                                                       int layer, int ksplit, int n_tok) {
     constexpr int HALF = D / 2, PER = HALF / 32;
     const int t = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_heads = s.nq + 2 * s.nkv;
@@ -207,8 +221,12 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepL
         float ss = 0.f;
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
-            lo[i] = raw[head * D + lane + 32 * i];
-            hi[i] = raw[head * D + lane + 32 * i + HALF];
+            lo[i] = hi[i] = 0.f;
+            for (int sp = 0; sp < ksplit; ++sp) {      // split-K partials, fixed order
+                const float* part = raw + (size_t)sp * n_tok * n_heads * D;
+                lo[i] += part[head * D + lane + 32 * i];
+                hi[i] += part[head * D + lane + 32 * i + HALF];
+            }
             ss += lo[i] * lo[i] + hi[i] * hi[i];
         }
         if (!is_q && !is_k) {  // value head: stored as is
@@ -253,30 +271,32 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepL
 
 int launch_qkv(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
                int n_tok, cudaStream_t st) {
-    GemmParams p{w.wqkv, b.h, nullptr, b.qkv, (s.nq + 2 * s.nkv) * s.D, s.H, n_tok};
-    int n = launch_gemm<EPI_STORE>(p, st);
-    if (s.D == 128) qkv_post_kernel<128><<<n_tok, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer);
-    else qkv_post_kernel<64><<<n_tok, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer);
+    GemmParams p{w.wqkv, b.h, nullptr, b.qkv, (s.nq + 2 * s.nkv) * s.D, s.H, n_tok, 0, 0};
+    int n = launch_gemm(p, false, st);
+    int ks, ksplit, phases;
+    gemm_plan(s.H, n_tok, false, &ks, &ksplit, &phases);
+    if (s.D == 128)
+        qkv_post_kernel<128><<<n_tok, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
+    else
+        qkv_post_kernel<64><<<n_tok, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
     return n + 1;
 }
 
+// Output projection: writes split-K partials of W_o o; the router kernel adds them to the residual.
 int launch_oproj(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st) {
-    GemmParams p{w.wo, b.o, nullptr, b.x, s.H, s.nq * s.D, n_tok};
-    return launch_gemm<EPI_RESID>(p, st);
+    GemmParams p{w.wo, b.o, nullptr, b.opart, s.H, s.nq * s.D, n_tok, 0, 0};
+    return launch_gemm(p, false, st);
 }
 
 int launch_lm_head(const Shape& s, const Buffers& b, const StepLayout& lay, const __nv_bfloat16* lm_head, int n_emit,
                    cudaStream_t st) {
-    GemmParams p{lm_head, b.h, b.step + lay.emit_rows, b.logits, s.V, s.H, n_emit};
-    return launch_gemm<EPI_STORE>(p, st);
+    GemmParams p{lm_head, b.h, b.step + lay.emit_rows, b.logits, s.V, s.H, n_emit, 0, 0};
+    return launch_gemm(p, true, st);
 }
 
 cudaError_t init_dense_kernels() {
-    cudaError_t e = cudaFuncSetAttribute(dense_gemm_kernel<EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         2 * kGemmXBytes);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(dense_gemm_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                2 * kGemmXBytes);
+    return cudaFuncSetAttribute(stream_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)gemm_smem_bytes(kGemmMaxKS));
 }
 
 }  // namespace mars

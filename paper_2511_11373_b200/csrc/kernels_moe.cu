@@ -17,40 +17,61 @@ constexpr int kMaxTopK = 32;
 // pi (ties: lower index) and their renormalised weights.
 __global__ void __launch_bounds__(kRouterThreads) router_kernel(Shape s, Buffers b, const __nv_bfloat16* gain,
                                                                 const __nv_bfloat16* Wr, DebugTaps dbg, int layer,
-                                                                int n_tok) {
-    extern __shared__ float hs[];          // [H] normalised activations
+                                                                int n_tok, int o_ksplit) {
+    // one column tile of activations: row 0 = hi, row 1 = lo of this token, rows 2..7 zero
+    extern __shared__ __align__(16) unsigned char xt[];
     __shared__ float scratch[32];
     __shared__ float z[kMaxExperts];
-    const int t = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int t = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tig = lane & 3;
     const int H = s.H, E = s.E, k = s.k;
+    const int xrow = x_row_bytes(H);
 
+    // residual: x += W_o o, delivered as split-K partials that are added here in a fixed order
+    float v[kRowMaxPer];
     float ss = 0.f;
-    for (int c = tid; c < H; c += kRouterThreads) {
-        const float v = b.x[(size_t)t * H + c];
-        hs[c] = v;
-        ss += v * v;
+#pragma unroll
+    for (int i = 0; i < kRowMaxPer; ++i) {
+        const int c = tid + i * kRouterThreads;
+        v[i] = 0.f;
+        if (c < H) {
+            float acc = b.x[(size_t)t * H + c];
+            for (int sp = 0; sp < o_ksplit; ++sp) acc += b.opart[((size_t)sp * n_tok + t) * H + c];
+            b.x[(size_t)t * H + c] = acc;
+            v[i] = acc;
+            ss += acc * acc;
+        }
     }
     ss = block_sum(ss, scratch);
     const float r = rsqrtf(ss / (float)H + s.eps);
-    for (int c = tid; c < H; c += kRouterThreads) {
-        const float v = hs[c] * r * __bfloat162float(gain[c]);
-        hs[c] = v;
-        split_bf16(v, b.h[(size_t)t * 2 * H + c], b.h[(size_t)t * 2 * H + H + c]);
+#pragma unroll
+    for (int i = 0; i < kRowMaxPer; ++i) {
+        const int c = tid + i * kRouterThreads;
+        if (c < H) {
+            __nv_bfloat16 hi, lo;
+            split_bf16(v[i] * r * __bfloat162float(gain[c]), hi, lo);
+            b.h[(size_t)t * 2 * H + c] = hi;
+            b.h[(size_t)t * 2 * H + H + c] = lo;
+            reinterpret_cast<__nv_bfloat16*>(xt)[c] = hi;
+            reinterpret_cast<__nv_bfloat16*>(xt + xrow)[c] = lo;
+        }
+    }
+    for (int i = tid; i < 6 * (H / 8); i += kRouterThreads) {
+        const int rw = 2 + i / (H / 8), pc = i % (H / 8);
+        *reinterpret_cast<uint4*>(xt + (size_t)rw * xrow + pc * 16) = make_uint4(0, 0, 0, 0);
     }
     __syncthreads();
 
-    for (int e = warp; e < E; e += kRouterThreads / 32) {
-        const __nv_bfloat16* w = Wr + (size_t)e * H;
-        float acc = 0.f;
-        for (int c = lane * 8; c < H; c += 256) {
-            const uint4 v = *reinterpret_cast<const uint4*>(w + c);
-            acc = fmaf(bf16_lo(v.x), hs[c], acc);     acc = fmaf(bf16_hi(v.x), hs[c + 1], acc);
-            acc = fmaf(bf16_lo(v.y), hs[c + 2], acc); acc = fmaf(bf16_hi(v.y), hs[c + 3], acc);
-            acc = fmaf(bf16_lo(v.z), hs[c + 4], acc); acc = fmaf(bf16_hi(v.z), hs[c + 5], acc);
-            acc = fmaf(bf16_lo(v.w), hs[c + 6], acc); acc = fmaf(bf16_hi(v.w), hs[c + 7], acc);
+    // gate logits with the streaming contraction: 16 experts per warp pass, columns 0/1 = hi/lo.
+    // The (hi, lo) pair carries ~16 mantissa bits of h2 and the sum is kept in fp32.
+    for (int rb = warp; rb * 16 < E; rb += kRouterThreads / 32) {
+        const int r0 = min(rb * 16 + gid, E - 1), r1 = min(rb * 16 + gid + 8, E - 1);
+        const __nv_bfloat16* wrow[1][2] = {{Wr + (size_t)r0 * H + tig * 8, Wr + (size_t)r1 * H + tig * 8}};
+        float acc[1][1][4] = {{{0.f, 0.f, 0.f, 0.f}}};
+        stream_mma<1, 1, 8>(wrow, H / 32, xt + (size_t)gid * xrow + tig * 16, 8 * xrow, acc);
+        if (tig == 0) {
+            if (rb * 16 + gid < E) z[rb * 16 + gid] = acc[0][0][0] + acc[0][0][1];
+            if (rb * 16 + gid + 8 < E) z[rb * 16 + gid + 8] = acc[0][0][2] + acc[0][0][3];
         }
-        acc = warp_sum(acc);
-        if (lane == 0) z[e] = acc;
     }
     __syncthreads();
 
@@ -109,7 +130,7 @@ __global__ void __launch_bounds__(kRouterThreads) router_kernel(Shape s, Buffers
 // Token permutation: histogram of expert ids, exclusive offsets, and for every expert the list of
 // token rows it serves (slot order inside an expert is arbitrary: every (token, expert) product is
 // computed independently of its slot).  Single block; also counts the distinct experts used.
-__global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int layer, int n_pairs) {
+__global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int layer, int n_pairs, int tok_cap) {
     __shared__ int cnt[kMaxExperts];
     __shared__ int off[kMaxExperts + 1];
     const int tid = threadIdx.x, E = s.E;
@@ -126,6 +147,17 @@ __global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int l
         }
         off[E] = acc;
         b.active[layer] = active;
+        // token groups for the expert kernels: (expert, first slot, tokens <= tok_cap, 0)
+        int ng = 0;
+        for (int e = 0; e < E; ++e)
+            for (int t0 = 0; t0 < cnt[e]; t0 += tok_cap) {
+                b.groups[4 * ng + 0] = e;
+                b.groups[4 * ng + 1] = off[e] + t0;
+                b.groups[4 * ng + 2] = min(tok_cap, cnt[e] - t0);
+                b.groups[4 * ng + 3] = 0;
+                ++ng;
+            }
+        *b.n_groups = ng;
     }
     __syncthreads();
     for (int e = tid; e <= E; e += blockDim.x) b.expert_off[e] = off[e];
@@ -140,77 +172,143 @@ __global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int l
 }
 
 // ---------------------------------------------------------------------------------------------
-// Grouped SwiGLU, first half: act[slot, i] = silu(<W_gate[e, i], h>) * <W_up[e, i], h> for the
-// tokens of expert e.  grid = (row blocks, experts); a warp owns 16 gate rows and the matching 16
-// up rows and streams them once over the full K; the expert's activation rows sit in shared memory.
+// Grouped SwiGLU, first half: act[slot, i] = silu(<W_gate[e, i], h>) * <W_up[e, i], h>.
+//
+// Work is cut into units of 8 gate rows + the matching 8 up rows of one token group (an expert and
+// at most `cap` of its tokens, listed by the permute kernel).  A unit is one MMA row tile: gate rows
+// on MMA rows 0..7, up rows on rows 8..15, so silu(gate) * up pairs up inside a thread.  The grid is
+// persistent (one CTA per SM); CTA c owns the contiguous range [c U / G, (c+1) U / G) of the U
+// units, i.e. parts of two or three groups, and walks it group by group: the group's activation
+// rows are put in shared memory, then warp w takes the group's units w, w + W, ...  Each warp
+// streams its weight rows through its own cp.async ring, and the ring keeps filling across unit
+// and group boundaries, so the stream into an SM only pauses while a group's activations load.
+constexpr int kGuMaxWarps = 16;
 constexpr int kExpMaxWarps = 12;
 
+struct GuCursor {               // position of a warp in its sequence of (group, unit, slice)
+    int g, u, sl;
+    const __nv_bfloat16 *p0, *p1;
+};
+
 template <int NT>
-__device__ __forceinline__ void gate_up_tile(const __nv_bfloat16* Wg, const __nv_bfloat16* Wu, int H, int I,
-                                             int row_base, const unsigned char* xs_base, int xrow, int m_here,
-                                             __nv_bfloat16* act_out /* slot t0 of this expert, [slot][2][I] */,
-                                             int lane) {
-    const int gid = lane >> 2, tig = lane & 3;
-    const __nv_bfloat16* wrow[2][2] = {
-        {Wg + (size_t)(row_base + gid) * H + tig * 8, Wg + (size_t)(row_base + gid + 8) * H + tig * 8},
-        {Wu + (size_t)(row_base + gid) * H + tig * 8, Wu + (size_t)(row_base + gid + 8) * H + tig * 8}};
-    float acc[2][NT][4];
+__device__ __forceinline__ void gate_up_epilogue(const float (&acc)[NT][4], int m_here, int row, int I,
+                                                 __nv_bfloat16* act_out, int tig) {
 #pragma unroll
-    for (int m = 0; m < 2; ++m)
-#pragma unroll
-        for (int n = 0; n < NT; ++n) acc[m][n][0] = acc[m][n][1] = acc[m][n][2] = acc[m][n][3] = 0.f;
-    stream_mma<2, NT, 4>(wrow, H / 32, xs_base + (size_t)gid * xrow + tig * 16, 8 * xrow, acc);
-#pragma unroll
-    for (int n = 0; n < NT; ++n)
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-            const int row = row_base + gid + hf * 8;
-            const int t = n * 4 + tig;                 // columns 2t (hi) and 2t+1 (lo) of token t
-            if (t < m_here) {
-                const float gte = acc[0][n][2 * hf] + acc[0][n][2 * hf + 1];
-                const float up = acc[1][n][2 * hf] + acc[1][n][2 * hf + 1];
-                __nv_bfloat16* dst = act_out + (size_t)t * 2 * I + row;
-                split_bf16(gte / (1.f + expf(-gte)) * up, dst[0], dst[I]);
-            }
+    for (int n = 0; n < NT; ++n) {
+        const int t = n * 4 + tig;                 // columns 2t (hi) and 2t+1 (lo) of token t
+        if (t < m_here) {
+            const float gte = acc[n][0] + acc[n][1], up = acc[n][2] + acc[n][3];
+            __nv_bfloat16* dst = act_out + (size_t)t * 2 * I + row;
+            split_bf16(gte / (1.f + expf(-gte)) * up, dst[0], dst[I]);
         }
+    }
 }
 
-__global__ void __launch_bounds__(kExpMaxWarps * 32) expert_gate_up_kernel(Shape s, Buffers b, const __nv_bfloat16* Wgu,
-                                                                        int tok_cap) {
+__global__ void __launch_bounds__(kGuMaxWarps * 32, 1) expert_gate_up_kernel(Shape s, Buffers b, const __nv_bfloat16* Wgu,
+                                                                          int tok_cap) {
     extern __shared__ __align__(128) unsigned char smem[];
-    const int e = blockIdx.y;
-    const int o0 = b.expert_off[e], m = b.expert_off[e + 1] - o0;
-    if (m == 0) return;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tig = lane & 3;
     const int H = s.H, I = s.I;
-    const int row_base = (blockIdx.x * (blockDim.x >> 5) + warp) * 16;
-    const bool row_ok = row_base < I;       // I is a multiple of 16
+    const int n_warps = blockDim.x >> 5;
     const int xrow = x_row_bytes(H);
-    const __nv_bfloat16* Wg = Wgu + (size_t)e * 2 * I * H;
-    const __nv_bfloat16* Wu = Wg + (size_t)I * H;
-    const int pieces = H / 8;
-    for (int t0 = 0; t0 < m; t0 += tok_cap) {
-        const int m_here = min(tok_cap, m - t0);
-        const int cols_ld = (2 * m_here + 7) & ~7;      // column v = 2 * token + plane
-        for (int i = threadIdx.x; i < cols_ld * pieces; i += blockDim.x) {
-            const int v = i / pieces, pc = i - v * pieces;
-            unsigned char* d = smem + (size_t)v * xrow + pc * 16;
-            if ((v >> 1) < m_here)
-                cp_async16(d, b.h + ((size_t)b.slot_token[o0 + t0 + (v >> 1)] * 2 + (v & 1)) * H + pc * 8);
-            else *reinterpret_cast<uint4*>(d) = make_uint4(0, 0, 0, 0);
+    unsigned char* xt = smem;
+    unsigned char* ring = smem + (size_t)2 * tok_cap * xrow + (size_t)warp * kRingWarpBytes;
+    const int4* groups = reinterpret_cast<const int4*>(b.groups);
+    const int n_groups = *b.n_groups;
+    const int upe = I / 8;                                   // units per group
+    const long long total = (long long)n_groups * upe;
+    const int u_begin = (int)(total * blockIdx.x / gridDim.x), u_end = (int)(total * (blockIdx.x + 1) / gridDim.x);
+    if (u_begin >= u_end) return;
+    const int g_first = u_begin / upe, g_last = (u_end - 1) / upe;
+    const int n_slices = H / 32;
+
+    auto seg_lo = [&](int g) { return max(u_begin, g * upe); };
+    auto seg_hi = [&](int g) { return min(u_end, (g + 1) * upe); };
+    // move the cursor to the warp's next unit at or after (g, u) and set its weight row pointers
+    auto settle = [&](GuCursor& c) {
+        while (c.g <= g_last && c.u >= seg_hi(c.g)) {
+            ++c.g;
+            if (c.g <= g_last) c.u = seg_lo(c.g) + warp;
+        }
+        if (c.g <= g_last) {
+            const int e = groups[c.g].x;
+            const int row = (c.u - c.g * upe) * 8 + gid;
+            c.p0 = Wgu + ((size_t)e * 2 * I + row) * H + tig * 8;
+            c.p1 = c.p0 + (size_t)I * H;
+        }
+    };
+    GuCursor ic;
+    ic.g = g_first; ic.u = seg_lo(g_first) + warp; ic.sl = 0; ic.p0 = ic.p1 = nullptr;
+    settle(ic);
+    int icount = 0, ccount = 0;
+    auto issue_next = [&]() {                                // one slice (or nothing) and one commit group
+        if (ic.g <= g_last) {
+            ring_issue(ring, icount % kRing, lane, ic.p0 + (size_t)ic.sl * 32, ic.p1 + (size_t)ic.sl * 32);
+            if (++ic.sl == n_slices) {
+                ic.sl = 0;
+                ic.u += n_warps;
+                settle(ic);
+            }
         }
         cp_async_commit();
-        cp_async_wait<0>();
-        __syncthreads();
-        if (row_ok) {
-            __nv_bfloat16* out = b.act + (size_t)(o0 + t0) * 2 * I;
-            const int nt = (m_here + 3) >> 2;
-            if (nt == 1) gate_up_tile<1>(Wg, Wu, H, I, row_base, smem, xrow, m_here, out, lane);
-            else if (nt == 2) gate_up_tile<2>(Wg, Wu, H, I, row_base, smem, xrow, m_here, out, lane);
-            else gate_up_tile<4>(Wg, Wu, H, I, row_base, smem, xrow, m_here, out, lane);
+        ++icount;
+    };
+#pragma unroll 1
+    for (int i = 0; i < kRing; ++i) issue_next();
+
+    const int pieces = H / 8;
+    for (int g = g_first; g <= g_last; ++g) {
+        const int4 grp = groups[g];                          // (expert, first slot, tokens, 0)
+        const int m_here = grp.z;
+        if (g > g_first) __syncthreads();                    // everyone is done with the previous group's rows
+        const int cols_ld = (2 * m_here + 7) & ~7;           // column v = 2 * token + plane
+        for (int i = tid; i < cols_ld * pieces; i += blockDim.x) {
+            const int v = i / pieces, pc = i - v * pieces;
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if ((v >> 1) < m_here)
+                val = *reinterpret_cast<const uint4*>(b.h + ((size_t)b.slot_token[grp.y + (v >> 1)] * 2 + (v & 1)) * H +
+                                                      pc * 8);
+            *reinterpret_cast<uint4*>(xt + (size_t)v * xrow + pc * 16) = val;
         }
         __syncthreads();
+        const unsigned char* xs = xt + (size_t)gid * xrow + tig * 16;
+        __nv_bfloat16* act_out = b.act + (size_t)grp.y * 2 * I;
+        const int nt = (m_here + 3) >> 2;
+        for (int u = seg_lo(g) + warp; u < seg_hi(g); u += n_warps) {
+            const int row = (u - g * upe) * 8 + gid;
+            if (nt == 1) {
+                float acc[1][4] = {{0.f, 0.f, 0.f, 0.f}};
+                for (int sl = 0; sl < n_slices; ++sl) {
+                    cp_async_wait<kRing - 1>();
+                    ring_consume<1>(ring, ccount % kRing, lane, xs + (size_t)sl * 64, 8 * xrow, acc);
+                    ++ccount;
+                    issue_next();
+                }
+                gate_up_epilogue<1>(acc, m_here, row, I, act_out, tig);
+            } else if (nt == 2) {
+                float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                for (int sl = 0; sl < n_slices; ++sl) {
+                    cp_async_wait<kRing - 1>();
+                    ring_consume<2>(ring, ccount % kRing, lane, xs + (size_t)sl * 64, 8 * xrow, acc);
+                    ++ccount;
+                    issue_next();
+                }
+                gate_up_epilogue<2>(acc, m_here, row, I, act_out, tig);
+            } else {
+                float acc[4][4];
+#pragma unroll
+                for (int n = 0; n < 4; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+                for (int sl = 0; sl < n_slices; ++sl) {
+                    cp_async_wait<kRing - 1>();
+                    ring_consume<4>(ring, ccount % kRing, lane, xs + (size_t)sl * 64, 8 * xrow, acc);
+                    ++ccount;
+                    issue_next();
+                }
+                gate_up_epilogue<4>(acc, m_here, row, I, act_out, tig);
+            }
+        }
     }
+    cp_async_wait<0>();
 }
 
 // Second half: y[slot, r] = <W_down[e, r], act[slot]>.  A warp owns 32 output rows (two M tiles).
@@ -286,62 +384,87 @@ __global__ void __launch_bounds__(kRouterThreads) combine_kernel(Shape s, Buffer
     const int t = blockIdx.x, tid = threadIdx.x, H = s.H, k = s.k;
     if (tid < k) { slots[tid] = b.slot_of[(size_t)t * k + tid]; ws[tid] = b.route_w[(size_t)t * k + tid]; }
     __syncthreads();
-    float v[kRowMaxPer];
+    // four columns per thread and visit; the k expert rows are fetched eight at a time so that the
+    // loads are in flight together, and added in the order j = 0, 1, ...
+    constexpr int kVec = kRowMaxPer / 4;
+    float4 v[kVec];
     float ss = 0.f;
 #pragma unroll
-    for (int i = 0; i < kRowMaxPer; ++i) {
-        const int c = tid + i * kRouterThreads;
-        v[i] = 0.f;
+    for (int i = 0; i < kVec; ++i) {
+        const int c = (tid + i * kRouterThreads) * 4;
+        v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (c < H) {
-            float acc = b.x[(size_t)t * H + c];
-            for (int j = 0; j < k; ++j) acc = fmaf(ws[j], b.y[(size_t)slots[j] * H + c], acc);
+            float4 acc = *reinterpret_cast<const float4*>(b.x + (size_t)t * H + c);
+            for (int j0 = 0; j0 < k; j0 += 8) {
+                float4 yv[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    yv[j] = j0 + j < k ? *reinterpret_cast<const float4*>(b.y + (size_t)slots[j0 + j] * H + c)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float wj = j0 + j < k ? ws[j0 + j] : 0.f;
+                    acc.x = fmaf(wj, yv[j].x, acc.x); acc.y = fmaf(wj, yv[j].y, acc.y);
+                    acc.z = fmaf(wj, yv[j].z, acc.z); acc.w = fmaf(wj, yv[j].w, acc.w);
+                }
+            }
             v[i] = acc;
-            b.x[(size_t)t * H + c] = acc;
-            if (hidden_tap) hidden_tap[(size_t)t * H + c] = acc;
-            ss += acc * acc;
+            *reinterpret_cast<float4*>(b.x + (size_t)t * H + c) = acc;
+            if (hidden_tap) *reinterpret_cast<float4*>(hidden_tap + (size_t)t * H + c) = acc;
+            ss += acc.x * acc.x + acc.y * acc.y + acc.z * acc.z + acc.w * acc.w;
         }
     }
     ss = block_sum(ss, scratch);
     const float r = rsqrtf(ss / (float)H + s.eps);
 #pragma unroll
-    for (int i = 0; i < kRowMaxPer; ++i) {
-        const int c = tid + i * kRouterThreads;
-        if (c < H)
-            split_bf16(v[i] * r * __bfloat162float(next_gain[c]), b.h[(size_t)t * 2 * H + c],
-                       b.h[(size_t)t * 2 * H + H + c]);
+    for (int i = 0; i < kVec; ++i) {
+        const int c = (tid + i * kRouterThreads) * 4;
+        if (c < H) {
+            __nv_bfloat16* hi = b.h + (size_t)t * 2 * H + c;
+            const float e[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) split_bf16(e[q] * r * __bfloat162float(next_gain[c + q]), hi[q], hi[H + q]);
+        }
     }
+}
+
+// Tokens per group (4 per column tile); experts with more tokens are cut into several groups and
+// stream their weights once per group.  `warps`: width of the gate/up CTA, limited by what is left
+// of shared memory after the group's activation rows.
+static void expert_plan(const Shape& s, int n_tok, int* cap, int* warps) {
+    const double avg = (double)n_tok * s.k / s.E;
+    *cap = avg <= 5.0 ? 8 : 16;
+    while ((size_t)*cap * 2 * x_row_bytes(s.H) > 140u * 1024u && *cap > 4) *cap /= 2;
+    const size_t left = 227u * 1024u - 1024u - (size_t)*cap * 2 * x_row_bytes(s.H);
+    int w = (int)(left / kRingWarpBytes);
+    *warps = w > kGuMaxWarps ? kGuMaxWarps : (w < 1 ? 1 : w);
 }
 
 // ---------------------------------------------------------------------------------------------
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,
                   cudaStream_t st) {
-    router_kernel<<<n_tok, kRouterThreads, s.H * sizeof(float), st>>>(s, b, w.mlp_norm, w.router, dbg, layer, n_tok);
-    permute_kernel<<<1, 1024, 0, st>>>(s, b, layer, n_tok * s.k);
+    int ks, o_ksplit, phases;
+    gemm_plan(s.nq * s.D, n_tok, false, &ks, &o_ksplit, &phases);
+    router_kernel<<<n_tok, kRouterThreads, 8 * x_row_bytes(s.H), st>>>(s, b, w.mlp_norm, w.router, dbg, layer, n_tok,
+                                                                       o_ksplit);
+    int cap, warps;
+    expert_plan(s, n_tok, &cap, &warps);
+    permute_kernel<<<1, 1024, 0, st>>>(s, b, layer, n_tok * s.k, cap);
     return 2;
 }
 
-// Tokens held in shared memory per pass (4 per column tile); experts with more tokens loop and
-// stream their weights again.  Small groups keep the footprint low enough for three CTAs of four
-// warps per SM; larger ones use one wide CTA per SM so that enough loads stay in flight.
-static void expert_plan(const Shape& s, int n_tok, int* cap, int* warps) {
-    const double avg = (double)n_tok * s.k / s.E;
-    *cap = avg <= 5.0 ? 8 : 16;
-    *warps = *cap == 8 ? 4 : kExpMaxWarps;
-    while ((size_t)*cap * 2 * x_row_bytes(s.H) > 200u * 1024u && *cap > 4) *cap /= 2;
-}
-
-int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st) {
+int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st) {
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
-    dim3 g1((s.I / 16 + warps - 1) / warps, s.E);
-    expert_gate_up_kernel<<<g1, warps * 32, (size_t)cap * 2 * x_row_bytes(s.H), st>>>(s, b, w.w_gate_up, cap);
+    const size_t smem = (size_t)cap * 2 * x_row_bytes(s.H) + (size_t)warps * kRingWarpBytes;
+    expert_gate_up_kernel<<<sm_count, warps * 32, smem, st>>>(s, b, w.w_gate_up, cap);
     return 1;
 }
 
 int launch_down(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st) {
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
-    const int w2 = warps == kExpMaxWarps ? 8 : warps;
+    const int w2 = cap > 8 ? 8 : 4;
     dim3 g2((s.H / 32 + w2 - 1) / w2, s.E);
     expert_down_kernel<<<g2, w2 * 32, (size_t)cap * 2 * x_row_bytes(s.I), st>>>(s, b, w.w_down, cap);
     return 1;
@@ -354,11 +477,11 @@ int launch_combine(const Shape& s, const Buffers& b, const __nv_bfloat16* next_g
 }
 
 cudaError_t init_moe_kernels() {
-    cudaError_t e = cudaFuncSetAttribute(expert_gate_up_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(expert_gate_up_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(expert_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(router_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    return cudaFuncSetAttribute(router_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * x_row_bytes(8192));
 }
 
 }  // namespace mars

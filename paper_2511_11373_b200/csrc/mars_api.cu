@@ -91,7 +91,11 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
     t.err = (int32_t*)take(256);
     t.x = (float*)take(n * H * 4);
     t.h = (__nv_bfloat16*)take(n * 2 * H * 2);
-    t.qkv = (float*)take(n * (nq + 2 * nkv) * D * 4);
+    // split-K partials: up to K/256 of them for decode-sized calls, one otherwise
+    const size_t n64 = n < 64 ? n : 64;
+    const size_t qkv_parts = std::max(n, n64 * (H / 256)), o_parts = std::max(n, n64 * (nq * D / 256));
+    t.qkv = (float*)take(qkv_parts * (nq + 2 * nkv) * D * 4);
+    t.opart = (float*)take(o_parts * H * 4);
     t.q = (__nv_bfloat16*)take(n * 2 * nq * D * 2);
     t.o = (__nv_bfloat16*)take(n * 2 * nq * D * 2);
     t.rope = (float2*)take(n * (D / 2) * 8);
@@ -103,6 +107,8 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
     t.expert_off = (int32_t*)take(((size_t)c.n_experts + 1) * 4);
     t.slot_token = (int32_t*)take(n * kk * 4);
     t.slot_of = (int32_t*)take(n * kk * 4);
+    t.groups = (int32_t*)take(((size_t)c.n_experts + n * kk / 4 + 1) * 16);
+    t.n_groups = (int32_t*)take(256);
     t.active = (int32_t*)take((size_t)c.n_layers * 4);
     t.act = (__nv_bfloat16*)take(n * kk * 2 * c.expert_inter * 2);
     t.y = (float*)take(n * kk * H * 4);
@@ -547,7 +553,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         run(MARS_K_ATTN_MERGE, [&] { return launch_attn_merge(s, b, lay, n_tok, st); });
         run(MARS_K_OPROJ, [&] { return launch_oproj(s, b, w, n_tok, st); });
         run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, st); });
-        run(MARS_K_GATE_UP, [&] { return launch_gate_up(s, b, w, n_tok, st); });
+        run(MARS_K_GATE_UP, [&] { return launch_gate_up(s, b, w, n_tok, m->sm_count, st); });
         run(MARS_K_DOWN, [&] { return launch_down(s, b, w, n_tok, st); });
         const __nv_bfloat16* next_gain = l + 1 < s.L ? m->layers[l + 1].attn_norm : m->final_norm;
         float* tap = taps.hidden ? taps.hidden + (size_t)(l + 1) * hid_stride : nullptr;
@@ -867,7 +873,7 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
         launch_attn_merge(s, buf, lay, n_seqs, st);
         launch_oproj(s, buf, lw, n_seqs, st);
         launch_router(s, buf, lw, taps, l, n_seqs, st);
-        launch_gate_up(s, buf, lw, n_seqs, st);
+        launch_gate_up(s, buf, lw, n_seqs, sms, st);
         launch_down(s, buf, lw, n_seqs, st);
         const __nv_bfloat16* next_gain =
             l + 1 < s.L ? (const __nv_bfloat16*)w->layers[l + 1].attn_norm : (const __nv_bfloat16*)w->final_norm;

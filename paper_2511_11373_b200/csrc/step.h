@@ -47,7 +47,8 @@ struct Buffers {
     int32_t* err;           // status word
     float* x;               // [n_tok, H] residual stream (fp32)
     __nv_bfloat16* h;       // [n_tok, 2, H] normalised input of the next projection, (hi, lo) rows
-    float* qkv;             // [n_tok, (nq + 2 nkv) D] raw projection
+    float* qkv;             // [ksplit, n_tok, (nq + 2 nkv) D] raw projection (split-K partials)
+    float* opart;           // [ksplit, n_tok, H] output-projection partials, added to x by the router kernel
     __nv_bfloat16* q;       // [n_tok, 2, nq D] rotated queries, (hi, lo) rows
     __nv_bfloat16* o;       // [n_tok, 2, nq D] attention output, (hi, lo) rows
     float2* rope;           // [n_tok, D/2] (cos, sin) of pos * theta_i
@@ -59,6 +60,8 @@ struct Buffers {
     int32_t* expert_off;    // [E + 1]
     int32_t* slot_token;    // [n_tok k] token row served by every expert slot
     int32_t* slot_of;       // [n_tok k] slot of (token, j)
+    int32_t* groups;        // [n_groups][4] (expert, first slot, tokens, 0): the expert kernels' work list
+    int32_t* n_groups;
     int32_t* active;        // [L] distinct experts per layer
     __nv_bfloat16* act;     // [n_tok k, 2, I] SwiGLU activations, (hi, lo) rows
     float* y;               // [n_tok k, H]
