@@ -290,19 +290,39 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
 }
 
-// Merge of the spans of one (token row, query head): log-sum-exp rule on (max, sum, O).
+// Merge of the spans of one (token row, query head): log-sum-exp rule on (max, sum, O).  The span
+// statistics are fetched in one round trip (one span per thread), then the partial outputs are
+// read four spans at a time.
 template <int D>
 __global__ void __launch_bounds__(D) attn_combine_kernel(Buffers b, StepLayout lay, int nq) {
+    __shared__ float2 sml[D];
     const int t = blockIdx.x, j = blockIdx.y, d = threadIdx.x;
     const int i0 = b.step[lay.tok_item_off + t], i1 = b.step[lay.tok_item_off + t + 1];
-    float M = -INFINITY;
-    for (int i = i0; i < i1; ++i) M = fmaxf(M, b.part_ml[(size_t)i * nq + j].x);
     float den = 0.f, o = 0.f;
-    for (int i = i0; i < i1; ++i) {
-        const float2 ml = b.part_ml[(size_t)i * nq + j];
-        const float sc = exp2f(ml.x - M);
-        den += ml.y * sc;
-        o += b.part_o[((size_t)i * nq + j) * D + d] * sc;
+    float M = -INFINITY;
+    for (int c0 = i0; c0 < i1; c0 += D) {               // chunks of D spans (one chunk unless the context is huge)
+        const int n = min(D, i1 - c0);
+        __syncthreads();
+        if (d < n) sml[d] = b.part_ml[(size_t)(c0 + d) * nq + j];
+        __syncthreads();
+        float Mc = M;
+        for (int i = 0; i < n; ++i) Mc = fmaxf(Mc, sml[i].x);
+        const float rescale = exp2f(M - Mc);            // 0 for the first chunk (M = -inf)
+        den *= rescale; o *= rescale;
+        M = Mc;
+        for (int i = 0; i < n; i += 4) {
+            float pv[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                pv[q] = i + q < n ? b.part_o[((size_t)(c0 + i + q) * nq + j) * D + d] : 0.f;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (i + q < n) {
+                    const float sc = exp2f(sml[i + q].x - M);
+                    den += sml[i + q].y * sc;
+                    o += pv[q] * sc;
+                }
+        }
     }
     // (hi, lo) rows of the token: b.o is [n_tok][2][nq D]
     __nv_bfloat16* dst = b.o + (size_t)t * 2 * nq * D + (size_t)j * D + d;

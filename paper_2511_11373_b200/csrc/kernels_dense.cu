@@ -76,9 +76,12 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(Shape s, Buffers b, 
 #pragma unroll
     for (int i = 0; i < kRowMaxPer; ++i) {
         const int c = threadIdx.x + i * kRowThreads;
-        v[i] = 0.f;
+        v[i] = c < s.H ? __bfloat162float(embed[(size_t)tok * s.H + c]) : 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < kRowMaxPer; ++i) {
+        const int c = threadIdx.x + i * kRowThreads;
         if (c < s.H) {
-            v[i] = __bfloat162float(embed[(size_t)tok * s.H + c]);
             b.x[(size_t)t * s.H + c] = v[i];
             if (hidden_tap) hidden_tap[(size_t)t * s.H + c] = v[i];
         }
@@ -215,7 +218,7 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepL
     const int page = kv.block_table[(size_t)seq * kv.max_pages_per_seq + pos / kv.page_size];
     const int slot = pos % kv.page_size;
     const float* raw = b.qkv + (size_t)t * n_heads * D;
-    for (int head = warp; head < n_heads; head += 4) {
+    for (int head = blockIdx.y * 4 + warp; head < n_heads; head += 4 * gridDim.y) {   // one head per warp
         const bool is_q = head < s.nq, is_k = !is_q && head < s.nq + s.nkv;
         float lo[PER], hi[PER];
         float ss = 0.f;
@@ -275,10 +278,11 @@ int launch_qkv(const Shape& s, const Buffers& b, const StepLayout& lay, const La
     int n = launch_gemm(p, false, st);
     int ks, ksplit, phases;
     gemm_plan(s.H, n_tok, false, &ks, &ksplit, &phases);
+    const dim3 grid(n_tok, (s.nq + 2 * s.nkv + 3) / 4);
     if (s.D == 128)
-        qkv_post_kernel<128><<<n_tok, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
+        qkv_post_kernel<128><<<grid, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
     else
-        qkv_post_kernel<64><<<n_tok, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
+        qkv_post_kernel<64><<<grid, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
     return n + 1;
 }
 

@@ -27,18 +27,32 @@ __global__ void __launch_bounds__(kRouterThreads) router_kernel(Shape s, Buffers
     const int xrow = x_row_bytes(H);
 
     // residual: x += W_o o, delivered as split-K partials that are added here in a fixed order
+    // (all loads of a partial are issued before any store, so that they overlap)
     float v[kRowMaxPer];
     float ss = 0.f;
+    const float* __restrict__ xin = b.x + (size_t)t * H;
 #pragma unroll
     for (int i = 0; i < kRowMaxPer; ++i) {
         const int c = tid + i * kRouterThreads;
-        v[i] = 0.f;
+        v[i] = c < H ? xin[c] : 0.f;
+    }
+    for (int sp = 0; sp < o_ksplit; ++sp) {
+        const float* __restrict__ part = b.opart + ((size_t)sp * n_tok + t) * H;
+        float pv[kRowMaxPer];
+#pragma unroll
+        for (int i = 0; i < kRowMaxPer; ++i) {
+            const int c = tid + i * kRouterThreads;
+            pv[i] = c < H ? part[c] : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < kRowMaxPer; ++i) v[i] += pv[i];
+    }
+#pragma unroll
+    for (int i = 0; i < kRowMaxPer; ++i) {
+        const int c = tid + i * kRouterThreads;
         if (c < H) {
-            float acc = b.x[(size_t)t * H + c];
-            for (int sp = 0; sp < o_ksplit; ++sp) acc += b.opart[((size_t)sp * n_tok + t) * H + c];
-            b.x[(size_t)t * H + c] = acc;
-            v[i] = acc;
-            ss += acc * acc;
+            b.x[(size_t)t * H + c] = v[i];
+            ss += v[i] * v[i];
         }
     }
     ss = block_sum(ss, scratch);
@@ -138,26 +152,44 @@ __global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int l
     __syncthreads();
     for (int i = tid; i < n_pairs; i += blockDim.x) atomicAdd(&cnt[b.route_idx[i]], 1);
     __syncthreads();
-    if (tid == 0) {
-        int acc = 0, active = 0;
-        for (int e = 0; e < E; ++e) {
-            off[e] = acc;
-            acc += cnt[e];
-            active += cnt[e] > 0;
-        }
-        off[E] = acc;
-        b.active[layer] = active;
-        // token groups for the expert kernels: (expert, first slot, tokens <= tok_cap, 0)
-        int ng = 0;
-        for (int e = 0; e < E; ++e)
-            for (int t0 = 0; t0 < cnt[e]; t0 += tok_cap) {
-                b.groups[4 * ng + 0] = e;
-                b.groups[4 * ng + 1] = off[e] + t0;
-                b.groups[4 * ng + 2] = min(tok_cap, cnt[e] - t0);
-                b.groups[4 * ng + 3] = 0;
-                ++ng;
+    // one expert per thread (E <= 1024): exclusive scans of the token counts (slot offsets), of the
+    // group counts (positions in the group list) and of "has tokens" (distinct experts)
+    {
+        __shared__ int wtot[3][32];
+        const int lane = tid & 31, warp = tid >> 5;
+        const int c = tid < E ? cnt[tid] : 0;
+        int inc[3] = {c, (c + tok_cap - 1) / tok_cap, c > 0 ? 1 : 0};
+        const int own[3] = {inc[0], inc[1], inc[2]};
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int nb = __shfl_up_sync(0xffffffffu, inc[q], o);
+                if (lane >= o) inc[q] += nb;
             }
-        *b.n_groups = ng;
+            if (lane == 31) wtot[q][warp] = inc[q];
+        }
+        __syncthreads();
+        int base[3] = {0, 0, 0}, tot[3] = {0, 0, 0};
+        for (int w = 0; w < 32; ++w)
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+                if (w < warp) base[q] += wtot[q][w];
+                tot[q] += wtot[q][w];
+            }
+        if (tid < E) {
+            const int o0 = base[0] + inc[0] - own[0];
+            off[tid] = o0;
+            // token groups for the expert kernels: (expert, first slot, tokens <= tok_cap, 0)
+            int ng = base[1] + inc[1] - own[1];
+            for (int t0 = 0; t0 < c; t0 += tok_cap, ++ng)
+                reinterpret_cast<int4*>(b.groups)[ng] = make_int4(tid, o0 + t0, min(tok_cap, c - t0), 0);
+        }
+        if (tid == 0) {
+            off[E] = tot[0];
+            *b.n_groups = tot[1];
+            b.active[layer] = tot[2];
+        }
     }
     __syncthreads();
     for (int e = tid; e <= E; e += blockDim.x) b.expert_off[e] = off[e];
