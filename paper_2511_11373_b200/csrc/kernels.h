@@ -31,12 +31,12 @@ int launch_prep(const Shape& s, const Buffers& b, const StepLayout& lay, const K
 int launch_embed(const Shape& s, const Buffers& b, const StepLayout& lay, const __nv_bfloat16* embed,
                  const int32_t* tokens, const __nv_bfloat16* first_gain, float* hidden_tap, int n_tok, cudaStream_t st);
 int launch_qkv(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
-               int n_tok, cudaStream_t st);
+               int n_tok, int sm_count, cudaStream_t st);
 // K elements per phase, number of K splits (partials) and phases per CTA of the streaming GEMM.
 void gemm_plan(int K, int n_tok, bool many_rows, int* ks, int* ksplit, int* phases);
-int launch_oproj(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
+int launch_oproj(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st);
 int launch_lm_head(const Shape& s, const Buffers& b, const StepLayout& lay, const __nv_bfloat16* lm_head, int n_emit,
-                   cudaStream_t st);
+                   int sm_count, cudaStream_t st);
 
 int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_k,
                      const CUtensorMap& tm_v, int layer, int sm_count, cudaStream_t st);

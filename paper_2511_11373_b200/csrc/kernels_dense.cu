@@ -102,7 +102,7 @@ int launch_embed(const Shape& s, const Buffers& b, const StepLayout&, const __nv
 // cp.async rings and keep streaming while a phase's activations are swapped.  With split-K
 // (gridDim.y > 1) every K range writes its own fp32 partial [ksplit][tokens][rows]; the consumer
 // kernel adds the partials in a fixed order, so results do not depend on scheduling.
-constexpr int kGemmWarps = 8;
+constexpr int kGemmMaxWarps = 10;   // 16 rows each; the CTA width is chosen per matrix (see launch_gemm)
 constexpr int kGemmTok = 64;
 constexpr int kGemmCols = 2 * kGemmTok;
 constexpr int kGemmNT = kGemmCols / 8;
@@ -118,15 +118,17 @@ struct GemmParams {
     int phases;                 // phases per CTA; gridDim.y * phases * ks == K
 };
 
-static size_t gemm_smem_bytes(int ks) { return (size_t)kGemmCols * x_row_bytes(ks) + (size_t)kGemmWarps * kRingWarpBytes; }
+static size_t gemm_smem_bytes(int ks, int warps) {
+    return (size_t)kGemmCols * x_row_bytes(ks) + (size_t)warps * kRingWarpBytes;
+}
 
-__global__ void __launch_bounds__(kGemmWarps * 32, 1) stream_gemm_kernel(GemmParams p) {
+__global__ void __launch_bounds__(kGemmMaxWarps * 32, 1) stream_gemm_kernel(GemmParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, tig = lane & 3;
     const int xrow = x_row_bytes(p.ks);
     unsigned char* xt = smem;
     unsigned char* ring = smem + (size_t)kGemmCols * xrow + (size_t)warp * kRingWarpBytes;
-    const int row_base = (blockIdx.x * kGemmWarps + warp) * 16;
+    const int row_base = (blockIdx.x * (blockDim.x >> 5) + warp) * 16;
     const int tok0 = blockIdx.z * kGemmTok;
     const int n_here = min(kGemmTok, p.n_tok - tok0);
     const int k_begin = blockIdx.y * p.phases * p.ks;
@@ -151,17 +153,19 @@ __global__ void __launch_bounds__(kGemmWarps * 32, 1) stream_gemm_kernel(GemmPar
     const int pieces = p.ks / 8;   // 16-byte pieces per activation row
     for (int ph = 0; ph < p.phases; ++ph) {
         if (ph > 0) __syncthreads();             // every warp is done with the previous phase's activations
+        // activation rows of this phase by cp.async (columns past the last token repeat token 0: their
+        // results are never stored)
         for (int i = threadIdx.x; i < kGemmCols * pieces; i += blockDim.x) {
             const int v = i / pieces, pc = i - v * pieces;     // v: column = 2 * token + plane
-            const int t = v >> 1;
-            uint4 val = make_uint4(0, 0, 0, 0);
-            if (t < n_here) {
-                const int src_tok = p.row_index ? p.row_index[tok0 + t] : tok0 + t;
-                val = *reinterpret_cast<const uint4*>(p.X + ((size_t)src_tok * 2 + (v & 1)) * p.K + k_begin +
-                                                      (size_t)ph * p.ks + pc * 8);
-            }
-            *reinterpret_cast<uint4*>(xt + (size_t)v * xrow + pc * 16) = val;
+            const int t = (v >> 1) < n_here ? (v >> 1) : 0;
+            const int src_tok = p.row_index ? p.row_index[tok0 + t] : tok0 + t;
+            cp_async16(xt + (size_t)v * xrow + pc * 16,
+                       p.X + ((size_t)src_tok * 2 + (v & 1)) * p.K + k_begin + (size_t)ph * p.ks + pc * 8);
         }
+        cp_async_commit();
+        // the activation group is the youngest: waiting for it also drains the ring, which costs one
+        // memory round trip per phase
+        cp_async_wait<0>();
         __syncthreads();
         const unsigned char* xs = xt + (size_t)gid * xrow + tig * 16;
         for (int sl = 0; sl < slices_per_phase; ++sl) {
@@ -195,11 +199,20 @@ void gemm_plan(int K, int n_tok, bool many_rows, int* ks, int* ksplit, int* phas
     else { *ksplit = 1; *phases = n_ph; }
 }
 
-static int launch_gemm(GemmParams p, bool many_rows, cudaStream_t st) {
+static int launch_gemm(GemmParams p, bool many_rows, int sm_count, cudaStream_t st) {
     int ksplit;
     gemm_plan(p.K, p.n_tok, many_rows, &p.ks, &ksplit, &p.phases);
-    dim3 grid((p.rows + kGemmWarps * 16 - 1) / (kGemmWarps * 16), ksplit, (p.n_tok + kGemmTok - 1) / kGemmTok);
-    stream_gemm_kernel<<<grid, kGemmWarps * 32, gemm_smem_bytes(p.ks), st>>>(p);
+    // CTA width: the number of 16-row warps that minimises waves x rows per CTA on this many SMs
+    const int tok_tiles = (p.n_tok + kGemmTok - 1) / kGemmTok;
+    int best_w = 8;
+    long best_cost = -1;
+    for (int w = 6; w <= kGemmMaxWarps; ++w) {
+        const long ctas = (long)((p.rows + w * 16 - 1) / (w * 16)) * ksplit * tok_tiles;
+        const long cost = ((ctas + sm_count - 1) / sm_count) * w;
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_w = w; }
+    }
+    dim3 grid((p.rows + best_w * 16 - 1) / (best_w * 16), ksplit, tok_tiles);
+    stream_gemm_kernel<<<grid, best_w * 32, gemm_smem_bytes(p.ks, best_w), st>>>(p);
     return 1;
 }
 
@@ -273,9 +286,9 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepL
 }
 
 int launch_qkv(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
-               int n_tok, cudaStream_t st) {
+               int n_tok, int sm_count, cudaStream_t st) {
     GemmParams p{w.wqkv, b.h, nullptr, b.qkv, (s.nq + 2 * s.nkv) * s.D, s.H, n_tok, 0, 0};
-    int n = launch_gemm(p, false, st);
+    int n = launch_gemm(p, false, sm_count, st);
     int ks, ksplit, phases;
     gemm_plan(s.H, n_tok, false, &ks, &ksplit, &phases);
     const dim3 grid(n_tok, (s.nq + 2 * s.nkv + 3) / 4);
@@ -287,20 +300,20 @@ int launch_qkv(const Shape& s, const Buffers& b, const StepLayout& lay, const La
 }
 
 // Output projection: writes split-K partials of W_o o; the router kernel adds them to the residual.
-int launch_oproj(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st) {
+int launch_oproj(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st) {
     GemmParams p{w.wo, b.o, nullptr, b.opart, s.H, s.nq * s.D, n_tok, 0, 0};
-    return launch_gemm(p, false, st);
+    return launch_gemm(p, false, sm_count, st);
 }
 
 int launch_lm_head(const Shape& s, const Buffers& b, const StepLayout& lay, const __nv_bfloat16* lm_head, int n_emit,
-                   cudaStream_t st) {
+                   int sm_count, cudaStream_t st) {
     GemmParams p{lm_head, b.h, b.step + lay.emit_rows, b.logits, s.V, s.H, n_emit, 0, 0};
-    return launch_gemm(p, true, st);
+    return launch_gemm(p, true, sm_count, st);
 }
 
 cudaError_t init_dense_kernels() {
     return cudaFuncSetAttribute(stream_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)gemm_smem_bytes(kGemmMaxKS));
+                                (int)gemm_smem_bytes(kGemmMaxKS, kGemmMaxWarps));
 }
 
 }  // namespace mars

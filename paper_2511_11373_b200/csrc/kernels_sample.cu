@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(Shape s, Buffers
     __shared__ float red_f[32];
     __shared__ int red_i[32];
     __shared__ double red_d[32];
+    __shared__ unsigned int red_u[2][32];
     __shared__ unsigned int sel_prefix;
     __shared__ unsigned long long sel_above;
     __shared__ int sel_token;
@@ -115,45 +116,60 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(Shape s, Buffers
     }
 
     // ---- nucleus threshold: radix search on the bit pattern of e_v, by mass
-    // total mass in fixed point
+    // total mass in fixed point, and which key bits differ at all: near-flat logits share their sign,
+    // most of the exponent and often some mantissa bits, and a radix digit taken from shared bits
+    // would send every token to the same bucket (one hot shared-memory atomic).
     unsigned long long part = 0;
-    for (int v = tid; v < V; v += kSampleThreads) part += to_fix(expf((l[v] - mx) * inv_t));
+    unsigned int k_or = 0u, k_and = 0xffffffffu;
+    for (int v = tid; v < V; v += kSampleThreads) {
+        const float e = expf((l[v] - mx) * inv_t);
+        part += to_fix(e);
+        k_or |= __float_as_uint(e);
+        k_and &= __float_as_uint(e);
+    }
+    k_or = __reduce_or_sync(0xffffffffu, k_or);
+    k_and = __reduce_and_sync(0xffffffffu, k_and);
+    if (lane == 0) { red_u[0][warp] = k_or; red_u[1][warp] = k_and; }
     unsigned long long z_fix;
-    block_excl_scan(part, warp_tot, &z_fix);
+    block_excl_scan(part, warp_tot, &z_fix);          // (its barriers also publish red_u)
+    for (int w = 0; w < kSampleThreads / 32; ++w) { k_or |= red_u[0][w]; k_and &= red_u[1][w]; }
     const bool everything = top_p >= 1.f;
     unsigned long long target = (unsigned long long)((double)top_p * (double)z_fix);
     if (target < 1) target = 1;
     if (target > z_fix) target = z_fix;
 
-    unsigned int prefix = 0;            // selected high bits so far
-    unsigned long long above = 0;       // mass of buckets strictly above the selected one
+    const unsigned int differ = k_or ^ k_and;
+    int remaining = differ ? 32 - __clz(differ) : 0;  // low bits that vary (the sign bit never does: <= 31)
+    unsigned int prefix = k_and >> remaining;          // the shared high bits
+    unsigned long long above = 0;                      // mass of buckets strictly above the selected one
     if (!everything) {
-        const int shifts[3] = {20, 10, 0};
-        const int widths[3] = {11, 10, 10};
-        for (int pass = 0; pass < 3; ++pass) {
-            const int sh = shifts[pass], wd = widths[pass];
+        while (remaining > 0) {
+            const int wd = remaining < 11 ? remaining : 11, sh = remaining - wd;
             for (int i = tid; i < kBins; i += kSampleThreads) hist[i] = 0ull;
+            if (tid == 0) { sel_prefix = prefix << wd; sel_above = above; }
             __syncthreads();
             for (int v = tid; v < V; v += kSampleThreads) {
                 const float e = expf((l[v] - mx) * inv_t);
                 const unsigned int key = __float_as_uint(e);
-                const bool match = pass == 0 || (key >> (sh + wd)) == prefix;
-                if (match) atomicAdd(&hist[(key >> sh) & ((1u << wd) - 1u)], to_fix(e));
+                if ((key >> (sh + wd)) == prefix) atomicAdd(&hist[(key >> sh) & ((1u << wd) - 1u)], to_fix(e));
             }
             __syncthreads();
-            if (tid == 0) {
-                unsigned long long acc = above;
-                int bsel = 0;
-                for (int bin = (1 << wd) - 1; bin >= 0; --bin) {
-                    if (acc + hist[bin] >= target) { bsel = bin; break; }
-                    acc += hist[bin];
-                }
-                sel_above = acc;
-                sel_prefix = (prefix << wd) | (unsigned int)bsel;
+            // descending scan over the buckets, two per thread
+            const int b0 = kBins - 1 - 2 * tid;
+            const unsigned long long h0 = hist[b0], h1 = hist[b0 - 1];
+            unsigned long long pass_total;
+            const unsigned long long before = above + block_excl_scan(h0 + h1, warp_tot, &pass_total);
+            if (before < target && before + h0 >= target) {
+                sel_prefix = (prefix << wd) | (unsigned int)b0;
+                sel_above = before;
+            } else if (before + h0 < target && before + h0 + h1 >= target) {
+                sel_prefix = (prefix << wd) | (unsigned int)(b0 - 1);
+                sel_above = before + h0;
             }
             __syncthreads();
             prefix = sel_prefix;
             above = sel_above;
+            remaining = sh;
             __syncthreads();
         }
     }

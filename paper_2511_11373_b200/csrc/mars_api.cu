@@ -548,10 +548,10 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     });
     for (int l = 0; l < s.L; ++l) {
         const LayerW& w = m->layers[l];
-        run(MARS_K_QKV, [&] { return launch_qkv(s, b, lay, w, kv->view, l, n_tok, st); });
+        run(MARS_K_QKV, [&] { return launch_qkv(s, b, lay, w, kv->view, l, n_tok, m->sm_count, st); });
         run(MARS_K_ATTN, [&] { return launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st); });
         run(MARS_K_ATTN_MERGE, [&] { return launch_attn_merge(s, b, lay, n_tok, st); });
-        run(MARS_K_OPROJ, [&] { return launch_oproj(s, b, w, n_tok, st); });
+        run(MARS_K_OPROJ, [&] { return launch_oproj(s, b, w, n_tok, m->sm_count, st); });
         run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, st); });
         run(MARS_K_GATE_UP, [&] { return launch_gate_up(s, b, w, n_tok, m->sm_count, st); });
         run(MARS_K_DOWN, [&] { return launch_down(s, b, w, n_tok, st); });
@@ -560,7 +560,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         run(MARS_K_COMBINE, [&] { return launch_combine(s, b, next_gain, tap, n_tok, st); });
     }
     if (n_emit) {
-        run(MARS_K_LM_HEAD, [&] { return launch_lm_head(s, b, lay, m->lm_head, n_emit, st); });
+        run(MARS_K_LM_HEAD, [&] { return launch_lm_head(s, b, lay, m->lm_head, n_emit, m->sm_count, st); });
         if (dbg && dbg->logits)
             CUDA_TRY(cudaMemcpyAsync(dbg->logits, b.logits, (size_t)n_emit * s.V * 4, cudaMemcpyDeviceToDevice, st));
         run(MARS_K_SAMPLE, [&] {
@@ -868,10 +868,10 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
                  nullptr, n_seqs, st);
     for (int l = 0; l < s.L; ++l) {
         const LayerW lw = layer_w(l);
-        launch_qkv(s, buf, lay, lw, view, l, n_seqs, st);
+        launch_qkv(s, buf, lay, lw, view, l, n_seqs, sms, st);
         launch_attention(s, buf, lay, view, tm_k, tm_v, l, sms, st);
         launch_attn_merge(s, buf, lay, n_seqs, st);
-        launch_oproj(s, buf, lw, n_seqs, st);
+        launch_oproj(s, buf, lw, n_seqs, sms, st);
         launch_router(s, buf, lw, taps, l, n_seqs, st);
         launch_gate_up(s, buf, lw, n_seqs, sms, st);
         launch_down(s, buf, lw, n_seqs, st);
@@ -879,7 +879,7 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
             l + 1 < s.L ? (const __nv_bfloat16*)w->layers[l + 1].attn_norm : (const __nv_bfloat16*)w->final_norm;
         launch_combine(s, buf, next_gain, nullptr, n_seqs, st);
     }
-    launch_lm_head(s, buf, lay, (const __nv_bfloat16*)w->lm_head, n_seqs, st);
+    launch_lm_head(s, buf, lay, (const __nv_bfloat16*)w->lm_head, n_seqs, sms, st);
     launch_sample(s, buf, lay, n_seqs, out_tokens, out_logprobs, nullptr, st);
     CUDA_TRY(cudaGetLastError());
     return MARS_OK;
