@@ -15,41 +15,44 @@ constexpr int kMaxTopK = 32;
 // One block per token row.  h2 = rms(x) * g (kept in fp32 for the gate, stored as a (hi, lo) bf16
 // pair for the experts); z_e = <W_r[e], h2> accumulated in fp32 in a fixed order; pi = softmax(z); the k largest
 // pi (ties: lower index) and their renormalised weights.
-__global__ void __launch_bounds__(kRouterThreads) router_kernel(Shape s, Buffers b, const __nv_bfloat16* gain,
-                                                                const __nv_bfloat16* Wr, DebugTaps dbg, int layer,
-                                                                int n_tok, int o_ksplit) {
+constexpr int kRouterCta = 1024;
+constexpr int kRouterPer = 8;    // hidden <= 8192
+__global__ void __launch_bounds__(kRouterCta) router_kernel(Shape s, Buffers b, const __nv_bfloat16* gain,
+                                                            const __nv_bfloat16* Wr, DebugTaps dbg, int layer, int n_tok,
+                                                            int o_ksplit) {
     // one column tile of activations: row 0 = hi, row 1 = lo of this token, rows 2..7 zero
     extern __shared__ __align__(16) unsigned char xt[];
     __shared__ float scratch[32];
     __shared__ float z[kMaxExperts];
+    __shared__ float zp[kMaxExperts];     // partial logits of the K quarters: [quarter][expert]
     const int t = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tig = lane & 3;
     const int H = s.H, E = s.E, k = s.k;
     const int xrow = x_row_bytes(H);
 
     // residual: x += W_o o, delivered as split-K partials that are added here in a fixed order
     // (all loads of a partial are issued before any store, so that they overlap)
-    float v[kRowMaxPer];
+    float v[kRouterPer];
     float ss = 0.f;
     const float* __restrict__ xin = b.x + (size_t)t * H;
 #pragma unroll
-    for (int i = 0; i < kRowMaxPer; ++i) {
-        const int c = tid + i * kRouterThreads;
+    for (int i = 0; i < kRouterPer; ++i) {
+        const int c = tid + i * kRouterCta;
         v[i] = c < H ? xin[c] : 0.f;
     }
     for (int sp = 0; sp < o_ksplit; ++sp) {
         const float* __restrict__ part = b.opart + ((size_t)sp * n_tok + t) * H;
-        float pv[kRowMaxPer];
+        float pv[kRouterPer];
 #pragma unroll
-        for (int i = 0; i < kRowMaxPer; ++i) {
-            const int c = tid + i * kRouterThreads;
+        for (int i = 0; i < kRouterPer; ++i) {
+            const int c = tid + i * kRouterCta;
             pv[i] = c < H ? part[c] : 0.f;
         }
 #pragma unroll
-        for (int i = 0; i < kRowMaxPer; ++i) v[i] += pv[i];
+        for (int i = 0; i < kRouterPer; ++i) v[i] += pv[i];
     }
 #pragma unroll
-    for (int i = 0; i < kRowMaxPer; ++i) {
-        const int c = tid + i * kRouterThreads;
+    for (int i = 0; i < kRouterPer; ++i) {
+        const int c = tid + i * kRouterCta;
         if (c < H) {
             b.x[(size_t)t * H + c] = v[i];
             ss += v[i] * v[i];
@@ -58,8 +61,8 @@ __global__ void __launch_bounds__(kRouterThreads) router_kernel(Shape s, Buffers
     ss = block_sum(ss, scratch);
     const float r = rsqrtf(ss / (float)H + s.eps);
 #pragma unroll
-    for (int i = 0; i < kRowMaxPer; ++i) {
-        const int c = tid + i * kRouterThreads;
+    for (int i = 0; i < kRouterPer; ++i) {
+        const int c = tid + i * kRouterCta;
         if (c < H) {
             __nv_bfloat16 hi, lo;
             split_bf16(v[i] * r * __bfloat162float(gain[c]), hi, lo);
@@ -69,23 +72,35 @@ __global__ void __launch_bounds__(kRouterThreads) router_kernel(Shape s, Buffers
             reinterpret_cast<__nv_bfloat16*>(xt + xrow)[c] = lo;
         }
     }
-    for (int i = tid; i < 6 * (H / 8); i += kRouterThreads) {
+    for (int i = tid; i < 6 * (H / 8); i += kRouterCta) {
         const int rw = 2 + i / (H / 8), pc = i % (H / 8);
         *reinterpret_cast<uint4*>(xt + (size_t)rw * xrow + pc * 16) = make_uint4(0, 0, 0, 0);
     }
     __syncthreads();
 
-    // gate logits with the streaming contraction: 16 experts per warp pass, columns 0/1 = hi/lo.
-    // The (hi, lo) pair carries ~16 mantissa bits of h2 and the sum is kept in fp32.
-    for (int rb = warp; rb * 16 < E; rb += kRouterThreads / 32) {
+    // gate logits with the streaming contraction: a warp task is 16 experts x one quarter of K,
+    // columns 0/1 = hi/lo.  The (hi, lo) pair carries ~16 mantissa bits of h2, sums are fp32 and
+    // the K quarters are added in a fixed order.
+    const int n_rb = (E + 15) / 16;
+    const int kq = n_rb <= 8 ? 4 : (n_rb <= 16 ? 2 : 1);
+    const int spq = (H / 32) / kq;                              // slices per quarter (H is a multiple of 256)
+    for (int task = warp; task < n_rb * kq; task += kRouterCta / 32) {
+        const int rb = task / kq, q = task - rb * kq;
         const int r0 = min(rb * 16 + gid, E - 1), r1 = min(rb * 16 + gid + 8, E - 1);
-        const __nv_bfloat16* wrow[1][2] = {{Wr + (size_t)r0 * H + tig * 8, Wr + (size_t)r1 * H + tig * 8}};
+        const size_t koff = (size_t)q * spq * 32;
+        const __nv_bfloat16* wrow[1][2] = {{Wr + (size_t)r0 * H + koff + tig * 8, Wr + (size_t)r1 * H + koff + tig * 8}};
         float acc[1][1][4] = {{{0.f, 0.f, 0.f, 0.f}}};
-        stream_mma<1, 1, 8>(wrow, H / 32, xt + (size_t)gid * xrow + tig * 16, 8 * xrow, acc);
+        stream_mma<1, 1, 8>(wrow, spq, xt + (size_t)gid * xrow + koff * 2 + tig * 16, 8 * xrow, acc);
         if (tig == 0) {
-            if (rb * 16 + gid < E) z[rb * 16 + gid] = acc[0][0][0] + acc[0][0][1];
-            if (rb * 16 + gid + 8 < E) z[rb * 16 + gid + 8] = acc[0][0][2] + acc[0][0][3];
+            if (rb * 16 + gid < E) zp[q * E + rb * 16 + gid] = acc[0][0][0] + acc[0][0][1];
+            if (rb * 16 + gid + 8 < E) zp[q * E + rb * 16 + gid + 8] = acc[0][0][2] + acc[0][0][3];
         }
+    }
+    __syncthreads();
+    for (int e = tid; e < E; e += kRouterCta) {
+        float acc = zp[e];
+        for (int q = 1; q < kq; ++q) acc += zp[q * E + e];
+        z[e] = acc;
     }
     __syncthreads();
 
@@ -477,7 +492,7 @@ int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const Debug
                   cudaStream_t st) {
     int ks, o_ksplit, phases;
     gemm_plan(s.nq * s.D, n_tok, false, &ks, &o_ksplit, &phases);
-    router_kernel<<<n_tok, kRouterThreads, 8 * x_row_bytes(s.H), st>>>(s, b, w.mlp_norm, w.router, dbg, layer, n_tok,
+    router_kernel<<<n_tok, kRouterCta, 8 * x_row_bytes(s.H), st>>>(s, b, w.mlp_norm, w.router, dbg, layer, n_tok,
                                                                        o_ksplit);
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
