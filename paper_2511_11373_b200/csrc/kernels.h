@@ -43,7 +43,16 @@ int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, co
 int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st);
 
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,
-                  cudaStream_t st);
+                  int group_cap, cudaStream_t st);
+
+// Prefill-sized contractions on tcgen05: out[m][n_cols] = A[m][2][K] (hi + lo planes) . B[n_cols][K]^T, and
+// the grouped expert pair (gather rows to slot order, gate/up + SwiGLU, down) over the group list.
+int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
+                      int32_t* err, cudaStream_t st);
+int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_xperm, const CUtensorMap& tm_wgu,
+                        const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, cudaStream_t st);
+int launch_qkv_post(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
+                    int n_tok, int ksplit, cudaStream_t st);
 int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st);
 int launch_down(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cudaStream_t st);
 int launch_combine(const Shape& s, const Buffers& b, const __nv_bfloat16* next_gain, float* hidden_tap, int n_tok,

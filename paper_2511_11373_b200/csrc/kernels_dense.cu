@@ -291,12 +291,17 @@ int launch_qkv(const Shape& s, const Buffers& b, const StepLayout& lay, const La
     int n = launch_gemm(p, false, sm_count, st);
     int ks, ksplit, phases;
     gemm_plan(s.H, n_tok, false, &ks, &ksplit, &phases);
+    return n + launch_qkv_post(s, b, lay, w, kv, layer, n_tok, ksplit, st);
+}
+
+int launch_qkv_post(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
+                    int n_tok, int ksplit, cudaStream_t st) {
     const dim3 grid(n_tok, (s.nq + 2 * s.nkv + 3) / 4);
     if (s.D == 128)
         qkv_post_kernel<128><<<grid, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
     else
         qkv_post_kernel<64><<<grid, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
-    return n + 1;
+    return 1;
 }
 
 // Output projection: writes split-K partials of W_o o; the router kernel adds them to the residual.

@@ -489,13 +489,14 @@ static void expert_plan(const Shape& s, int n_tok, int* cap, int* warps) {
 
 // ---------------------------------------------------------------------------------------------
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,
-                  cudaStream_t st) {
+                  int group_cap, cudaStream_t st) {
     int ks, o_ksplit, phases;
     gemm_plan(s.nq * s.D, n_tok, false, &ks, &o_ksplit, &phases);
     router_kernel<<<n_tok, kRouterCta, 8 * x_row_bytes(s.H), st>>>(s, b, w.mlp_norm, w.router, dbg, layer, n_tok,
                                                                        o_ksplit);
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
+    if (group_cap > 0) cap = group_cap;          // the tensor-core expert path wants one 128-row tile per group
     permute_kernel<<<1, 1024, 0, st>>>(s, b, layer, n_tok * s.k, cap);
     return 2;
 }

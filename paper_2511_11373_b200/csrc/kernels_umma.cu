@@ -1,0 +1,278 @@
+// Dense contractions of chunked prefill on the 5th-generation tensor cores (tcgen05 + TMEM).
+//
+// C[m, n] = sum_k X[m, k] W[n, k] for hundreds to thousands of token rows m: a real dense
+// contraction, unlike the decode-sized streams.  One CTA computes a 128 x 128 output tile:
+//   warp 0 (one lane)  TMA producer: per 64-wide K stage the hi plane and the lo plane of 128
+//                      activation rows and two 64-row boxes of weights, 128-byte swizzle, into a
+//                      4-stage ring (mbarrier full/empty pairs);
+//   warp 1 (one lane)  issues tcgen05.mma (M 128, N 128, K 16, bf16 x bf16 -> fp32 in TMEM): per
+//                      stage four K steps for the hi plane and four for the lo plane, all into the
+//                      same accumulator, then tcgen05.commit to release the stage;
+//   warps 2..5         epilogue: wait for the accumulator, tcgen05.ld (each warp its 32-lane
+//                      quarter of TMEM), then either store fp32 rows or apply SwiGLU to the
+//                      (gate, up) column halves and store (hi, lo) bf16 pairs.
+// Activations are (hi, lo) bf16 pairs stored [row][2][K]; a 3-D tensor map (K, plane, row) picks a
+// plane of 128 rows as one box.  For the experts the rows are expert slots (tokens gathered in
+// expert order) and a tile is one entry of the permute kernel's group list.
+// Every wait is bounded: a wait that gives up sets the device status word, the CTA stops issuing,
+// frees its TMEM columns and returns.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace mars {
+
+constexpr int kUmStages = 4;
+constexpr int kUmTileM = 128, kUmTileN = 128, kUmStageK = 64;
+constexpr int kUmTileBytes = kUmTileM * kUmStageK * 2;              // 16 KB: 128 rows x 128 B
+constexpr int kUmStageBytes = 3 * kUmTileBytes;                      // A hi, A lo, B
+constexpr int kUmThreads = 192;
+constexpr uint32_t kUmSpin = 1u << 22;
+
+__device__ __forceinline__ void um_mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void um_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool um_wait(uint64_t* bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kUmSpin; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void um_tma_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"((uint64_t)tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void um_tma_3d(void* dst, const CUtensorMap* tm, int x, int y, int z, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(dst)), "l"((uint64_t)tm), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)) : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile written by TMA with the 128-byte swizzle:
+// rows of 128 bytes, groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1,
+// layout type 2 (128-byte swizzle); the leading byte offset is unused for swizzled K-major tiles.
+__device__ __forceinline__ uint64_t um_smem_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N = 128, M = 128.
+constexpr uint32_t kUmIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kUmTileN >> 3) << 17) |
+                              ((uint32_t)(kUmTileM >> 4) << 24);
+
+__device__ __forceinline__ void um_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(kUmIdesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void um_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void um_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct UmmaParams {
+    int K;                    // contraction length, multiple of 64
+    int m_rows;               // rows of A (tokens or slots)
+    const int32_t* groups;    // null: tile y covers rows 128 y ..; else tile y = group y (expert, first slot, rows, 0)
+    const int32_t* n_groups;
+    int b_rows_per_expert;    // rows of B per expert (grouped calls)
+    int n_cols;               // output columns (store mode) or expert_inter (SwiGLU mode)
+    int swiglu;               // 0: out[m][n_cols] fp32; 1: act[m][2][n_cols] from (gate, up) column halves
+    float* out;
+    __nv_bfloat16* act;
+    int32_t* err;
+};
+
+__global__ void __launch_bounds__(kUmThreads, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, UmmaParams p) {
+    extern __shared__ unsigned char um_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)um_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t full_bar[kUmStages], empty_bar[kUmStages], accum_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ volatile int dead;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // which rows of A and B this tile contracts
+    int m0, m_valid, b_row0, b_row1, col0;
+    if (p.groups) {
+        if ((int)blockIdx.y >= *p.n_groups) return;                 // uniform for the CTA
+        const int4 g = reinterpret_cast<const int4*>(p.groups)[blockIdx.y];
+        m0 = g.y; m_valid = g.z;
+        const int base = g.x * p.b_rows_per_expert;
+        if (p.swiglu) { col0 = blockIdx.x * 64; b_row0 = base + col0; b_row1 = base + p.n_cols + col0; }
+        else { col0 = blockIdx.x * kUmTileN; b_row0 = base + col0; b_row1 = b_row0 + 64; }
+    } else {
+        m0 = blockIdx.y * kUmTileM; m_valid = min(kUmTileM, p.m_rows - m0);
+        col0 = blockIdx.x * kUmTileN; b_row0 = col0; b_row1 = col0 + 64;
+    }
+    const int nk = p.K / kUmStageK;
+
+    if (tid == 0) {
+        for (int i = 0; i < kUmStages; ++i) { um_mbar_init(&full_bar[i], 1); um_mbar_init(&empty_bar[i], 1); }
+        um_mbar_init(&accum_bar, 1);
+        dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 2) {   // one warp allocates 128 TMEM columns (fp32 accumulator 128 lanes x 128 columns)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                     "r"(128));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int ks = 0; ks < nk && !dead; ++ks) {
+                const int s = ks % kUmStages;
+                if (ks >= kUmStages && !um_wait(&empty_bar[s], ((ks / kUmStages) - 1) & 1)) {
+                    dead = 1; atomicOr(p.err, kErrTimeout); break;
+                }
+                unsigned char* st = smem + (size_t)s * kUmStageBytes;
+                um_expect_tx(&full_bar[s], kUmStageBytes);
+                um_tma_3d(st, &tm_a, ks * kUmStageK, 0, m0, &full_bar[s]);
+                um_tma_3d(st + kUmTileBytes, &tm_a, ks * kUmStageK, 1, m0, &full_bar[s]);
+                um_tma_2d(st + 2 * kUmTileBytes, &tm_b, ks * kUmStageK, b_row0, &full_bar[s]);
+                um_tma_2d(st + 2 * kUmTileBytes + kUmTileBytes / 2, &tm_b, ks * kUmStageK, b_row1, &full_bar[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            for (int ks = 0; ks < nk && !dead; ++ks) {
+                const int s = ks % kUmStages;
+                if (!um_wait(&full_bar[s], (ks / kUmStages) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_hi = smem_u32(smem + (size_t)s * kUmStageBytes);
+                const uint64_t d_hi = um_smem_desc(a_hi), d_lo = um_smem_desc(a_hi + kUmTileBytes),
+                               d_b = um_smem_desc(a_hi + 2 * kUmTileBytes);
+#pragma unroll
+                for (int kk = 0; kk < kUmStageK / 16; ++kk) {       // 32 bytes along K per step: +2 in the address field
+                    um_mma(tmem_d, d_hi + 2 * kk, d_b + 2 * kk, (ks | kk) != 0);
+                    um_mma(tmem_d, d_lo + 2 * kk, d_b + 2 * kk, 1u);
+                }
+                um_commit(&empty_bar[s]);                            // the stage is free once these MMAs retire
+            }
+            um_commit(&accum_bar);
+        }
+    } else {
+        // epilogue: a warp may touch the TMEM lanes 32 (warp % 4) .. +31
+        const int quarter = warp & 3;
+        const int r = quarter * 32 + lane;                           // row of the tile = TMEM lane
+        bool ok = true;
+        if (lane == 0 && !um_wait(&accum_bar, 0)) { dead = 1; atomicOr(p.err, kErrTimeout); }
+        __syncwarp();
+        ok = !dead;
+        ok = __all_sync(0xffffffffu, ok);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            const uint32_t lane_base = tmem_d + ((uint32_t)(quarter * 32) << 16);
+            if (!p.swiglu) {
+#pragma unroll 1
+                for (int c = 0; c < kUmTileN; c += 32) {
+                    uint32_t v[32];
+                    um_ld32(lane_base + c, v);
+                    if (r < m_valid) {
+                        float* dst = p.out + (size_t)(m0 + r) * p.n_cols + col0 + c;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            if (col0 + c + j < p.n_cols)
+                                *reinterpret_cast<float4*>(dst + j) =
+                                    make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int c = 0; c < 64; c += 32) {
+                    uint32_t gt[32], up[32];
+                    um_ld32(lane_base + c, gt);
+                    um_ld32(lane_base + 64 + c, up);
+                    if (r < m_valid) {
+                        __nv_bfloat16* dst = p.act + (size_t)(m0 + r) * 2 * p.n_cols + col0 + c;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + c + j < p.n_cols) {
+                                const float gte = __uint_as_float(gt[j]);
+                                split_bf16(gte / (1.f + expf(-gte)) * __uint_as_float(up[j]), dst[j], dst[p.n_cols + j]);
+                            }
+                    }
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 2) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(128));
+    }
+}
+
+// Rows of the normalised activations gathered into expert-slot order: xperm[slot] = h[slot_token[slot]]
+// (both planes), so that a group's rows are one contiguous TMA box.
+__global__ void __launch_bounds__(256) gather_rows_kernel(Buffers b, int H, int n_slots) {
+    const int slot = blockIdx.x;
+    if (slot >= n_slots) return;
+    const uint4* src = reinterpret_cast<const uint4*>(b.h + (size_t)b.slot_token[slot] * 2 * H);
+    uint4* dst = reinterpret_cast<uint4*>(b.xperm + (size_t)slot * 2 * H);
+    for (int i = threadIdx.x; i < 2 * H / 8; i += blockDim.x) dst[i] = src[i];
+}
+
+static size_t umma_smem_bytes() { return (size_t)kUmStages * kUmStageBytes + 1024; }
+
+int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
+                      int32_t* err, cudaStream_t st) {
+    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err};
+    dim3 grid((n_cols + kUmTileN - 1) / kUmTileN, (m_rows + kUmTileM - 1) / kUmTileM);
+    umma_gemm_kernel<<<grid, kUmThreads, umma_smem_bytes(), st>>>(tm_a, tm_b, p);
+    return 1;
+}
+
+int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_xperm, const CUtensorMap& tm_wgu,
+                        const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, cudaStream_t st) {
+    const int n_slots = n_tok * s.k;
+    const int max_groups = s.E + (n_slots + kUmTileM - 1) / kUmTileM;
+    gather_rows_kernel<<<n_slots, 256, 0, st>>>(b, s.H, n_slots);
+    UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err};
+    umma_gemm_kernel<<<dim3((s.I + 63) / 64, max_groups), kUmThreads, umma_smem_bytes(), st>>>(tm_xperm, tm_wgu, gu);
+    UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err};
+    umma_gemm_kernel<<<dim3((s.H + kUmTileN - 1) / kUmTileN, max_groups), kUmThreads, umma_smem_bytes(), st>>>(
+        tm_act, tm_wdown, dn);
+    return 3;
+}
+
+cudaError_t init_umma_kernels() {
+    return cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes());
+}
+
+}  // namespace mars

@@ -16,6 +16,7 @@ namespace mars {
 cudaError_t init_dense_kernels();
 cudaError_t init_attn_kernels();
 cudaError_t init_moe_kernels();
+cudaError_t init_umma_kernels();
 }  // namespace mars
 
 using namespace mars;
@@ -35,6 +36,7 @@ namespace {
 
 constexpr int kSpanTokens = 512;    // cached tokens per attention work item at decode
 constexpr int kStagingSlots = 4;
+constexpr int kUmmaMinTokens = 64;  // calls with more token rows take the tensor-core (tcgen05) contraction path
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -111,6 +113,7 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
     t.n_groups = (int32_t*)take(256);
     t.active = (int32_t*)take((size_t)c.n_layers * 4);
     t.act = (__nv_bfloat16*)take(n * kk * 2 * c.expert_inter * 2);
+    t.xperm = (__nv_bfloat16*)take(n > kUmmaMinTokens ? n * kk * 2 * H * 2 : 0);
     t.y = (float*)take(n * kk * H * 4);
     t.logits = (float*)take((size_t)k.n_emit * c.vocab * 4);
     int32_t* a = (int32_t*)take((size_t)k.n_emit * 4);
@@ -125,6 +128,41 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
 
 }  // namespace
 
+// bf16 tensor map with the 128-byte swizzle and a 64-element (128-byte) inner box.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static mars_status_t make_tiled_map(CUtensorMap* tm, const void* base, int rank, const cuuint64_t* dims,
+                                    const cuuint64_t* strides_bytes, const cuuint32_t* box) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return MARS_ERR_UNSUPPORTED;
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    CUresult r = ((EncodeTiledFn)fn)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims,
+                                     strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_last_cuda_error = (int32_t)r;
+        return MARS_ERR_CUDA;
+    }
+    return MARS_OK;
+}
+// weights [rows][K]: boxes of 64 rows x 64 elements
+static mars_status_t make_weight_map(CUtensorMap* tm, const void* w, uint64_t rows, uint64_t K) {
+    const cuuint64_t dims[2] = {K, rows}, strides[1] = {K * 2};
+    const cuuint32_t box[2] = {64u, 64u};
+    return make_tiled_map(tm, w, 2, dims, strides, box);
+}
+// activations [rows][2][K] (hi plane, lo plane): boxes of 128 rows of one plane x 64 elements
+static mars_status_t make_pair_map(CUtensorMap* tm, const void* x, uint64_t rows, uint64_t K) {
+    const cuuint64_t dims[3] = {K, 2, rows}, strides[2] = {K * 2, K * 4};
+    const cuuint32_t box[3] = {64u, 1u, 128u};
+    return make_tiled_map(tm, x, 3, dims, strides, box);
+}
+
 struct mars_model {
     mars_config_t cfg;
     Shape shape;
@@ -132,6 +170,10 @@ struct mars_model {
     StepLayout lay;
     Buffers buf;
     std::vector<LayerW> layers;
+    // tensor maps of the prefill (tcgen05) path: weights per layer, activation buffers
+    std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
+    CUtensorMap tm_h, tm_o, tm_xperm, tm_act;
+    bool umma_ready;
     const __nv_bfloat16 *embed, *final_norm, *lm_head;
     int32_t *io_in, *io_out;
     float* io_lp;
@@ -219,6 +261,7 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
     CUDA_TRY(init_dense_kernels());
     CUDA_TRY(init_attn_kernels());
     CUDA_TRY(init_moe_kernels());
+    CUDA_TRY(init_umma_kernels());
 
     mars_model* m = new (std::nothrow) mars_model();
     if (!m) return MARS_ERR_INVALID_ARG;
@@ -271,6 +314,31 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
     if (e != cudaSuccess) return fail(e);
     e = cudaMemset(m->buf.active, 0, (size_t)cfg->n_layers * 4);
     if (e != cudaSuccess) return fail(e);
+    // tensor maps of the prefill path (calls with more than kUmmaMinTokens token rows)
+    m->umma_ready = false;
+    if (k.n_tok > kUmmaMinTokens) {
+        const uint64_t H = cfg->hidden, QD = (uint64_t)cfg->n_q_heads * cfg->head_dim, I = cfg->expert_inter;
+        const uint64_t E = cfg->n_experts, n = k.n_tok, slots = (uint64_t)k.n_tok * cfg->top_k;
+        m->tm_wqkv.resize(cfg->n_layers); m->tm_wo.resize(cfg->n_layers);
+        m->tm_wgu.resize(cfg->n_layers); m->tm_wdown.resize(cfg->n_layers);
+        mars_status_t rc = MARS_OK;
+        for (int l = 0; l < cfg->n_layers && rc == MARS_OK; ++l) {
+            const LayerW& q = m->layers[l];
+            rc = make_weight_map(&m->tm_wqkv[l], q.wqkv, (uint64_t)(cfg->n_q_heads + 2 * cfg->n_kv_heads) * cfg->head_dim, H);
+            if (rc == MARS_OK) rc = make_weight_map(&m->tm_wo[l], q.wo, H, QD);
+            if (rc == MARS_OK) rc = make_weight_map(&m->tm_wgu[l], q.w_gate_up, E * 2 * I, H);
+            if (rc == MARS_OK) rc = make_weight_map(&m->tm_wdown[l], q.w_down, E * H, I);
+        }
+        if (rc == MARS_OK) rc = make_pair_map(&m->tm_h, m->buf.h, n, H);
+        if (rc == MARS_OK) rc = make_pair_map(&m->tm_o, m->buf.o, n, QD);
+        if (rc == MARS_OK) rc = make_pair_map(&m->tm_xperm, m->buf.xperm, slots, H);
+        if (rc == MARS_OK) rc = make_pair_map(&m->tm_act, m->buf.act, slots, I);
+        if (rc != MARS_OK) {
+            mars_model_free(m);
+            return rc;
+        }
+        m->umma_ready = true;
+    }
     *out = m;
     return MARS_OK;
 }
@@ -546,15 +614,34 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     run(MARS_K_OTHER, [&] {
         return launch_embed(s, b, lay, m->embed, plan.tokens_dev, m->layers[0].attn_norm, taps.hidden, n_tok, st);
     });
+    const bool umma = m->umma_ready && n_tok > kUmmaMinTokens;
     for (int l = 0; l < s.L; ++l) {
         const LayerW& w = m->layers[l];
-        run(MARS_K_QKV, [&] { return launch_qkv(s, b, lay, w, kv->view, l, n_tok, m->sm_count, st); });
+        if (umma) {   // prefill-sized call: dense contractions on tcgen05 / TMEM
+            const int qkv_rows = (s.nq + 2 * s.nkv) * s.D;
+            run(MARS_K_QKV, [&] {
+                int n = launch_umma_dense(m->tm_h, m->tm_wqkv[l], n_tok, qkv_rows, s.H, b.qkv, b.err, st);
+                return n + launch_qkv_post(s, b, lay, w, kv->view, l, n_tok, 1, st);
+            });
+        } else {
+            run(MARS_K_QKV, [&] { return launch_qkv(s, b, lay, w, kv->view, l, n_tok, m->sm_count, st); });
+        }
         run(MARS_K_ATTN, [&] { return launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st); });
         run(MARS_K_ATTN_MERGE, [&] { return launch_attn_merge(s, b, lay, n_tok, st); });
-        run(MARS_K_OPROJ, [&] { return launch_oproj(s, b, w, n_tok, m->sm_count, st); });
-        run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, st); });
-        run(MARS_K_GATE_UP, [&] { return launch_gate_up(s, b, w, n_tok, m->sm_count, st); });
-        run(MARS_K_DOWN, [&] { return launch_down(s, b, w, n_tok, st); });
+        if (umma) {
+            run(MARS_K_OPROJ, [&] {
+                return launch_umma_dense(m->tm_o, m->tm_wo[l], n_tok, s.H, s.nq * s.D, b.opart, b.err, st);
+            });
+            run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, 128, st); });
+            run(MARS_K_GATE_UP, [&] {
+                return launch_umma_experts(s, b, m->tm_xperm, m->tm_wgu[l], m->tm_act, m->tm_wdown[l], n_tok, st);
+            });
+        } else {
+            run(MARS_K_OPROJ, [&] { return launch_oproj(s, b, w, n_tok, m->sm_count, st); });
+            run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, 0, st); });
+            run(MARS_K_GATE_UP, [&] { return launch_gate_up(s, b, w, n_tok, m->sm_count, st); });
+            run(MARS_K_DOWN, [&] { return launch_down(s, b, w, n_tok, st); });
+        }
         const __nv_bfloat16* next_gain = l + 1 < s.L ? m->layers[l + 1].attn_norm : m->final_norm;
         float* tap = taps.hidden ? taps.hidden + (size_t)(l + 1) * hid_stride : nullptr;
         run(MARS_K_COMBINE, [&] { return launch_combine(s, b, next_gain, tap, n_tok, st); });
@@ -872,7 +959,7 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
         launch_attention(s, buf, lay, view, tm_k, tm_v, l, sms, st);
         launch_attn_merge(s, buf, lay, n_seqs, st);
         launch_oproj(s, buf, lw, n_seqs, sms, st);
-        launch_router(s, buf, lw, taps, l, n_seqs, st);
+        launch_router(s, buf, lw, taps, l, n_seqs, 0, st);
         launch_gate_up(s, buf, lw, n_seqs, sms, st);
         launch_down(s, buf, lw, n_seqs, st);
         const __nv_bfloat16* next_gain =

@@ -64,6 +64,7 @@ struct Buffers {
     int32_t* n_groups;
     int32_t* active;        // [L] distinct experts per layer
     __nv_bfloat16* act;     // [n_tok k, 2, I] SwiGLU activations, (hi, lo) rows
+    __nv_bfloat16* xperm;   // [n_tok k, 2, H] activations gathered into expert-slot order (prefill path only)
     float* y;               // [n_tok k, H]
     float* logits;          // [n_emit, V]
 };
