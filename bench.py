@@ -111,7 +111,8 @@ def algorithmic_bytes(model: dict, kv_tokens: int, active_per_layer, n_lm_rows: 
 class DecodeWorkload:
     """Builds a config (weights, cache, page tables) on one GPU and steps it through the C ABI."""
 
-    def __init__(self, cfg: dict, total_steps: int, device: torch.device, seed: int = 0):
+    def __init__(self, cfg: dict, total_steps: int, device: torch.device, seed: int = 0, prefill_reqs: int = 0,
+                 prefill_chunk: int = 0):
         from paper_2511_11373_b200 import binding
         self.binding = binding
         self.cfg, self.device = cfg, device
@@ -121,8 +122,8 @@ class DecodeWorkload:
         B = len(self.ctx)
         self.B = B
         cap = [c + total_steps + 1 for c in self.ctx]
-        n_pages = sum(wl.pages_needed(c, ps) for c in cap) + 8
-        max_pages = max(wl.pages_needed(c, ps) for c in cap) + 1
+        n_pages = sum(wl.pages_needed(c, ps) for c in cap) + 8 + prefill_reqs * (wl.pages_needed(prefill_chunk, ps) + 1)
+        max_pages = max(wl.pages_needed(c, ps) for c in cap + [prefill_chunk]) + 1
         free, _ = torch.cuda.mem_get_info(device)
         t0 = time.time()
         self.weights = wl.make_weights(model, seed=seed, device=device, gains="ones")
@@ -130,8 +131,9 @@ class DecodeWorkload:
         torch.cuda.synchronize(device)
         self.setup_s = time.time() - t0
         self.pages = wl.make_page_assignment(cap, ps, n_pages, seed=seed)
-        self.model = binding.Model(model, self.weights, max_decode_seqs=B, max_prefill_tokens=0, max_pos=max(cap) + 8)
-        self.kv = binding.KvCache(self.model, self.k_pool, self.v_pool, ps, B, max_pages)
+        self.model = binding.Model(model, self.weights, max_decode_seqs=B, max_prefill_tokens=prefill_reqs * prefill_chunk,
+                                   max_pos=max(cap + [prefill_chunk]) + 8)
+        self.kv = binding.KvCache(self.model, self.k_pool, self.v_pool, ps, B + prefill_reqs, max_pages)
         for b in range(B):
             self.kv.seq_adopt(b, self.pages[b], self.ctx[b])
         self.tok_a = wl.make_tokens(B, model["vocab"], seed=seed).to(device)
@@ -254,6 +256,75 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_mixed(args):
+    """Config 4: one chunked-prefill call (8 fresh prompts of 2048 tokens) followed by one decode step
+    over 192 sequences = one mixed step.  Prints decode-only against the HBM roofline, prefill-only
+    against the bf16 tensor peak, and the pair."""
+    from paper_2511_11373_b200 import binding
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    cfg = wl.CONFIGS[4]
+    pf = cfg["prefill"]
+    w = DecodeWorkload(cfg, args.warmup + args.steps + 4, device, prefill_reqs=pf["requests"], prefill_chunk=pf["chunk"])
+    model = cfg["model"]
+    n_pf = pf["requests"] * pf["chunk"]
+    toks = wl.make_tokens(n_pf, model["vocab"], seed=1, name="prompts").to(device)
+    out_t = torch.empty(pf["requests"], dtype=torch.int32, device=device)
+    out_l = torch.empty(pf["requests"], dtype=torch.float32, device=device)
+    ids = list(range(w.B, w.B + pf["requests"]))
+    smp = binding.make_sampling(seed=3, step=0, **w.sampling)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    stream = torch.cuda.current_stream()
+    t_pf, t_dec = [], []
+    for it in range(args.warmup + args.steps):
+        for s_ in ids:
+            w.kv.seq_reserve(s_, 0)
+        ev[0].record(stream)
+        st = binding.mars_prefill_chunk(w.model, w.kv, ids, [pf["chunk"]] * pf["requests"], toks, [1] * pf["requests"],
+                                        smp, out_t, out_l)
+        assert st == 0, binding.STATUS_NAMES.get(st, st)
+        ev[1].record(stream)
+        w.step()
+        ev[2].record(stream)
+        torch.cuda.synchronize()
+        assert w.model.poll_status() == 0
+        for s_ in ids:
+            w.kv.seq_release(s_)
+        if it >= args.warmup:
+            t_pf.append(ev[0].elapsed_time(ev[1])); t_dec.append(ev[1].elapsed_time(ev[2]))
+    # per-kernel-class device time of one more prefill call
+    for s_ in ids:
+        w.kv.seq_reserve(s_, 0)
+    w.model.profile_enable(True)
+    st = binding.mars_prefill_chunk(w.model, w.kv, ids, [pf["chunk"]] * pf["requests"], toks, [1] * pf["requests"], smp,
+                                    out_t, out_l)
+    assert st == 0
+    pf_classes = {k: round(v[0], 3) for k, v in w.model.profile_read().items() if v[1]}
+    w.model.profile_enable(False)
+    for s_ in ids:
+        w.kv.seq_release(s_)
+    active = w.model.active_experts().tolist()
+    peaks = load_peaks()
+    tflops_peak = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"] if peaks["source"] == "measured" else 1590.0
+    H, nq, nkv, D, I, L = model["hidden"], model["n_q_heads"], model["n_kv_heads"], model["head_dim"], model["expert_inter"], model["n_layers"]
+    per_tok = 2 * L * (H * (nq + 2 * nkv) * D + nq * D * H + model["top_k"] * 3 * H * I + model["n_experts"] * H)
+    attn = L * pf["requests"] * 4 * nq * D * pf["chunk"] * (pf["chunk"] + 1) // 2
+    flops = per_tok * n_pf + attn
+    pf_ms, dec_ms = statistics.median(t_pf), statistics.median(t_dec)
+    dec_bytes = algorithmic_bytes(model, w.kv_tokens_now(), active)
+    line = dict(metric=METRIC, value=w.B / (dec_ms / 1e3), unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
+                ms_per_step=pf_ms + dec_ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic",
+                config=dict(workload=cfg["name"], decode_seqs=w.B, prefill_requests=pf["requests"], prefill_chunk=pf["chunk"],
+                            l2="inputs larger than L2"),
+                decode=dict(ms=dec_ms, bytes=dec_bytes["total"], frac_of_measured_hbm=dec_bytes["total"] / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]),
+                prefill=dict(ms=pf_ms, tokens_per_s=n_pf / (pf_ms / 1e3), algorithmic_tflop=flops / 1e12,
+                             achieved_tflops=flops / (pf_ms * 1e-3) / 1e12, frac_of_measured_bf16=flops / (pf_ms * 1e-3) / 1e12 / tflops_peak,
+                             note="activations are (hi, lo) bf16 pairs: the tensor cores execute twice the algorithmic flops in the projections"),
+                mixed_ms=pf_ms + dec_ms, prefill_ms_by_class=pf_classes)
+    print(json.dumps(line))
+
+
 def run_cuda(args):
     rank, local_rank, world = dist_env()
     if world > 1:
@@ -363,7 +434,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", type=int, default=3, choices=[2, 3, 5])
+    ap.add_argument("--workload", type=int, default=3, choices=[2, 3, 4, 5])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     args = ap.parse_args()
     if args.impl == "reference":
@@ -371,7 +442,10 @@ def main():
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
-        run_cuda(args)
+        if args.workload == 4:
+            run_mixed(args)
+        else:
+            run_cuda(args)
 
 
 if __name__ == "__main__":
