@@ -40,6 +40,9 @@ int launch_lm_head(const Shape& s, const Buffers& b, const StepLayout& lay, cons
 
 int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_k,
                      const CUtensorMap& tm_v, int layer, int sm_count, cudaStream_t st);
+// Causal attention of a prefill chunk: items are blocks of up to 4 consecutive prompt tokens; writes b.o.
+int launch_attention_prefill(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv,
+                             const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int sm_count, cudaStream_t st);
 int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st);
 
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,

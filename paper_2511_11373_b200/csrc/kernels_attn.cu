@@ -290,6 +290,205 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Causal attention of chunked prefill.  A work item is a block of up to kPfQueries consecutive
+// prompt tokens of one request (items: first token row, 0, keys visible to the LAST query of the
+// block, number of queries); a unit is (item, KV head).  The K/V tiles of positions 0 .. last are
+// streamed once per unit through the same TMA ring as in the decode kernel, and warp w owns query
+// w of the block: it scores all 64 tokens of every stage (four 16-token blocks), masks by its own
+// causal length, and keeps its own online softmax and output accumulator.  Nothing is split along
+// the keys, so the normalised output goes straight to b.o as (hi, lo) pairs.
+constexpr int kPfQueries = 4;
+
+template <int D>
+__device__ __forceinline__ void attend16(uint32_t kbase, uint32_t vbase, int w0, int n_valid, const uint32_t (&qa)[D / 16][4],
+                                         float (&oacc)[D / 8][4], float& m_run, float& l_run, float scale_log2, int lane) {
+    constexpr int NTILES = D / 8;
+    const int tig = lane & 3;
+    float sacc[2][4];
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+        sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+        const int r = w0 + nt * 8 + (lane & 7);
+#pragma unroll
+        for (int kk = 0; kk < D / 32; ++kk) {
+            uint32_t kb[4];
+            ldmatrix_x4(kb, kbase + tile_off(kk >> 1, r, (kk & 1) * 4 + (lane >> 3)));
+            mma_16816(sacc[nt], qa[2 * kk][0], qa[2 * kk][1], qa[2 * kk][2], qa[2 * kk][3], kb[0], kb[1]);
+            mma_16816(sacc[nt], qa[2 * kk + 1][0], qa[2 * kk + 1][1], qa[2 * kk + 1][2], qa[2 * kk + 1][3], kb[2], kb[3]);
+        }
+    }
+    float sv[4];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int tl = w0 + (i >> 1) * 8 + 2 * tig + (i & 1);
+        sv[i] = tl < n_valid ? (sacc[i >> 1][i & 1] + sacc[i >> 1][2 + (i & 1)]) * scale_log2 : -INFINITY;
+        mx = fmaxf(mx, sv[i]);
+    }
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float m_new = fmaxf(m_run, mx);
+    const float alpha = exp2f(m_run - m_new);
+    float pv[4], pl[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        pv[i] = exp2f(sv[i] - m_new);
+        pl[i] = pv[i] - __bfloat162float(__float2bfloat16_rn(pv[i]));
+    }
+    l_run = l_run * alpha + (pv[0] + pv[1] + pv[2] + pv[3]);
+    m_run = m_new;
+    const uint32_t pa0 = pack_bf16(pv[0], pv[1]), pa2 = pack_bf16(pv[2], pv[3]);
+    const uint32_t pa1 = pack_bf16(pl[0], pl[1]), pa3 = pack_bf16(pl[2], pl[3]);
+#pragma unroll
+    for (int c = 0; c < NTILES; c += 2) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { oacc[c][i] *= alpha; oacc[c + 1][i] *= alpha; }
+        const int mi = lane >> 3;
+        const int r = w0 + (mi & 1) * 8 + (lane & 7);
+        const int ch = c + (mi >> 1);
+        uint32_t vb[4];
+        ldmatrix_x4_trans(vb, vbase + tile_off(ch >> 3, r, ch & 7));
+        mma_16816(oacc[c], pa0, pa1, pa2, pa3, vb[0], vb[1]);
+        mma_16816(oacc[c + 1], pa0, pa1, pa2, pa3, vb[2], vb[3]);
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kPfQueries * 32, 2)
+attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, AttnParams p,
+                    __nv_bfloat16* o_out) {
+    constexpr int TILE_BYTES = kStageTok * D * 2;
+    constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+    constexpr int HALVES = D / 64;
+    constexpr int KSTEPS = D / 16;
+    constexpr int NTILES = D / 8;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t full_bar[kAttnStages];
+    __shared__ volatile int dead;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tig = lane & 3;
+    if (tid == 0) {
+        for (int i = 0; i < kAttnStages; ++i) mbar_init(&full_bar[i], 1);
+        dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int n_units = p.step[H_NITEMS] * p.nkv;
+    const int4* items = reinterpret_cast<const int4*>(p.step + p.lay.items);
+    const uint64_t pol = l2_evict_first_policy();
+    uint32_t gs = 0;
+
+    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+        const int item = u / p.nkv, hk = u - item * p.nkv;
+        const int4 it = items[item];
+        const int row0 = it.x, len = it.z, nq_blk = it.w;          // len: keys visible to the last query
+        const int seq = p.step[p.lay.tok_seq + row0];
+        const int n_st = (len + kStageTok - 1) / kStageTok;
+        const int32_t* bt = p.block_table + (size_t)seq * p.max_pages_per_seq;
+        const bool has_q = warp < nq_blk;
+        const int my_len = len - (nq_blk - 1 - warp);              // keys visible to this warp's query
+
+        auto issue = [&](int j, uint32_t g_stage) {
+            const int slot = g_stage % kAttnStages;
+            unsigned char* kdst = smem + (size_t)slot * STAGE_BYTES;
+            unsigned char* vdst = kdst + TILE_BYTES;
+            const int n_valid = min(kStageTok, len - j * kStageTok);
+            const int n_boxes = (n_valid + p.box_rows - 1) / p.box_rows;
+            mbar_expect_tx(&full_bar[slot], (uint32_t)(n_boxes * p.box_rows * D * 2 * 2));
+            for (int bi = 0; bi < n_boxes; ++bi) {
+                const int tok = j * kStageTok + bi * p.box_rows;
+                const int page = bt[tok / p.page_size];
+                const int y = (((p.layer * p.n_pages + page) * p.nkv + hk) * p.page_size) + tok % p.page_size;
+#pragma unroll
+                for (int hf = 0; hf < HALVES; ++hf) {
+                    const int off = hf * (kStageTok * 128) + bi * p.box_rows * 128;
+                    tma_load_2d(kdst + off, &tm_k, hf * 64, y, &full_bar[slot], pol);
+                    tma_load_2d(vdst + off, &tm_v, hf * 64, y, &full_bar[slot], pol);
+                }
+            }
+        };
+        if (tid == 0 && !dead) {
+            const int pre = min(kAttnStages - 1, n_st);
+            for (int j = 0; j < pre; ++j) issue(j, gs + j);
+        }
+
+        uint32_t qa[KSTEPS][4];
+        {
+            const int qrow_i = row0 + (has_q ? warp : 0);
+            const __nv_bfloat16* qhi = p.q + (size_t)qrow_i * 2 * p.nq * D + (size_t)(hk * p.g + gid) * D;
+            const __nv_bfloat16* qlo = qhi + (size_t)p.nq * D;
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                qa[ks][0] = qa[ks][1] = qa[ks][2] = qa[ks][3] = 0u;
+                if (gid < p.g && has_q) {
+                    qa[ks][0] = *reinterpret_cast<const uint32_t*>(qhi + ks * 16 + 2 * tig);
+                    qa[ks][1] = *reinterpret_cast<const uint32_t*>(qlo + ks * 16 + 2 * tig);
+                    qa[ks][2] = *reinterpret_cast<const uint32_t*>(qhi + ks * 16 + 8 + 2 * tig);
+                    qa[ks][3] = *reinterpret_cast<const uint32_t*>(qlo + ks * 16 + 8 + 2 * tig);
+                }
+            }
+        }
+        float oacc[NTILES][4];
+#pragma unroll
+        for (int c = 0; c < NTILES; ++c) oacc[c][0] = oacc[c][1] = oacc[c][2] = oacc[c][3] = 0.f;
+        float m_run = -INFINITY, l_run = 0.f;
+
+        for (int j = 0; j < n_st; ++j) {
+            if (tid == 0 && !dead && j + kAttnStages - 1 < n_st) issue(j + kAttnStages - 1, gs + j + kAttnStages - 1);
+            const uint32_t g_stage = gs + j;
+            const int slot = g_stage % kAttnStages;
+            int my_ok = 1;
+            if (dead) {
+                my_ok = 0;
+            } else if (!mbar_wait(&full_bar[slot], (g_stage / kAttnStages) & 1)) {
+                my_ok = 0;
+                dead = 1;
+                atomicOr(p.err, kErrTimeout);
+            }
+            const bool ok = __all_sync(0xffffffffu, my_ok);
+            const int blk_valid = min(kStageTok, len - j * kStageTok);       // rows that hold this request's tokens
+            if (blk_valid < kStageTok) {
+                // last stage: clear the value rows past the end (0 * NaN), all warps read all rows
+                unsigned char* vt = smem + (size_t)slot * STAGE_BYTES + TILE_BYTES;
+                for (int i = tid; i < (kStageTok - blk_valid) * HALVES * 8; i += kPfQueries * 32) {
+                    const int r = blk_valid + i / (HALVES * 8), rem = i % (HALVES * 8);
+                    *reinterpret_cast<uint4*>(vt + (rem / 8) * (kStageTok * 128) + r * 128 + (rem % 8) * 16) =
+                        make_uint4(0, 0, 0, 0);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncthreads();
+            }
+            const int n_valid = min(kStageTok, my_len - j * kStageTok);      // causal: keys this query may see
+            if (has_q && ok && n_valid > 0) {
+                const uint32_t kbase = smem_u32(smem + (size_t)slot * STAGE_BYTES);
+                const uint32_t vbase = kbase + TILE_BYTES;
+                for (int w0 = 0; w0 < n_valid; w0 += 16)
+                    attend16<D>(kbase, vbase, w0, n_valid, qa, oacc, m_run, l_run, p.scale_log2, lane);
+            }
+            __syncthreads();
+        }
+        gs += n_st;
+
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        if (has_q && gid < p.g) {
+            const float inv = 1.f / l_run;
+            __nv_bfloat16* dst = o_out + (size_t)(row0 + warp) * 2 * p.nq * D + (size_t)(hk * p.g + gid) * D;
+#pragma unroll
+            for (int c = 0; c < NTILES; ++c)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int d = c * 8 + 2 * tig + e;
+                    split_bf16((oacc[c][e] + oacc[c][2 + e]) * inv, dst[d], dst[(size_t)p.nq * D + d]);
+                }
+        }
+    }
+}
+
 // Merge of the spans of one (token row, query head): log-sum-exp rule on (max, sum, O).  The span
 // statistics are fetched in one round trip (one span per thread), then the partial outputs are
 // read four spans at a time.
@@ -347,6 +546,21 @@ int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, co
     return 1;
 }
 
+int launch_attention_prefill(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv,
+                             const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int sm_count, cudaStream_t st) {
+    AttnParams p;
+    p.q = b.q; p.part_o = b.part_o; p.part_ml = b.part_ml; p.step = b.step; p.lay = lay;
+    p.block_table = kv.block_table; p.err = b.err;
+    p.max_pages_per_seq = kv.max_pages_per_seq; p.n_pages = kv.n_pages; p.page_size = kv.page_size;
+    p.box_rows = kv.page_size < kStageTok ? kv.page_size : kStageTok;
+    p.nkv = s.nkv; p.nq = s.nq; p.g = s.nq / s.nkv; p.layer = layer;
+    p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
+    const int grid = sm_count * 2;
+    if (s.D == 128) attn_prefill_kernel<128><<<grid, kPfQueries * 32, attn_smem_bytes<128>(), st>>>(tm_k, tm_v, p, b.o);
+    else attn_prefill_kernel<64><<<grid, kPfQueries * 32, attn_smem_bytes<64>(), st>>>(tm_k, tm_v, p, b.o);
+    return 1;
+}
+
 int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st) {
     if (s.D == 128) attn_combine_kernel<128><<<dim3(n_tok, s.nq), 128, 0, st>>>(b, lay, s.nq);
     else attn_combine_kernel<64><<<dim3(n_tok, s.nq), 64, 0, st>>>(b, lay, s.nq);
@@ -357,7 +571,13 @@ cudaError_t init_attn_kernels() {
     cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)attn_smem_bytes<128>());
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attn_decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(attn_decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes<64>());
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes<128>());
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attn_prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)attn_smem_bytes<64>());
 }
 

@@ -515,7 +515,8 @@ namespace {
 struct StepPlan {
     std::vector<int32_t> tok_seq, tok_pos, emit_rows, emit_slot, updates;
     const int32_t* tokens_dev;
-    int span;   // cached tokens per attention item
+    int span;   // cached tokens per attention item (decode)
+    bool prefill = false;   // attention items are blocks of consecutive prompt tokens (causal kernel)
 };
 
 mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPlan& plan, const mars_sampling_t& smp,
@@ -527,12 +528,23 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     // attention work items: spans of `span` cached tokens per token row (widened until they fit)
     int span = plan.span;
     int64_t n_items = 0;
-    for (;;) {
-        n_items = 0;
-        for (int t = 0; t < n_tok; ++t) n_items += ((int64_t)plan.tok_pos[t] + 1 + span - 1) / span;
-        if (n_items <= m->caps.n_items) break;
-        if (span > (1 << 28)) return MARS_ERR_INVALID_ARG;
-        span *= 2;
+    constexpr int kPrefillBlock = 4;   // consecutive prompt tokens per item of the causal prefill kernel
+    if (plan.prefill) {
+        for (int t = 0; t < n_tok;) {
+            int e = t + 1;
+            while (e < n_tok && e - t < kPrefillBlock && plan.tok_seq[e] == plan.tok_seq[t]) ++e;
+            t = e;
+            ++n_items;
+        }
+        if (n_items > m->caps.n_items) return MARS_ERR_INVALID_ARG;
+    } else {
+        for (;;) {
+            n_items = 0;
+            for (int t = 0; t < n_tok; ++t) n_items += ((int64_t)plan.tok_pos[t] + 1 + span - 1) / span;
+            if (n_items <= m->caps.n_items) break;
+            if (span > (1 << 28)) return MARS_ERR_INVALID_ARG;
+            span *= 2;
+        }
     }
 
     const int slot = m->next_slot;
@@ -563,16 +575,31 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         int32_t* items = blk + lay.items;
         int32_t* off = blk + lay.tok_item_off;
         int at = 0;
-        for (int t = 0; t < n_tok; ++t) {
-            off[t] = at;
-            const int len = plan.tok_pos[t] + 1;
-            kv_tokens += len;
-            for (int s0 = 0; s0 < len; s0 += span) {
+        if (plan.prefill) {
+            // blocks of consecutive tokens of one request: (first row, 0, keys visible to the last one, count)
+            for (int t = 0; t < n_tok;) {
+                int e = t + 1;
+                while (e < n_tok && e - t < kPrefillBlock && plan.tok_seq[e] == plan.tok_seq[t]) ++e;
                 items[4 * at + 0] = t;
-                items[4 * at + 1] = s0;
-                items[4 * at + 2] = std::min(span, len - s0);
-                items[4 * at + 3] = 0;
+                items[4 * at + 1] = 0;
+                items[4 * at + 2] = plan.tok_pos[e - 1] + 1;
+                items[4 * at + 3] = e - t;
+                for (int q = t; q < e; ++q) { off[q] = at; kv_tokens += plan.tok_pos[q] + 1; }
                 ++at;
+                t = e;
+            }
+        } else {
+            for (int t = 0; t < n_tok; ++t) {
+                off[t] = at;
+                const int len = plan.tok_pos[t] + 1;
+                kv_tokens += len;
+                for (int s0 = 0; s0 < len; s0 += span) {
+                    items[4 * at + 0] = t;
+                    items[4 * at + 1] = s0;
+                    items[4 * at + 2] = std::min(span, len - s0);
+                    items[4 * at + 3] = 0;
+                    ++at;
+                }
             }
         }
         off[n_tok] = at;
@@ -626,8 +653,14 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         } else {
             run(MARS_K_QKV, [&] { return launch_qkv(s, b, lay, w, kv->view, l, n_tok, m->sm_count, st); });
         }
-        run(MARS_K_ATTN, [&] { return launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st); });
-        run(MARS_K_ATTN_MERGE, [&] { return launch_attn_merge(s, b, lay, n_tok, st); });
+        if (plan.prefill) {   // causal kernel over blocks of prompt tokens; writes the merged output itself
+            run(MARS_K_ATTN, [&] {
+                return launch_attention_prefill(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st);
+            });
+        } else {
+            run(MARS_K_ATTN, [&] { return launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st); });
+            run(MARS_K_ATTN_MERGE, [&] { return launch_attn_merge(s, b, lay, n_tok, st); });
+        }
         if (umma) {
             run(MARS_K_OPROJ, [&] {
                 return launch_umma_dense(m->tm_o, m->tm_wo[l], n_tok, s.H, s.nq * s.D, b.opart, b.err, st);
@@ -757,7 +790,8 @@ mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stre
 
     StepPlan plan;
     plan.tokens_dev = tokens;
-    plan.span = 1 << 30;   // one work item per token row
+    plan.span = 1 << 30;
+    plan.prefill = true;   // attention items are blocks of consecutive prompt tokens
     std::vector<std::pair<int, int32_t>> taken;
     int row = 0;
     for (int r = 0; r < n_reqs; ++r) {

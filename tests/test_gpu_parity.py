@@ -250,3 +250,80 @@ def test_library_allocator_path_matches_adopted_pages():
     gb = b.gpu_decode(tokens, GREEDY)
     assert torch.equal(ga["logits"], gb["logits"])
     assert len(b.kv.block_table(1)) == 2
+
+
+def prefill_and_compare(model, ps, ctx, lens, seed, label):
+    """One mars_prefill_chunk call over several requests (each continuing its cached context)
+    against the oracle with the GPU's routing forced; returns the case for follow-up steps."""
+    n = sum(lens)
+    case = Case(model, ps, ctx, seed=seed, headroom=max(lens) + 4, max_prefill_tokens=n, poison=True)
+    dev = case.device
+    L, H, k, V = model["n_layers"], model["hidden"], model["top_k"], model["vocab"]
+    toks = wl.make_tokens(n, V, seed=seed + 100)
+    R = len(lens)
+    out_t = torch.empty(R, dtype=torch.int32, device=dev)
+    out_l = torch.empty(R, dtype=torch.float32, device=dev)
+    logits = torch.empty(R, V, dtype=torch.float32, device=dev)
+    hidden = torch.empty(L + 1, n, H, dtype=torch.float32, device=dev)
+    ridx = torch.empty(L, n, k, dtype=torch.int32, device=dev)
+    rw = torch.empty(L, n, k, dtype=torch.float32, device=dev)
+    dbg = binding.make_debug(logits, hidden, rw, ridx)
+    st = binding.mars_prefill_chunk(case.model, case.kv, list(range(R)), lens, toks.to(dev), [1] * R,
+                                    binding.make_sampling(greedy=1), out_t, out_l, dbg)
+    assert st == 0 and case.model.poll_status() == 0
+    seq = torch.tensor([r for r in range(R) for _ in range(lens[r])], dtype=torch.int32)
+    pos = torch.tensor([ctx[r] + i for r in range(R) for i in range(lens[r])], dtype=torch.int32)
+    orc = oracle.forward(case.ocfg, case.w_cpu, toks, seq, pos, case.k_cpu, case.v_cpu, case.bt, ps,
+                         forced_idx=ridx.cpu().contiguous())
+    last = torch.tensor([sum(lens[: r + 1]) - 1 for r in range(R)])
+    gpu = dict(router_idx=ridx.cpu(), router_w=rw.cpu(), hidden=hidden.cpu(), logits=logits.cpu(), tokens=out_t.cpu(),
+               logp=out_l.cpu())
+    stats = compare_step(gpu, dict(orc, logits=orc["logits"][last]), k, greedy=True, label=label)
+    print(label, stats)
+    for r in range(R):
+        assert case.kv.seq_len(r) == ctx[r] + lens[r]
+    # the appended cache rows of every request agree with the oracle's
+    kg = case.k_pool.cpu()
+    for r in range(R):
+        for t in (ctx[r], ctx[r] + lens[r] - 1):
+            page, slot = case.pages[r][t // ps], t % ps
+            g, w = kg[:, page, :, slot].float(), case.k_cpu[:, page, :, slot].float()
+            assert ((g - w).norm(dim=-1) <= 1e-2 * w.norm(dim=-1)).all()
+    case.cur = [c + l for c, l in zip(ctx, lens)]
+    return case, out_t.cpu()
+
+
+def test_prefill_small_chunks_use_the_causal_kernel():
+    model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=1)
+    case, toks = prefill_and_compare(model, 16, [0, 21, 64], [10, 5, 33], seed=21, label="prefill-small")
+    run_and_compare(case, toks, label="decode after small prefill")
+
+
+def test_prefill_many_tokens_tensor_core_path():
+    """More than 64 token rows: QKV, output projection and the experts run on tcgen05 (several
+    128-row tiles, several groups per expert), attention on the causal block kernel; chunks continue
+    contexts that end inside a page, at a page boundary and at zero."""
+    model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=1)
+    case, toks = prefill_and_compare(model, 16, [0, 37, 512, 129], [300, 150, 70, 1], seed=22, label="prefill-large")
+    run_and_compare(case, toks, label="decode after large prefill")
+
+
+def test_prefill_in_two_calls_equals_one_call():
+    model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=0)
+    V = model["vocab"]
+    toks = wl.make_tokens(200, V, seed=77)
+    res = []
+    for split in ((200,), (90, 110)):
+        case = Case(model, 32, [11], seed=23, headroom=210, max_prefill_tokens=200, poison=False)
+        dev = case.device
+        out_t = torch.empty(1, dtype=torch.int32, device=dev)
+        out_l = torch.empty(1, dtype=torch.float32, device=dev)
+        logits = torch.empty(1, V, dtype=torch.float32, device=dev)
+        at = 0
+        for n in split:
+            st = binding.mars_prefill_chunk(case.model, case.kv, [0], [n], toks[at:at + n].to(dev), [1],
+                                            binding.make_sampling(greedy=1), out_t, out_l, binding.make_debug(logits))
+            assert st == 0 and case.model.poll_status() == 0
+            at += n
+        res.append((logits.cpu(), int(out_t[0])))
+    assert (res[0][0] - res[1][0]).abs().max() < 1e-3 and res[0][1] == res[1][1]
