@@ -50,6 +50,9 @@ int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const Debug
 
 // Prefill-sized contractions on tcgen05: out[m][n_cols] = A[m][2][K] (hi + lo planes) . B[n_cols][K]^T, and
 // the grouped expert pair (gather rows to slot order, gate/up + SwiGLU, down) over the group list.
+int launch_resid_norm(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int o_ksplit, cudaStream_t st);
+int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int group_cap,
+                        cudaStream_t st);
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
                       int32_t* err, cudaStream_t st);
 int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_xperm, const CUtensorMap& tm_wgu,

@@ -11,6 +11,60 @@ constexpr int kRowMaxPer = 32;   // hidden <= 8192
 constexpr int kMaxExperts = 1024;
 constexpr int kMaxTopK = 32;
 
+// Softmax over the gate logits z[0..E) (shared memory, overwritten), the k largest probabilities
+// (ties: lower index) or the forced experts, and their renormalised weights.  Executed by one warp.
+__device__ void route_select(float* z, const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int t,
+                             int lane) {
+    const int E = s.E, k = s.k;
+    float mx = -INFINITY;
+    for (int e = lane; e < E; e += 32) mx = fmaxf(mx, z[e]);
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int e = lane; e < E; e += 32) {
+        const float ev = expf(z[e] - mx);
+        z[e] = ev;
+        sum += ev;
+    }
+    sum = warp_sum(sum);
+    __syncwarp();
+    for (int e = lane; e < E; e += 32) z[e] = z[e] / sum;   // pi
+    __syncwarp();
+
+    const int32_t* forced = dbg.forced_idx ? dbg.forced_idx + ((size_t)layer * n_tok + t) * k : nullptr;
+    int my_idx = -1;        // lane j keeps the j-th selection
+    float my_p = 0.f;
+    if (forced) {
+        if (lane < k) { my_idx = forced[lane]; my_p = z[my_idx]; }
+    } else {
+        for (int j = 0; j < k; ++j) {
+            float best = -1.f;
+            int bi = 0x7fffffff;
+            for (int e = lane; e < E; e += 32) {
+                const float v = z[e];
+                if (v > best) { best = v; bi = e; }   // ascending e: the lower index wins ties
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+            }
+            if (lane == j) { my_idx = bi; my_p = best; }
+            if (lane == 0) z[bi] = -1.f;               // taken
+            __syncwarp();
+        }
+    }
+    float tot = lane < k ? my_p : 0.f;
+    tot = warp_sum(tot);
+    if (lane < k) {
+        const float w = my_p / tot;
+        b.route_idx[(size_t)t * k + lane] = my_idx;
+        b.route_w[(size_t)t * k + lane] = w;
+        if (dbg.router_idx) dbg.router_idx[((size_t)layer * n_tok + t) * k + lane] = my_idx;
+        if (dbg.router_w) dbg.router_w[((size_t)layer * n_tok + t) * k + lane] = w;
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // One block per token row.  h2 = rms(x) * g (kept in fp32 for the gate, stored as a (hi, lo) bf16
 // pair for the experts); z_e = <W_r[e], h2> accumulated in fp32 in a fixed order; pi = softmax(z); the k largest
@@ -104,55 +158,7 @@ __global__ void __launch_bounds__(kRouterCta) router_kernel(Shape s, Buffers b, 
     }
     __syncthreads();
 
-    if (warp == 0) {
-        float mx = -INFINITY;
-        for (int e = lane; e < E; e += 32) mx = fmaxf(mx, z[e]);
-        mx = warp_max(mx);
-        float sum = 0.f;
-        for (int e = lane; e < E; e += 32) {
-            const float ev = expf(z[e] - mx);
-            z[e] = ev;
-            sum += ev;
-        }
-        sum = warp_sum(sum);
-        __syncwarp();
-        for (int e = lane; e < E; e += 32) z[e] = z[e] / sum;   // pi
-        __syncwarp();
-
-        const int32_t* forced = dbg.forced_idx ? dbg.forced_idx + ((size_t)layer * n_tok + t) * k : nullptr;
-        int my_idx = -1;        // lane j keeps the j-th selection
-        float my_p = 0.f;
-        if (forced) {
-            if (lane < k) { my_idx = forced[lane]; my_p = z[my_idx]; }
-        } else {
-            for (int j = 0; j < k; ++j) {
-                float best = -1.f;
-                int bi = 0x7fffffff;
-                for (int e = lane; e < E; e += 32) {
-                    const float v = z[e];
-                    if (v > best) { best = v; bi = e; }   // ascending e: the lower index wins ties
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
-                    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                    if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
-                }
-                if (lane == j) { my_idx = bi; my_p = best; }
-                if (lane == 0) z[bi] = -1.f;               // taken
-                __syncwarp();
-            }
-        }
-        float tot = lane < k ? my_p : 0.f;
-        tot = warp_sum(tot);
-        if (lane < k) {
-            const float w = my_p / tot;
-            b.route_idx[(size_t)t * k + lane] = my_idx;
-            b.route_w[(size_t)t * k + lane] = w;
-            if (dbg.router_idx) dbg.router_idx[((size_t)layer * n_tok + t) * k + lane] = my_idx;
-            if (dbg.router_w) dbg.router_w[((size_t)layer * n_tok + t) * k + lane] = w;
-        }
-    }
+    if (warp == 0) route_select(z, s, b, dbg, layer, n_tok, t, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -473,6 +479,67 @@ __global__ void __launch_bounds__(kRouterThreads) combine_kernel(Shape s, Buffer
             for (int q = 0; q < 4; ++q) split_bf16(e[q] * r * __bfloat162float(next_gain[c + q]), hi[q], hi[H + q]);
         }
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Prefill-sized calls split the router in three: residual + RMSNorm here, the gate logits as one
+// tensor-core contraction over all token rows, and the selection below.
+__global__ void __launch_bounds__(kRouterThreads) resid_norm_kernel(Shape s, Buffers b, const __nv_bfloat16* gain, int n_tok,
+                                                                   int o_ksplit) {
+    __shared__ float scratch[32];
+    const int t = blockIdx.x, tid = threadIdx.x, H = s.H;
+    float v[kRowMaxPer];
+    const float* __restrict__ xin = b.x + (size_t)t * H;
+#pragma unroll
+    for (int i = 0; i < kRowMaxPer; ++i) {
+        const int c = tid + i * kRouterThreads;
+        v[i] = c < H ? xin[c] : 0.f;
+    }
+    for (int sp = 0; sp < o_ksplit; ++sp) {
+        const float* __restrict__ part = b.opart + ((size_t)sp * n_tok + t) * H;
+#pragma unroll
+        for (int i = 0; i < kRowMaxPer; ++i) {
+            const int c = tid + i * kRouterThreads;
+            if (c < H) v[i] += part[c];
+        }
+    }
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < kRowMaxPer; ++i) {
+        const int c = tid + i * kRouterThreads;
+        if (c < H) { b.x[(size_t)t * H + c] = v[i]; ss += v[i] * v[i]; }
+    }
+    ss = block_sum(ss, scratch);
+    const float r = rsqrtf(ss / (float)H + s.eps);
+#pragma unroll
+    for (int i = 0; i < kRowMaxPer; ++i) {
+        const int c = tid + i * kRouterThreads;
+        if (c < H) split_bf16(v[i] * r * __bfloat162float(gain[c]), b.h[(size_t)t * 2 * H + c], b.h[(size_t)t * 2 * H + H + c]);
+    }
+}
+
+// One warp per token row: logits [n_tok][E] (fp32, from the contraction) -> routing.
+__global__ void __launch_bounds__(128) route_select_kernel(Shape s, Buffers b, DebugTaps dbg, int layer, int n_tok) {
+    extern __shared__ float zs[];     // [4][E]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * 4 + warp;
+    if (t >= n_tok) return;
+    float* z = zs + (size_t)warp * s.E;
+    for (int e = lane; e < s.E; e += 32) z[e] = b.rlogits[(size_t)t * s.E + e];
+    __syncwarp();
+    route_select(z, s, b, dbg, layer, n_tok, t, lane);
+}
+
+int launch_resid_norm(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int o_ksplit, cudaStream_t st) {
+    resid_norm_kernel<<<n_tok, kRouterThreads, 0, st>>>(s, b, w.mlp_norm, n_tok, o_ksplit);
+    return 1;
+}
+
+int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int group_cap,
+                        cudaStream_t st) {
+    route_select_kernel<<<(n_tok + 3) / 4, 128, 4 * s.E * sizeof(float), st>>>(s, b, dbg, layer, n_tok);
+    permute_kernel<<<1, 1024, 0, st>>>(s, b, layer, n_tok * s.k, group_cap);
+    return 2;
 }
 
 // Tokens per group (4 per column tile); experts with more tokens are cut into several groups and

@@ -104,6 +104,7 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
     t.inv_freq = (double*)take((D / 2) * 8);
     t.part_o = (float*)take((size_t)k.n_items * nq * D * 4);
     t.part_ml = (float2*)take((size_t)k.n_items * nq * 8);
+    t.rlogits = (float*)take(n > kUmmaMinTokens ? n * c.n_experts * 4 : 0);
     t.route_idx = (int32_t*)take(n * kk * 4);
     t.route_w = (float*)take(n * kk * 4);
     t.expert_off = (int32_t*)take(((size_t)c.n_experts + 1) * 4);
@@ -171,7 +172,7 @@ struct mars_model {
     Buffers buf;
     std::vector<LayerW> layers;
     // tensor maps of the prefill (tcgen05) path: weights per layer, activation buffers
-    std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
+    std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown, tm_router;
     CUtensorMap tm_h, tm_o, tm_xperm, tm_act;
     bool umma_ready;
     const __nv_bfloat16 *embed, *final_norm, *lm_head;
@@ -320,7 +321,7 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
         const uint64_t H = cfg->hidden, QD = (uint64_t)cfg->n_q_heads * cfg->head_dim, I = cfg->expert_inter;
         const uint64_t E = cfg->n_experts, n = k.n_tok, slots = (uint64_t)k.n_tok * cfg->top_k;
         m->tm_wqkv.resize(cfg->n_layers); m->tm_wo.resize(cfg->n_layers);
-        m->tm_wgu.resize(cfg->n_layers); m->tm_wdown.resize(cfg->n_layers);
+        m->tm_wgu.resize(cfg->n_layers); m->tm_wdown.resize(cfg->n_layers); m->tm_router.resize(cfg->n_layers);
         mars_status_t rc = MARS_OK;
         for (int l = 0; l < cfg->n_layers && rc == MARS_OK; ++l) {
             const LayerW& q = m->layers[l];
@@ -328,6 +329,7 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_wo[l], q.wo, H, QD);
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_wgu[l], q.w_gate_up, E * 2 * I, H);
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_wdown[l], q.w_down, E * H, I);
+            if (rc == MARS_OK) rc = make_weight_map(&m->tm_router[l], q.router, E, H);
         }
         if (rc == MARS_OK) rc = make_pair_map(&m->tm_h, m->buf.h, n, H);
         if (rc == MARS_OK) rc = make_pair_map(&m->tm_o, m->buf.o, n, QD);
@@ -665,7 +667,11 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             run(MARS_K_OPROJ, [&] {
                 return launch_umma_dense(m->tm_o, m->tm_wo[l], n_tok, s.H, s.nq * s.D, b.opart, b.err, st);
             });
-            run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, 128, st); });
+            run(MARS_K_ROUTER, [&] {
+                int n = launch_resid_norm(s, b, w, n_tok, 1, st);
+                n += launch_umma_dense(m->tm_h, m->tm_router[l], n_tok, s.E, s.H, b.rlogits, b.err, st);
+                return n + launch_route_select(s, b, taps, l, n_tok, 128, st);
+            });
             run(MARS_K_GATE_UP, [&] {
                 return launch_umma_experts(s, b, m->tm_xperm, m->tm_wgu[l], m->tm_act, m->tm_wdown[l], n_tok, st);
             });

@@ -55,6 +55,7 @@ struct Buffers {
     double* inv_freq;       // [D/2] theta^(-2i/D)
     float* part_o;          // [items, nq, D] unnormalised partial outputs
     float2* part_ml;        // [items, nq] (running max in log2 units, sum)
+    float* rlogits;         // [n_tok, E] gate logits (prefill path: computed by one contraction for all rows)
     int32_t* route_idx;     // [n_tok, k]
     float* route_w;         // [n_tok, k]
     int32_t* expert_off;    // [E + 1]
