@@ -1,11 +1,11 @@
 // Dense contractions of chunked prefill on the 5th-generation tensor cores (tcgen05 + TMEM).
 //
 // C[m, n] = sum_k X[m, k] W[n, k] for hundreds to thousands of token rows m: a real dense
-// contraction, unlike the decode-sized streams.  One CTA computes a 128 x 128 output tile:
+// contraction, unlike the decode-sized streams.  One CTA computes a 128 x 256 output tile:
 //   warp 0 (one lane)  TMA producer: per 64-wide K stage the hi plane and the lo plane of 128
-//                      activation rows and two 64-row boxes of weights, 128-byte swizzle, into a
-//                      4-stage ring (mbarrier full/empty pairs);
-//   warp 1 (one lane)  issues tcgen05.mma (M 128, N 128, K 16, bf16 x bf16 -> fp32 in TMEM): per
+//                      activation rows and four 64-row boxes of weights, 128-byte swizzle, into a
+//                      3-stage ring (mbarrier full/empty pairs);
+//   warp 1 (one lane)  issues tcgen05.mma (M 128, N 256, K 16, bf16 x bf16 -> fp32 in TMEM): per
 //                      stage four K steps for the hi plane and four for the lo plane, all into the
 //                      same accumulator, then tcgen05.commit to release the stage;
 //   warps 2..5         epilogue: wait for the accumulator, tcgen05.ld (each warp its 32-lane
@@ -21,10 +21,11 @@
 
 namespace mars {
 
-constexpr int kUmStages = 4;
-constexpr int kUmTileM = 128, kUmTileN = 128, kUmStageK = 64;
+constexpr int kUmStages = 3;
+constexpr int kUmTileM = 128, kUmTileN = 256, kUmStageK = 64;
 constexpr int kUmTileBytes = kUmTileM * kUmStageK * 2;              // 16 KB: 128 rows x 128 B
-constexpr int kUmStageBytes = 3 * kUmTileBytes;                      // A hi, A lo, B
+constexpr int kUmBBytes = kUmTileN * kUmStageK * 2;                 // 32 KB: 256 weight rows x 128 B
+constexpr int kUmStageBytes = 2 * kUmTileBytes + kUmBBytes;         // A hi, A lo, B
 constexpr int kUmThreads = 192;
 constexpr uint32_t kUmSpin = 1u << 22;
 
@@ -68,7 +69,7 @@ __device__ __forceinline__ uint64_t um_smem_desc(uint32_t smem_addr) {
     d |= (uint64_t)2 << 61;
     return d;
 }
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N = 128, M = 128.
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N = 256, M = 128.
 constexpr uint32_t kUmIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kUmTileN >> 3) << 17) |
                               ((uint32_t)(kUmTileM >> 4) << 24);
 
@@ -120,17 +121,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // which rows of A and B this tile contracts
-    int m0, m_valid, b_row0, b_row1, col0;
+    int m0, m_valid, b_row0, b_row1, col0;     // b_row0 / b_row1: first weight row of each 128-column half
     if (p.groups) {
         if ((int)blockIdx.y >= *p.n_groups) return;                 // uniform for the CTA
         const int4 g = reinterpret_cast<const int4*>(p.groups)[blockIdx.y];
         m0 = g.y; m_valid = g.z;
         const int base = g.x * p.b_rows_per_expert;
-        if (p.swiglu) { col0 = blockIdx.x * 64; b_row0 = base + col0; b_row1 = base + p.n_cols + col0; }
-        else { col0 = blockIdx.x * kUmTileN; b_row0 = base + col0; b_row1 = b_row0 + 64; }
+        if (p.swiglu) { col0 = blockIdx.x * 128; b_row0 = base + col0; b_row1 = base + p.n_cols + col0; }
+        else { col0 = blockIdx.x * kUmTileN; b_row0 = base + col0; b_row1 = b_row0 + 128; }
     } else {
         m0 = blockIdx.y * kUmTileM; m_valid = min(kUmTileM, p.m_rows - m0);
-        col0 = blockIdx.x * kUmTileN; b_row0 = col0; b_row1 = col0 + 64;
+        col0 = blockIdx.x * kUmTileN; b_row0 = col0; b_row1 = col0 + 128;
     }
     const int nk = p.K / kUmStageK;
 
@@ -141,9 +142,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 2) {   // one warp allocates 128 TMEM columns (fp32 accumulator 128 lanes x 128 columns)
+    if (warp == 2) {   // one warp allocates the TMEM columns (fp32 accumulator: 128 lanes x 256 columns)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
-                     "r"(128));
+                     "r"(kUmTileN));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
@@ -162,8 +163,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                 um_expect_tx(&full_bar[s], kUmStageBytes);
                 um_tma_3d(st, &tm_a, ks * kUmStageK, 0, m0, &full_bar[s]);
                 um_tma_3d(st + kUmTileBytes, &tm_a, ks * kUmStageK, 1, m0, &full_bar[s]);
-                um_tma_2d(st + 2 * kUmTileBytes, &tm_b, ks * kUmStageK, b_row0, &full_bar[s]);
-                um_tma_2d(st + 2 * kUmTileBytes + kUmTileBytes / 2, &tm_b, ks * kUmStageK, b_row1, &full_bar[s]);
+                unsigned char* sb = st + 2 * kUmTileBytes;            // four boxes of 64 weight rows (8 KB each)
+                um_tma_2d(sb, &tm_b, ks * kUmStageK, b_row0, &full_bar[s]);
+                um_tma_2d(sb + 8192, &tm_b, ks * kUmStageK, b_row0 + 64, &full_bar[s]);
+                um_tma_2d(sb + 16384, &tm_b, ks * kUmStageK, b_row1, &full_bar[s]);
+                um_tma_2d(sb + 24576, &tm_b, ks * kUmStageK, b_row1 + 64, &full_bar[s]);
             }
         }
     } else if (warp == 1) {
@@ -213,10 +217,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                 }
             } else {
 #pragma unroll 1
-                for (int c = 0; c < 64; c += 32) {
+                for (int c = 0; c < 128; c += 32) {
                     uint32_t gt[32], up[32];
                     um_ld32(lane_base + c, gt);
-                    um_ld32(lane_base + 64 + c, up);
+                    um_ld32(lane_base + 128 + c, up);
                     if (r < m_valid) {
                         __nv_bfloat16* dst = p.act + (size_t)(m0 + r) * 2 * p.n_cols + col0 + c;
 #pragma unroll
@@ -234,7 +238,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     __syncthreads();
     if (warp == 2) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(128));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kUmTileN));
     }
 }
 
@@ -264,7 +268,7 @@ int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_
     const int max_groups = s.E + (n_slots + kUmTileM - 1) / kUmTileM;
     gather_rows_kernel<<<n_slots, 256, 0, st>>>(b, s.H, n_slots);
     UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err};
-    umma_gemm_kernel<<<dim3((s.I + 63) / 64, max_groups), kUmThreads, umma_smem_bytes(), st>>>(tm_xperm, tm_wgu, gu);
+    umma_gemm_kernel<<<dim3((s.I + 127) / 128, max_groups), kUmThreads, umma_smem_bytes(), st>>>(tm_xperm, tm_wgu, gu);
     UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err};
     umma_gemm_kernel<<<dim3((s.H + kUmTileN - 1) / kUmTileN, max_groups), kUmThreads, umma_smem_bytes(), st>>>(
         tm_act, tm_wdown, dn);
