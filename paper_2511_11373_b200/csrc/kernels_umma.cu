@@ -253,12 +253,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 // ---------------------------------------------------------------------------------------------
 // Decode-sized dense projections (QKV, output projection, lm_head) on the same tensor cores with the
 // operands swapped: 128 WEIGHT rows sit on the TMEM lanes and up to 64 token columns on N, so the
-// kernel streams each weight once from HBM (TMA, 4-stage ring) while the hi and lo activation planes
+// kernel streams each weight once from HBM (TMA, 3-stage ring, two CTAs per SM) while the hi and lo activation planes
 // of the K range are re-read from L2.  With 64 tokens carried as (hi, lo) pairs these projections
 // are tensor-bound on the mma.sync path (128 columns per weight row); here they are HBM streams again.
 // gridDim.y splits K; every split writes an fp32 partial [split][token][row] that the consumer adds
 // in a fixed order.
-constexpr int kSwStages = 4;
+constexpr int kSwStages = 3;
 constexpr int kSwTok = 64;
 constexpr int kSwABytes = 128 * kUmStageK * 2;                       // 16 KB of weights per stage
 constexpr int kSwBBytes = kSwTok * kUmStageK * 2;                    // 8 KB per activation plane
@@ -271,7 +271,7 @@ struct SwapParams {
     int32_t* err;
 };
 
-__global__ void __launch_bounds__(kUmThreads, 1)
+__global__ void __launch_bounds__(kUmThreads, 2)
 umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, SwapParams p) {
     extern __shared__ unsigned char um_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)um_raw + 1023) & ~(uintptr_t)1023);
