@@ -263,7 +263,7 @@ def run_mixed(args):
     from paper_2511_11373_b200 import binding
     device = torch.device("cuda", 0)
     torch.cuda.set_device(device)
-    cfg = wl.CONFIGS[4]
+    cfg = wl.CONFIGS[args.workload]
     pf = cfg["prefill"]
     w = DecodeWorkload(cfg, args.warmup + args.steps + 4, device, prefill_reqs=pf["requests"], prefill_chunk=pf["chunk"])
     model = cfg["model"]
@@ -434,7 +434,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", type=int, default=3, choices=[2, 3, 4, 5])
+    ap.add_argument("--workload", type=int, default=3, choices=[2, 3, 4, 5, 6])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     args = ap.parse_args()
     if args.impl == "reference":
@@ -442,7 +442,7 @@ def main():
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
-        if args.workload == 4:
+        if args.workload in (4, 6):
             run_mixed(args)
         else:
             run_cuda(args)

@@ -52,6 +52,10 @@ CONFIGS = {
     4: dict(name="qwen3-30b-a3b-48layer-mixed-b192+8x2048", model=MODEL_FULL, page_size=64, batch=192,
             ctx_lognormal=dict(sigma=0.6, medians=dict(solver=2896, verifier=4096, corrector=5793), clip=(512, 32768)),
             prefill=dict(requests=8, chunk=2048), steps=1, sampling=dict(greedy=0, temperature=1.0, top_p=0.95)),
+    # profiling-sized stand-in for config 4: one layer, 64 decode sequences + 4 prompts of 1024 tokens
+    6: dict(name="qwen3-30b-a3b-1layer-mixed-b64+4x1024", model=MODEL_LAYER, page_size=64, batch=64,
+            ctx_range=(1024, 16384), prefill=dict(requests=4, chunk=1024), steps=1,
+            sampling=dict(greedy=0, temperature=1.0, top_p=0.95)),
     5: dict(name="qwen3-30b-a3b-48layer-decode-b16-64k", model=MODEL_FULL, page_size=64, batch=16,
             ctx=[65536] * 16, steps=64, sampling=dict(greedy=1, temperature=1.0, top_p=1.0)),
 }
