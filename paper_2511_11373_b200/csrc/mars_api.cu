@@ -703,8 +703,11 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     }
     if (n_emit) {
         run(MARS_K_LM_HEAD, [&] {
-            if (!plan.prefill)   // decode: the emitting rows are the token rows in order
+            // decode: the emitting rows are the token rows in order, so the tensor maps over b.h apply
+            if (!plan.prefill && n_emit <= kUmmaMinTokens)
                 return launch_umma_swap(m->tm_lm, m->tm_h64, s.V, n_emit, s.H, 1, b.logits, b.err, st);
+            if (!plan.prefill && umma)
+                return launch_umma_dense(m->tm_h, m->tm_lm, n_emit, s.V, s.H, b.logits, b.err, st);
             return launch_lm_head(s, b, lay, m->lm_head, n_emit, m->sm_count, st);
         });
         if (dbg && dbg->logits)

@@ -327,3 +327,16 @@ def test_prefill_in_two_calls_equals_one_call():
             at += n
         res.append((logits.cpu(), int(out_t[0])))
     assert (res[0][0] - res[1][0]).abs().max() < 1e-3 and res[0][1] == res[1][1]
+
+
+def test_decode_with_more_than_64_sequences():
+    """More than 64 decode rows switch the dense projections and the lm_head to the 128-row
+    tensor-core tiles (and the experts to grouped tiles); results must not change."""
+    model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=1)
+    ctx = [5 + 7 * i for i in range(70)]
+    case = Case(model, 16, ctx, seed=31)
+    tokens = wl.make_tokens(len(ctx), model["vocab"], seed=8)
+    _, _, stats = run_and_compare(case, tokens, sampling=dict(greedy=0, temperature=0.85, top_p=0.95), step=3, seed=5,
+                                  label="decode-70")
+    print("decode-70", stats)
+    check_cache_append(case, ctx)
