@@ -34,7 +34,7 @@ static thread_local int32_t g_last_cuda_error = 0;
 
 namespace {
 
-constexpr int kSpanTokens = 512;    // cached tokens per attention work item at decode
+constexpr int kSpanTokens = 1024;   // cached tokens per attention work item at decode
 constexpr int kStagingSlots = 4;
 constexpr int kUmmaMinTokens = 64;  // calls with more token rows take the tensor-core (tcgen05) contraction path
 
