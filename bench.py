@@ -36,6 +36,11 @@ from paper_2511_11373_b200 import workloads as wl  # noqa: E402
 METRIC = "decode_tokens_per_sec"
 UNIT = "tokens/s"
 PEAKS_FALLBACK = dict(hbm_gbs=6650.0, source="fallback")
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of the captured launch, per kernel class.
+# Set an entry to None (or delete it) when that kernel changes after the capture.
+NCU_TRAFFIC_RATIO = {"attn": (1206.095e6 + 8.407e6) / 1201.844e6,     # attn_decode_kernel<128>, 586 166 cached tokens
+                     "gate_up": (795.326e6 + 5.083e6) / 786.432e6,      # expert_gate_up_kernel, 125 experts
+                     "down": (397.982e6 + 5.032e6) / 393.216e6}         # expert_down_kernel
 
 
 def load_peaks() -> dict:
@@ -405,8 +410,11 @@ def run_cuda(args):
             if name in per_launch:
                 kernels[name]["achieved_gbs"] = per_launch[name] / (kms / n * 1e-3) / 1e9
     top = max(per_launch, key=lambda k: kernels.get(k, {}).get("ms_per_step", 0.0))
+    # DRAM traffic per launch: ncu counters of a one-layer capture (profiles/decode_one_layer_b64_top_kernels.md),
+    # scaled to this launch by the units processed (traffic grows in proportion to the bytes streamed)
+    traffic = per_launch[top] * NCU_TRAFFIC_RATIO[top] if top in NCU_TRAFFIC_RATIO else None
     roofline = dict(bound="hbm", kernel=top, achieved=kernels[top]["achieved_gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
-                    frac=kernels[top]["achieved_gbs"] / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"],
+                    frac=kernels[top]["achieved_gbs"] / peaks["hbm_gbs"], traffic=traffic, peak_source=peaks["source"],
                     bytes_per_launch=per_launch[top], us_per_launch=kernels[top]["us_per_launch"])
 
     if rank != 0:
