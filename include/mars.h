@@ -151,6 +151,38 @@ MARS_API int32_t mars_kv_seq_len(const mars_kv_t *kv, int32_t seq); /* -1 if the
 /* Copies the slot's page ids (host array, capacity cap) and their count. */
 MARS_API mars_status_t mars_kv_block_table(const mars_kv_t *kv, int32_t seq, int32_t *pages_out, int32_t cap, int32_t *n);
 
+/* ---- carrying a sequence across rollout segments, and forking group members --------------------
+ * Rollouts are cut into fixed-length segments: a trajectory that has not finished when its segment
+ * ends keeps its prefix and resumes decoding in a later segment (Section 2.3, segment rollouts).
+ * A parked sequence either keeps its pages (the slot stays valid; nothing to do), or is packed into an image, released and restored later into whatever
+ * pages are free then, or is dropped and its prefix fed again through mars_prefill_chunk.  All
+ * three give the same next-token distribution; the first two bit for bit.
+ *
+ * Image layout (bf16, whole pages): [K | V][n_layers][pages of the sequence in order][n_kv_heads]
+ * [page_size][head_dim]; mars_kv_seq_image_bytes(kv, n) bytes for n cached tokens (0 on a bad
+ * handle).  `image` is device memory or PAGE-LOCKED host memory (the copy kernels address it
+ * directly), 16-byte aligned; pageable host memory is rejected with MARS_ERR_INVALID_ARG.
+ *   export: packs the slot's ceil(len / page_size) pages; asynchronous on the stream; the slot is
+ *           unchanged (release it afterwards on the same stream's order to free the pages).
+ *   import: the slot must be empty; reserves pages for n_tokens (MARS_ERR_KV_FULL leaves it
+ *           empty), unpacks the image on the stream and sets the length to n_tokens.
+ * The image must stay alive and unmodified until the stream has passed the call.
+ *
+ * fork: the members of a rollout group continue the same prompt (Section 3.3, grouped agentic
+ * rollouts: a group of 8 outputs per selected input).  dst (empty) becomes a sequence with src's
+ * cached tokens: full pages are
+ * SHARED (reference-counted; a page returns to the free list when its last holder releases it), a
+ * partly filled last page is copied into a fresh page on the stream, so both sequences append
+ * privately.  Shared pages are never written: set_len refuses a length whose next position falls
+ * into a shared page, and the step calls return MARS_ERR_BAD_HANDLE in that case.
+ * mars_kv_page_refs: number of slots that list the page (0 = free, -1 = bad argument). */
+MARS_API size_t mars_kv_seq_image_bytes(const mars_kv_t *kv, int32_t n_tokens);
+MARS_API mars_status_t mars_kv_seq_export(mars_kv_t *kv, int32_t seq, void *image, size_t image_bytes, void *cuda_stream);
+MARS_API mars_status_t mars_kv_seq_import(mars_kv_t *kv, int32_t seq, const void *image, size_t image_bytes,
+                                          int32_t n_tokens, void *cuda_stream);
+MARS_API mars_status_t mars_kv_seq_fork(mars_kv_t *kv, int32_t src, int32_t dst, void *cuda_stream);
+MARS_API int32_t mars_kv_page_refs(const mars_kv_t *kv, int32_t page);
+
 /* ---- the step ---------------------------------------------------------------------------------
  * mars_decode_step: for each listed sequence slot b (context length c_b), feed in_tokens[b] at
  * position c_b, append its key/value to the cache (a new page is taken from the free list when

@@ -78,6 +78,11 @@ SIGNATURES = {
     "mars_kv_seq_release": (c_int32, [c_void_p, c_int32]),
     "mars_kv_seq_len": (c_int32, [c_void_p, c_int32]),
     "mars_kv_block_table": (c_int32, [c_void_p, c_int32, POINTER(c_int32), c_int32, POINTER(c_int32)]),
+    "mars_kv_seq_image_bytes": (c_size_t, [c_void_p, c_int32]),
+    "mars_kv_seq_export": (c_int32, [c_void_p, c_int32, c_void_p, c_size_t, c_void_p]),
+    "mars_kv_seq_import": (c_int32, [c_void_p, c_int32, c_void_p, c_size_t, c_int32, c_void_p]),
+    "mars_kv_seq_fork": (c_int32, [c_void_p, c_int32, c_int32, c_void_p]),
+    "mars_kv_page_refs": (c_int32, [c_void_p, c_int32]),
     "mars_decode_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), c_void_p,
                                    POINTER(mars_sampling_t), c_void_p, c_void_p, POINTER(mars_debug_t)]),
     "mars_prefill_chunk": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), POINTER(c_int32), c_void_p,
@@ -271,6 +276,27 @@ class KvCache:
         n = c_int32()
         _check(lib().mars_kv_block_table(self.handle, seq, arr, self.max_pages_per_seq, byref(n)), "mars_kv_block_table")
         return list(arr[: n.value])
+
+    def seq_image_bytes(self, n_tokens: int) -> int:
+        return lib().mars_kv_seq_image_bytes(self.handle, n_tokens)
+
+    def seq_export(self, seq: int, image: torch.Tensor, stream=None) -> int:
+        """`image`: uint8 tensor on the device or in pinned host memory.  Returns the status code."""
+        with torch.cuda.device(self.k_pool.device):
+            return lib().mars_kv_seq_export(self.handle, seq, image.data_ptr(), image.numel() * image.element_size(),
+                                            _stream_handle(stream))
+
+    def seq_import(self, seq: int, image: torch.Tensor, n_tokens: int, stream=None) -> int:
+        with torch.cuda.device(self.k_pool.device):
+            return lib().mars_kv_seq_import(self.handle, seq, image.data_ptr(), image.numel() * image.element_size(),
+                                            n_tokens, _stream_handle(stream))
+
+    def seq_fork(self, src: int, dst: int, stream=None) -> int:
+        with torch.cuda.device(self.k_pool.device):
+            return lib().mars_kv_seq_fork(self.handle, src, dst, _stream_handle(stream))
+
+    def page_refs(self, page: int) -> int:
+        return lib().mars_kv_page_refs(self.handle, page)
 
     def close(self):
         if getattr(self, "handle", None):

@@ -70,6 +70,20 @@ int launch_combine(const Shape& s, const Buffers& b, const __nv_bfloat16* next_g
 int launch_sample(const Shape& s, const Buffers& b, const StepLayout& lay, int n_emit, int32_t* out_tokens,
                   float* out_logprobs, float* nucleus_mass, cudaStream_t st);
 
+// Copies n_pages pages in each of n_layers layers: unit (layer, i) goes from
+// src + layer * src_layer_stride + src_pages[i] * page_bytes to the same expression on the dst side
+// (a null page list means page index i itself, i.e. a packed image).  Page lists are device arrays.
+struct PageCopy {
+    const unsigned char* src;
+    unsigned char* dst;
+    size_t src_layer_stride, dst_layer_stride;
+    const int32_t* src_pages;
+    const int32_t* dst_pages;
+    int n_pages, n_layers;
+    uint32_t page_bytes;
+};
+int launch_kv_page_copy(const PageCopy& p, int sm_count, cudaStream_t st);
+
 // Opt-in shared-memory attributes etc.; call once per device before the first launch.
 cudaError_t init_kernels();
 

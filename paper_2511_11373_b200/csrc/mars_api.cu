@@ -206,7 +206,7 @@ struct mars_kv {
     int max_seqs;
     std::vector<SeqState> seqs;
     std::vector<int32_t> free_list;   // stack of free page ids
-    std::vector<uint8_t> owned;
+    std::vector<int32_t> refs;        // number of sequence slots that list the page (0 = free)
 };
 
 extern "C" {
@@ -419,7 +419,7 @@ mars_status_t mars_kv_alloc(mars_model_t* m, void* k_pool, void* v_pool, size_t 
     cudaError_t e = cudaMemset(meta, 0, mars_kv_meta_bytes(max_seqs, max_pages_per_seq));
     if (e != cudaSuccess) { g_last_cuda_error = (int32_t)e; delete kv; return MARS_ERR_CUDA; }
     kv->seqs.resize(max_seqs);
-    kv->owned.assign(n_pages, 0);
+    kv->refs.assign(n_pages, 0);
     kv->free_list.resize(n_pages);
     for (size_t i = 0; i < n_pages; ++i) kv->free_list[i] = (int32_t)(n_pages - 1 - i);   // page 0 is handed out first
     *out = kv;
@@ -442,6 +442,13 @@ static mars_status_t upload_row(mars_kv* kv, int seq, int first, int count) {
     return MARS_OK;
 }
 
+// The page that receives position `len` must belong to this slot alone (pages shared by
+// mars_kv_seq_fork hold only positions below the fork point and are never written again).
+static bool next_write_is_private(const mars_kv* kv, const SeqState& s, int len) {
+    const size_t idx = (size_t)(len / kv->view.page_size);
+    return idx >= s.pages.size() || kv->refs[s.pages[idx]] == 1;
+}
+
 mars_status_t mars_kv_seq_reserve(mars_kv_t* kv, int32_t seq, int32_t n_tokens_total) {
     if (!kv || seq < 0 || seq >= kv->max_seqs) return MARS_ERR_BAD_HANDLE;
     if (n_tokens_total < 0 || n_tokens_total > kv->model->cfg.max_pos) return MARS_ERR_INVALID_ARG;
@@ -454,7 +461,7 @@ mars_status_t mars_kv_seq_reserve(mars_kv_t* kv, int32_t seq, int32_t n_tokens_t
     for (int i = have; i < need; ++i) {
         const int32_t p = kv->free_list.back();
         kv->free_list.pop_back();
-        kv->owned[p] = 1;
+        kv->refs[p] = 1;
         s.pages.push_back(p);
     }
     s.used = true;
@@ -472,9 +479,9 @@ mars_status_t mars_kv_seq_adopt(mars_kv_t* kv, int32_t seq, const int32_t* pages
     std::sort(sorted.begin(), sorted.end());
     for (int i = 0; i < n_pages; ++i) {
         if (sorted[i] < 0 || sorted[i] >= kv->view.n_pages) return MARS_ERR_INVALID_ARG;
-        if (kv->owned[sorted[i]] || (i > 0 && sorted[i] == sorted[i - 1])) return MARS_ERR_BAD_HANDLE;
+        if (kv->refs[sorted[i]] || (i > 0 && sorted[i] == sorted[i - 1])) return MARS_ERR_BAD_HANDLE;
     }
-    for (int i = 0; i < n_pages; ++i) kv->owned[pages[i]] = 1;
+    for (int i = 0; i < n_pages; ++i) kv->refs[pages[i]] = 1;
     kv->free_list.erase(std::remove_if(kv->free_list.begin(), kv->free_list.end(),
                                        [&](int32_t p) { return std::binary_search(sorted.begin(), sorted.end(), p); }),
                         kv->free_list.end());
@@ -488,6 +495,7 @@ mars_status_t mars_kv_seq_set_len(mars_kv_t* kv, int32_t seq, int32_t ctx_len) {
     if (!kv || seq < 0 || seq >= kv->max_seqs || !kv->seqs[seq].used) return MARS_ERR_BAD_HANDLE;
     if (ctx_len < 0 || (int64_t)ctx_len > (int64_t)kv->seqs[seq].pages.size() * kv->view.page_size)
         return MARS_ERR_INVALID_ARG;
+    if (!next_write_is_private(kv, kv->seqs[seq], ctx_len)) return MARS_ERR_INVALID_ARG;   // would append into a shared page
     kv->seqs[seq].len = ctx_len;
     return MARS_OK;
 }
@@ -495,10 +503,8 @@ mars_status_t mars_kv_seq_set_len(mars_kv_t* kv, int32_t seq, int32_t ctx_len) {
 mars_status_t mars_kv_seq_release(mars_kv_t* kv, int32_t seq) {
     if (!kv || seq < 0 || seq >= kv->max_seqs || !kv->seqs[seq].used) return MARS_ERR_BAD_HANDLE;
     SeqState& s = kv->seqs[seq];
-    for (auto it = s.pages.rbegin(); it != s.pages.rend(); ++it) {
-        kv->owned[*it] = 0;
-        kv->free_list.push_back(*it);
-    }
+    for (auto it = s.pages.rbegin(); it != s.pages.rend(); ++it)
+        if (--kv->refs[*it] == 0) kv->free_list.push_back(*it);   // shared pages stay until their last holder goes
     s = SeqState();
     return MARS_OK;
 }
@@ -515,6 +521,133 @@ mars_status_t mars_kv_block_table(const mars_kv_t* kv, int32_t seq, int32_t* pag
     *n = (int32_t)p.size();
     for (int i = 0; i < std::min<int>(cap, (int)p.size()); ++i) pages_out[i] = p[i];
     return MARS_OK;
+}
+
+// ---- parking, resuming and forking a sequence (segment rollouts, grouped agent rollouts)
+
+static size_t layer_page_bytes(const mars_kv* kv) {
+    const mars_config_t& c = kv->model->cfg;
+    return (size_t)c.n_kv_heads * kv->view.page_size * c.head_dim * 2;
+}
+
+size_t mars_kv_seq_image_bytes(const mars_kv_t* kv, int32_t n_tokens) {
+    if (!kv || n_tokens < 0) return 0;
+    const int ps = kv->view.page_size;
+    return 2 * (size_t)kv->model->cfg.n_layers * (size_t)((n_tokens + ps - 1) / ps) * layer_page_bytes(kv);
+}
+
+// A kernel will read or write `p`: it must be device memory or page-locked host memory.
+static mars_status_t kernel_visible(const void* p, unsigned char** dev_ptr) {
+    cudaPointerAttributes attr;
+    CUDA_TRY(cudaPointerGetAttributes(&attr, p));
+    if (attr.type == cudaMemoryTypeUnregistered || !attr.devicePointer) return MARS_ERR_INVALID_ARG;
+    *dev_ptr = (unsigned char*)attr.devicePointer;
+    return MARS_OK;
+}
+
+// Packed image: [K | V][layer][page index in the sequence][n_kv_heads][page_size][head_dim].
+static mars_status_t move_image(mars_kv* kv, int seq, unsigned char* image, int n_pages, bool to_image, cudaStream_t st) {
+    const mars_config_t& c = kv->model->cfg;
+    const size_t pb = layer_page_bytes(kv);
+    const int32_t* row = kv->view.block_table + (size_t)seq * kv->view.max_pages_per_seq;
+    for (int which = 0; which < 2; ++which) {
+        unsigned char* pool = (unsigned char*)(which ? kv->view.v_pool : kv->view.k_pool);
+        unsigned char* img = image + (size_t)which * c.n_layers * n_pages * pb;
+        PageCopy pc;
+        pc.n_pages = n_pages; pc.n_layers = c.n_layers; pc.page_bytes = (uint32_t)pb;
+        if (to_image) {
+            pc.src = pool; pc.src_layer_stride = (size_t)kv->view.n_pages * pb; pc.src_pages = row;
+            pc.dst = img;  pc.dst_layer_stride = (size_t)n_pages * pb;          pc.dst_pages = nullptr;
+        } else {
+            pc.src = img;  pc.src_layer_stride = (size_t)n_pages * pb;          pc.src_pages = nullptr;
+            pc.dst = pool; pc.dst_layer_stride = (size_t)kv->view.n_pages * pb; pc.dst_pages = row;
+        }
+        launch_kv_page_copy(pc, kv->model->sm_count, st);
+    }
+    CUDA_TRY(cudaGetLastError());
+    kv->model->last_stream = st;
+    return MARS_OK;
+}
+
+mars_status_t mars_kv_seq_export(mars_kv_t* kv, int32_t seq, void* image, size_t image_bytes, void* cuda_stream) {
+    if (!kv || seq < 0 || seq >= kv->max_seqs || !kv->seqs[seq].used) return MARS_ERR_BAD_HANDLE;
+    const SeqState& s = kv->seqs[seq];
+    const size_t need = mars_kv_seq_image_bytes(kv, s.len);
+    if (!image || image_bytes < need || (uintptr_t)image % 16) return MARS_ERR_INVALID_ARG;
+    if (need == 0) return MARS_OK;
+    unsigned char* img = nullptr;
+    const mars_status_t rc = kernel_visible(image, &img);
+    if (rc != MARS_OK) return rc;
+    const int ps = kv->view.page_size;
+    return move_image(kv, seq, img, (s.len + ps - 1) / ps, true, (cudaStream_t)cuda_stream);
+}
+
+mars_status_t mars_kv_seq_import(mars_kv_t* kv, int32_t seq, const void* image, size_t image_bytes, int32_t n_tokens,
+                                 void* cuda_stream) {
+    if (!kv || seq < 0 || seq >= kv->max_seqs || kv->seqs[seq].used) return MARS_ERR_BAD_HANDLE;
+    if (n_tokens < 0 || n_tokens > kv->model->cfg.max_pos) return MARS_ERR_INVALID_ARG;
+    const size_t need = mars_kv_seq_image_bytes(kv, n_tokens);
+    if (!image || image_bytes < need || (uintptr_t)image % 16) return MARS_ERR_INVALID_ARG;
+    unsigned char* img = nullptr;
+    if (need) {
+        const mars_status_t rc = kernel_visible(image, &img);
+        if (rc != MARS_OK) return rc;
+    }
+    mars_status_t rc = mars_kv_seq_reserve(kv, seq, n_tokens);
+    if (rc != MARS_OK) return rc;
+    const int ps = kv->view.page_size;
+    if (need) rc = move_image(kv, seq, img, (n_tokens + ps - 1) / ps, false, (cudaStream_t)cuda_stream);
+    if (rc != MARS_OK) {
+        mars_kv_seq_release(kv, seq);
+        return rc;
+    }
+    kv->seqs[seq].len = n_tokens;
+    return MARS_OK;
+}
+
+mars_status_t mars_kv_seq_fork(mars_kv_t* kv, int32_t src, int32_t dst, void* cuda_stream) {
+    if (!kv || src < 0 || src >= kv->max_seqs || dst < 0 || dst >= kv->max_seqs || src == dst) return MARS_ERR_BAD_HANDLE;
+    if (!kv->seqs[src].used || kv->seqs[dst].used) return MARS_ERR_BAD_HANDLE;
+    const SeqState& a = kv->seqs[src];
+    SeqState& b = kv->seqs[dst];
+    const int ps = kv->view.page_size;
+    const int full = a.len / ps;
+    const bool tail = a.len % ps != 0;
+    if (tail && kv->free_list.empty()) return MARS_ERR_KV_FULL;
+    b.pages.assign(a.pages.begin(), a.pages.begin() + full);
+    for (int32_t p : b.pages) ++kv->refs[p];
+    if (tail) {   // the page both would append to is copied, not shared
+        const int32_t p = kv->free_list.back();
+        kv->free_list.pop_back();
+        kv->refs[p] = 1;
+        b.pages.push_back(p);
+    }
+    b.len = a.len;
+    b.used = true;
+    mars_status_t rc = upload_row(kv, dst, 0, (int)b.pages.size());
+    if (rc == MARS_OK && tail) {
+        const size_t pb = layer_page_bytes(kv);
+        for (int which = 0; which < 2 && rc == MARS_OK; ++which) {
+            unsigned char* pool = (unsigned char*)(which ? kv->view.v_pool : kv->view.k_pool);
+            PageCopy pc;
+            pc.src = pool; pc.dst = pool;
+            pc.src_layer_stride = pc.dst_layer_stride = (size_t)kv->view.n_pages * pb;
+            pc.src_pages = kv->view.block_table + (size_t)src * kv->view.max_pages_per_seq + full;
+            pc.dst_pages = kv->view.block_table + (size_t)dst * kv->view.max_pages_per_seq + full;
+            pc.n_pages = 1; pc.n_layers = kv->model->cfg.n_layers; pc.page_bytes = (uint32_t)pb;
+            launch_kv_page_copy(pc, kv->model->sm_count, (cudaStream_t)cuda_stream);
+        }
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) { g_last_cuda_error = (int32_t)e; rc = MARS_ERR_CUDA; }
+        kv->model->last_stream = (cudaStream_t)cuda_stream;
+    }
+    if (rc != MARS_OK) mars_kv_seq_release(kv, dst);
+    return rc;
+}
+
+int32_t mars_kv_page_refs(const mars_kv_t* kv, int32_t page) {
+    if (!kv || page < 0 || page >= kv->view.n_pages) return -1;
+    return kv->refs[page];
 }
 
 // ------------------------------------------------------------------------------------- the step
@@ -747,6 +880,7 @@ mars_status_t mars_decode_step(mars_model_t* m, mars_kv_t* kv, void* cuda_stream
         seen[sq] = 1;
         const SeqState& s = kv->seqs[sq];
         if (s.len + 1 > m->cfg.max_pos) return MARS_ERR_INVALID_ARG;
+        if (!next_write_is_private(kv, s, s.len)) return MARS_ERR_BAD_HANDLE;
         if (s.len / ps >= (int)s.pages.size()) {
             if ((int)s.pages.size() + 1 > kv->view.max_pages_per_seq) return MARS_ERR_KV_FULL;
             ++new_pages;
@@ -761,7 +895,7 @@ mars_status_t mars_decode_step(mars_model_t* m, mars_kv_t* kv, void* cuda_stream
         if (s.len / ps >= (int)s.pages.size()) {
             const int32_t p = kv->free_list.back();
             kv->free_list.pop_back();
-            kv->owned[p] = 1;
+            kv->refs[p] = 1;
             plan.updates.push_back(sq);
             plan.updates.push_back((int32_t)s.pages.size());
             plan.updates.push_back(p);
@@ -777,7 +911,7 @@ mars_status_t mars_decode_step(mars_model_t* m, mars_kv_t* kv, void* cuda_stream
     if (r != MARS_OK) {
         for (auto it = taken.rbegin(); it != taken.rend(); ++it) {   // undo the page grabs
             kv->seqs[it->first].pages.pop_back();
-            kv->owned[it->second] = 0;
+            kv->refs[it->second] = 0;
             kv->free_list.push_back(it->second);
         }
         return r;
@@ -806,6 +940,7 @@ mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stre
         const SeqState& s = kv->seqs[sq];
         const int64_t end = (int64_t)s.len + chunk_lens[r];
         if (end > m->cfg.max_pos) return MARS_ERR_INVALID_ARG;
+        if (!next_write_is_private(kv, s, s.len)) return MARS_ERR_BAD_HANDLE;
         const int64_t need = (end + ps - 1) / ps;
         if (need > kv->view.max_pages_per_seq) return MARS_ERR_KV_FULL;
         new_pages += std::max<int64_t>(0, need - (int64_t)s.pages.size());
@@ -831,7 +966,7 @@ mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stre
         while ((int)s.pages.size() < need) {
             const int32_t p = kv->free_list.back();
             kv->free_list.pop_back();
-            kv->owned[p] = 1;
+            kv->refs[p] = 1;
             plan.updates.push_back(sq);
             plan.updates.push_back((int32_t)s.pages.size());
             plan.updates.push_back(p);
@@ -852,7 +987,7 @@ mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stre
     if (st != MARS_OK) {
         for (auto it = taken.rbegin(); it != taken.rend(); ++it) {
             kv->seqs[it->first].pages.pop_back();
-            kv->owned[it->second] = 0;
+            kv->refs[it->second] = 0;
             kv->free_list.push_back(it->second);
         }
         return st;
