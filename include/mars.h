@@ -204,6 +204,27 @@ MARS_API mars_status_t mars_prefill_chunk(mars_model_t *model, mars_kv_t *kv, vo
                                  const int32_t *emit_last, const mars_sampling_t *sampling, int32_t *out_tokens,
                                  float *out_logprobs, const mars_debug_t *debug);
 
+/* mars_score_chunk: teacher-forced scoring of tokens that are already known -- the pass that gives
+ * log pi_theta(o_t | q, o_<t) for every position of a response, i.e. the numerator of the importance
+ * ratio (Eq. 3) under the current weights, or the behaviour-policy term when it is recomputed.
+ * Arguments and cache effects are those of mars_prefill_chunk (the chunk tokens are appended to
+ * their sequences with causal attention; several calls may score one long response chunk by
+ * chunk), but nothing is sampled.  Instead, for every token row i of the call (requests
+ * concatenated, as in `tokens`):
+ *   out_logprobs[i] = log softmax(logits_i / temperature)[targets[i]]      when targets[i] >= 0,
+ *   out_logprobs[i] = 0                                                   when targets[i] <  0
+ * over the full vocabulary, where logits_i is the model output at that row's position; for a
+ * response the caller passes targets[i] = the token at the next position and -1 on prompt rows and
+ * on the last row.  targets, out_logprobs: device arrays of sum(chunk_lens) entries.  A target
+ * >= vocab writes 0 and is reported by mars_poll_status (MARS_ERR_BAD_TOKEN).  The logits are never
+ * materialised (debug->logits, if given, receives [rows, vocab] fp32; the other taps as usual).
+ * MARS_ERR_UNSUPPORTED when vocab / 256 exceeds top_k * hidden / 2 (the softmax partials borrow
+ * the expert-output workspace). */
+MARS_API mars_status_t mars_score_chunk(mars_model_t *model, mars_kv_t *kv, void *cuda_stream, int32_t n_reqs,
+                                        const int32_t *seq_ids, const int32_t *chunk_lens, const int32_t *tokens,
+                                        const int32_t *targets, float temperature, float *out_logprobs,
+                                        const mars_debug_t *debug);
+
 /* Host-buffer convenience for callers that keep tokens on the host: copies in_tokens to the
  * device, runs mars_decode_step, copies the results back and synchronises the stream. */
 MARS_API mars_status_t mars_decode_step_host(mars_model_t *model, mars_kv_t *kv, void *cuda_stream, int32_t n_seqs,

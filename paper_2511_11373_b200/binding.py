@@ -88,6 +88,8 @@ SIGNATURES = {
     "mars_prefill_chunk": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), POINTER(c_int32), c_void_p,
                                      POINTER(c_int32), POINTER(mars_sampling_t), c_void_p, c_void_p,
                                      POINTER(mars_debug_t)]),
+    "mars_score_chunk": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), POINTER(c_int32), c_void_p,
+                                   c_void_p, ctypes.c_float, c_void_p, POINTER(mars_debug_t)]),
     "mars_decode_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), c_void_p,
                                         POINTER(mars_sampling_t), c_void_p, c_void_p]),
     "mars_decode_step_static": (c_int32, [POINTER(mars_config_t), POINTER(mars_weights_t), c_void_p, c_void_p, c_size_t,
@@ -329,6 +331,16 @@ def mars_prefill_chunk(model: Model, kv: KvCache, seq_ids, chunk_lens, tokens: t
     return lib().mars_prefill_chunk(model.handle, kv.handle, _stream_handle(stream), n, ids, lens, _ptr(tokens), emit,
                                     byref(sampling), _ptr(out_tokens), _ptr(out_logprobs),
                                     byref(debug) if debug is not None else None)
+
+
+def mars_score_chunk(model: Model, kv: KvCache, seq_ids, chunk_lens, tokens: torch.Tensor, targets: torch.Tensor,
+                     temperature: float, out_logprobs: torch.Tensor, debug: mars_debug_t | None = None, stream=None) -> int:
+    """Teacher-forced log-probs of `targets` (one per token row, < 0 = none); returns the status code."""
+    ids, n = _i32_array(seq_ids)
+    lens, _ = _i32_array(chunk_lens)
+    return lib().mars_score_chunk(model.handle, kv.handle, _stream_handle(stream), n, ids, lens, _ptr(tokens),
+                                  _ptr(targets), float(temperature), _ptr(out_logprobs),
+                                  byref(debug) if debug is not None else None)
 
 
 def mars_decode_step_host(model: Model, kv: KvCache, seq_ids, in_tokens_host: torch.Tensor, sampling: mars_sampling_t,

@@ -60,6 +60,12 @@ int launch_umma_swap(const CUtensorMap& tm_w, const CUtensorMap& tm_x, int rows,
                      int32_t* err, cudaStream_t st);
 int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_xperm, const CUtensorMap& tm_wgu,
                         const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, cudaStream_t st);
+// Scoring pass: out_logprobs[row] = log softmax(lm_head(h[row]) * inv_temp)[targets[row]] (0 where the
+// target is negative).  score_ml: [score_vocab_tiles(vocab)][n_rows] scratch, score_tgt: [n_rows] scratch.
+int score_vocab_tiles(int vocab);
+int launch_umma_score(const CUtensorMap& tm_h, const CUtensorMap& tm_lm, int n_rows, int vocab, int K,
+                      const int32_t* targets, float inv_temp, float2* score_ml, float* score_tgt, float* logits_tap,
+                      float* out_logprobs, int32_t* err, cudaStream_t st);
 int launch_qkv_post(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
                     int n_tok, int ksplit, cudaStream_t st);
 int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st);

@@ -113,10 +113,18 @@ struct UmmaParams {
     const int32_t* n_groups;
     int b_rows_per_expert;    // rows of B per expert (grouped calls)
     int n_cols;               // output columns (store mode) or expert_inter (SwiGLU mode)
-    int swiglu;               // 0: out[m][n_cols] fp32; 1: act[m][2][n_cols] from (gate, up) column halves
-    float* out;
+    int swiglu;               // 0: out[m][n_cols] fp32; 1: act[m][2][n_cols] from (gate, up) column halves;
+                              // 2: per-row softmax statistics of the tile's columns (scoring pass, see below)
+    float* out;               // mode 2: optional copy of the raw logits [m][n_cols], or null
     __nv_bfloat16* act;
     int32_t* err;
+    // mode 2: the columns are vocabulary entries; z = logit * inv_temp.  Column tile x writes, for each of
+    // its rows, (max z, sum exp(z - max)) to score_ml[x * m_rows + row]; the tile that holds column
+    // targets[row] also writes that z to score_tgt[row].
+    const int32_t* targets;
+    float inv_temp;
+    float2* score_ml;
+    float* score_tgt;
 };
 
 __global__ void __launch_bounds__(kUmThreads, 1)
@@ -222,6 +230,43 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                                     make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
                                                 __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
                     }
+                }
+            } else if (p.swiglu == 2) {
+                const bool live = r < m_valid;
+                const int tgt = live ? p.targets[m0 + r] : -1;
+                float mx = -INFINITY, sum = 0.f, zt = 0.f;
+#pragma unroll 1
+                for (int c = 0; c < kUmTileN; c += 32) {
+                    uint32_t v[32];
+                    um_ld32(lane_base + c, v);
+                    const int cbase = col0 + c;
+                    if (live && cbase < p.n_cols) {
+                        float cm = -INFINITY;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (cbase + j < p.n_cols) cm = fmaxf(cm, __uint_as_float(v[j]) * p.inv_temp);
+                        const float nm = fmaxf(mx, cm);
+                        float add = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (cbase + j < p.n_cols) {
+                                const float z = __uint_as_float(v[j]) * p.inv_temp;
+                                add += __expf(z - nm);
+                                if (cbase + j == tgt) zt = z;
+                            }
+                        sum = sum * __expf(mx - nm) + add;     // exp(-inf) = 0 on the first chunk
+                        mx = nm;
+                        if (p.out) {
+                            float* dst = p.out + (size_t)(m0 + r) * p.n_cols + cbase;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (cbase + j < p.n_cols) dst[j] = __uint_as_float(v[j]);
+                        }
+                    }
+                }
+                if (live) {
+                    p.score_ml[(size_t)blockIdx.x * p.m_rows + m0 + r] = make_float2(mx, sum);
+                    if (tgt >= col0 && tgt < col0 + kUmTileN && tgt < p.n_cols) p.score_tgt[m0 + r] = zt;
                 }
             } else {
 #pragma unroll 1
@@ -387,7 +432,7 @@ static size_t umma_smem_bytes() { return (size_t)kUmStages * kUmStageBytes + 102
 
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
                       int32_t* err, cudaStream_t st) {
-    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err};
+    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err, nullptr, 0.f, nullptr, nullptr};
     dim3 grid((n_cols + kUmTileN - 1) / kUmTileN, (m_rows + kUmTileM - 1) / kUmTileM);
     umma_gemm_kernel<<<grid, kUmThreads, umma_smem_bytes(), st>>>(tm_a, tm_b, p);
     return 1;
@@ -398,13 +443,56 @@ int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_
     const int n_slots = n_tok * s.k;
     const int max_groups = s.E + (n_slots + kUmTileM - 1) / kUmTileM;
     gather_rows_kernel<<<n_slots, 256, 0, st>>>(b, s.H, n_slots);
-    UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err};
+    UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err, nullptr, 0.f, nullptr, nullptr};
     umma_gemm_kernel<<<dim3((s.I + 127) / 128, max_groups), kUmThreads, umma_smem_bytes(), st>>>(tm_xperm, tm_wgu, gu);
-    UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err};
+    UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err, nullptr, 0.f, nullptr, nullptr};
     umma_gemm_kernel<<<dim3((s.H + kUmTileN - 1) / kUmTileN, max_groups), kUmThreads, umma_smem_bytes(), st>>>(
         tm_act, tm_wdown, dn);
     return 3;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Teacher-forced scoring: log pi(target | prefix) = z_target - logsumexp(z) over the vocabulary, for
+// every token row, without materialising the logits.  The contraction above leaves one (max, sum)
+// pair per row and 256-column vocabulary tile; a warp per row merges them in a fixed order.
+__global__ void __launch_bounds__(256) score_combine_kernel(const float2* __restrict__ ml, const float* __restrict__ zt,
+                                                            const int32_t* __restrict__ targets, int n_rows, int n_tiles,
+                                                            int vocab, float* __restrict__ out, int32_t* err) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (row >= n_rows) return;
+    const int tgt = targets[row];
+    if (tgt < 0 || tgt >= vocab) {             // negative: no target at this position; too large: reported
+        if (lane == 0) {
+            out[row] = 0.f;
+            if (tgt >= vocab) atomicOr(err, kErrBadToken);
+        }
+        return;
+    }
+    float m = -INFINITY, l = 0.f;
+    for (int t = lane; t < n_tiles; t += 32) {
+        const float2 p = ml[(size_t)t * n_rows + row];
+        const float nm = fmaxf(m, p.x);
+        l = l * __expf(m - nm) + p.y * __expf(p.x - nm);
+        m = nm;
+    }
+    const float M = warp_max(m);
+    l = warp_sum(m == -INFINITY ? 0.f : l * __expf(m - M));
+    if (lane == 0) out[row] = zt[row] - (M + logf(l));
+}
+
+int launch_umma_score(const CUtensorMap& tm_h, const CUtensorMap& tm_lm, int n_rows, int vocab, int K,
+                      const int32_t* targets, float inv_temp, float2* score_ml, float* score_tgt, float* logits_tap,
+                      float* out_logprobs, int32_t* err, cudaStream_t st) {
+    UmmaParams p{K, n_rows, nullptr, nullptr, 0, vocab, 2, logits_tap, nullptr, err, targets, inv_temp, score_ml, score_tgt};
+    const int n_tiles = (vocab + kUmTileN - 1) / kUmTileN;
+    dim3 grid(n_tiles, (n_rows + kUmTileM - 1) / kUmTileM);
+    umma_gemm_kernel<<<grid, kUmThreads, umma_smem_bytes(), st>>>(tm_h, tm_lm, p);
+    score_combine_kernel<<<(n_rows + 7) / 8, 256, 0, st>>>(score_ml, score_tgt, targets, n_rows, n_tiles, vocab,
+                                                            out_logprobs, err);
+    return 2;
+}
+
+int score_vocab_tiles(int vocab) { return (vocab + kUmTileN - 1) / kUmTileN; }
 
 cudaError_t init_umma_kernels() {
     cudaError_t e = cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes());

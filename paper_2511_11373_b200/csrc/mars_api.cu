@@ -326,6 +326,7 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
         m->tm_wgu.resize(cfg->n_layers); m->tm_wdown.resize(cfg->n_layers); m->tm_router.resize(cfg->n_layers);
         mars_status_t rc = make_weight_map(&m->tm_lm, m->lm_head, (uint64_t)cfg->vocab, H);
         if (rc == MARS_OK) rc = make_pair_map(&m->tm_h64, m->buf.h, n, H, 64);
+        if (rc == MARS_OK) rc = make_pair_map(&m->tm_h, m->buf.h, n, H);   // 128-row boxes (scoring pass, prefill)
         if (rc == MARS_OK) rc = make_pair_map(&m->tm_o64, m->buf.o, n, QD, 64);
         for (int l = 0; l < cfg->n_layers && rc == MARS_OK; ++l) {
             const LayerW& q = m->layers[l];
@@ -337,7 +338,6 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_router[l], q.router, E, H);
         }
         if (big) {
-            if (rc == MARS_OK) rc = make_pair_map(&m->tm_h, m->buf.h, n, H);
             if (rc == MARS_OK) rc = make_pair_map(&m->tm_o, m->buf.o, n, QD);
             if (rc == MARS_OK) rc = make_pair_map(&m->tm_xperm, m->buf.xperm, slots, H);
             if (rc == MARS_OK) rc = make_pair_map(&m->tm_act, m->buf.act, slots, I);
@@ -659,6 +659,8 @@ struct StepPlan {
     const int32_t* tokens_dev;
     int span;   // cached tokens per attention item (decode)
     bool prefill = false;   // attention items are blocks of consecutive prompt tokens (causal kernel)
+    const int32_t* score_targets = nullptr;   // scoring pass: device [n_tok] target token per row (< 0: none)
+    float score_temperature = 1.f;
 };
 
 mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPlan& plan, const mars_sampling_t& smp,
@@ -849,6 +851,15 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             return launch_sample(s, b, lay, n_emit, out_tokens, out_logprobs, taps.nucleus_mass, st);
         });
     }
+    if (plan.score_targets) {
+        // the last combine left rms(x) * final_norm of EVERY row in b.h; the expert outputs in b.y are dead
+        float2* ml = reinterpret_cast<float2*>(b.y);
+        float* zt = b.y + 2 * (size_t)score_vocab_tiles(s.V) * n_tok;
+        run(MARS_K_LM_HEAD, [&] {
+            return launch_umma_score(m->tm_h, m->tm_lm, n_tok, s.V, s.H, plan.score_targets, 1.f / plan.score_temperature,
+                                     ml, zt, dbg ? dbg->logits : nullptr, out_logprobs, b.err, st);
+        });
+    }
     CUDA_TRY(ev_err);
     CUDA_TRY(cudaGetLastError());
     m->last_stream = st;
@@ -920,10 +931,13 @@ mars_status_t mars_decode_step(mars_model_t* m, mars_kv_t* kv, void* cuda_stream
     return MARS_OK;
 }
 
-mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_reqs,
+// Chunks of prompt tokens appended to their sequences: with score_targets == null the prefill call
+// (sampling from the last position where asked), otherwise the scoring pass (a log-prob per row).
+static mars_status_t feed_chunks(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_reqs,
                                  const int32_t* seq_ids, const int32_t* chunk_lens, const int32_t* tokens,
                                  const int32_t* emit_last, const mars_sampling_t* sampling, int32_t* out_tokens,
-                                 float* out_logprobs, const mars_debug_t* debug) {
+                                 float* out_logprobs, const mars_debug_t* debug, const int32_t* score_targets,
+                                 float score_temperature) {
     if (!m || !kv || kv->model != m) return MARS_ERR_BAD_HANDLE;
     if (!seq_ids || !chunk_lens || !tokens || !sampling || n_reqs < 1) return MARS_ERR_INVALID_ARG;
     if (!sampling->greedy && (!(sampling->temperature > 0.f) || !(sampling->top_p > 0.f) || sampling->top_p > 1.f))
@@ -956,6 +970,8 @@ mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stre
     plan.tokens_dev = tokens;
     plan.span = 1 << 30;
     plan.prefill = true;   // attention items are blocks of consecutive prompt tokens
+    plan.score_targets = score_targets;
+    plan.score_temperature = score_temperature;
     std::vector<std::pair<int, int32_t>> taken;
     int row = 0;
     for (int r = 0; r < n_reqs; ++r) {
@@ -994,6 +1010,28 @@ mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stre
     }
     for (int r = 0; r < n_reqs; ++r) kv->seqs[seq_ids[r]].len += chunk_lens[r];
     return MARS_OK;
+}
+
+mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_reqs,
+                                 const int32_t* seq_ids, const int32_t* chunk_lens, const int32_t* tokens,
+                                 const int32_t* emit_last, const mars_sampling_t* sampling, int32_t* out_tokens,
+                                 float* out_logprobs, const mars_debug_t* debug) {
+    return feed_chunks(m, kv, cuda_stream, n_reqs, seq_ids, chunk_lens, tokens, emit_last, sampling, out_tokens,
+                       out_logprobs, debug, nullptr, 1.f);
+}
+
+mars_status_t mars_score_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_reqs, const int32_t* seq_ids,
+                               const int32_t* chunk_lens, const int32_t* tokens, const int32_t* targets,
+                               float temperature, float* out_logprobs, const mars_debug_t* debug) {
+    if (!m) return MARS_ERR_BAD_HANDLE;
+    if (!targets || !out_logprobs || !(temperature > 0.f)) return MARS_ERR_INVALID_ARG;
+    // the per-tile softmax statistics borrow the expert-output buffer: [tiles][rows] pairs + [rows]
+    if ((size_t)score_vocab_tiles(m->cfg.vocab) * 8 + 4 > (size_t)m->cfg.top_k * m->cfg.hidden * 4) return MARS_ERR_UNSUPPORTED;
+    mars_sampling_t none;
+    std::memset(&none, 0, sizeof(none));
+    none.greedy = 1; none.temperature = 1.f; none.top_p = 1.f;
+    return feed_chunks(m, kv, cuda_stream, n_reqs, seq_ids, chunk_lens, tokens, nullptr, &none, nullptr, out_logprobs,
+                       debug, targets, temperature);
 }
 
 mars_status_t mars_decode_step_host(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_seqs,
