@@ -222,6 +222,20 @@ def test_config4_mixed_batch_decode_and_prefill(full_weights):
     kv.seq_release(slot)
     del hidden, ridx, rw
 
+    # --- the same chunk through the scoring pass: log-probs of sampled rows against the oracle (T = 0.85)
+    kv.seq_adopt(slot, pages[slot], prior)
+    tgt = torch.cat([ptoks[1:], ptoks[:1]]).to(torch.int32)
+    slp = torch.empty(n, device=DEV)
+    st = binding.mars_score_chunk(m, kv, [slot], [n], ptoks.to(DEV), tgt.to(DEV), 0.85, slp)
+    assert st == 0 and m.poll_status() == 0
+    rows = [0, 17, 50, n - 1]
+    olog = oracle.lm_head(oracle.Config(**model), full_weights["final_norm"].cpu(), full_weights["lm_head"].cpu(),
+                          x[torch.tensor(rows)].contiguous())
+    werr = max(abs(float(slp[r]) - oracle.logprob_of(olog[i].contiguous(), 0.85, int(tgt[r]))) for i, r in enumerate(rows))
+    print("config4 score chunk: max log-prob error on sampled rows", werr)
+    assert werr <= 2e-2
+    kv.seq_release(slot)
+
     # --- the benchmark's 8 x 2048 call: one call equals two half calls (same logits, same token)
     big = wl.make_tokens(R * CH, V, seed=1, name="prompts").to(DEV)
     ids = list(range(B, B + R))
@@ -251,3 +265,24 @@ def test_config4_mixed_batch_decode_and_prefill(full_weights):
     assert torch.equal(tk[0][sure], tk[1][sure])
     for s_ in ids:
         assert kv.seq_len(s_) == CH
+
+    # --- scoring the same 8 x 2048 tokens: the last row of every request must reproduce the log-prob that
+    # the prefill call's logits give to the token it sampled (vocabulary of 151936 = 593.5 column tiles)
+    for s_ in ids:
+        kv.seq_release(s_)
+        kv.seq_reserve(s_, 0)
+    tg = torch.cat([big[1:], big[:1]]).clone()
+    last = torch.arange(R, device=DEV) * CH + CH - 1
+    tg[last] = tk[0]
+    slp = torch.empty(R * CH, device=DEV)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    st = binding.mars_score_chunk(m, kv, ids, [CH] * R, big, tg, 1.0, slp)
+    e1.record()
+    assert st == 0 and m.poll_status() == 0
+    want = torch.log_softmax(lg[0].double(), -1).gather(-1, tk[0].long()[:, None])[:, 0]
+    diff = float((slp[last].double() - want).abs().max())
+    print(f"config4 score 8 x 2048: {e0.elapsed_time(e1):.1f} ms, last-row log-prob diff {diff:.2e}, "
+          f"mean log-prob {float(slp.mean()):.3f}")
+    assert diff <= 2e-3
+    assert torch.isfinite(slp).all() and float(slp.max()) <= 0.0
