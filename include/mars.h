@@ -204,6 +204,22 @@ MARS_API mars_status_t mars_prefill_chunk(mars_model_t *model, mars_kv_t *kv, vo
                                  const int32_t *emit_last, const mars_sampling_t *sampling, int32_t *out_tokens,
                                  float *out_logprobs, const mars_debug_t *debug);
 
+/* mars_mixed_step: the steady state of the agentic pipeline (Section 3.3: as soon as one agent's
+ * output is complete the next agent starts, so fresh Verifier / Corrector prompts arrive while
+ * other trajectories are still decoding) in ONE pass per layer: n_seqs decode rows (as in
+ * mars_decode_step) and n_reqs prompt chunks (as in mars_prefill_chunk) share every projection and
+ * every expert contraction, so each weight is read once for both; attention runs the span kernel on
+ * the decode rows and the causal kernel on the chunk rows.  Results are those of the two separate
+ * calls (up to fp32 summation order).  out_tokens / out_logprobs: n_seqs entries for the decode
+ * rows, then one entry per emitting request.  The slots of the two lists must be distinct.
+ * Limits: n_seqs + sum(chunk_lens) <= max(max_decode_seqs, max_prefill_tokens) of mars_model_load,
+ * and n_seqs + emitting requests <= max_decode_seqs. */
+MARS_API mars_status_t mars_mixed_step(mars_model_t *model, mars_kv_t *kv, void *cuda_stream, int32_t n_seqs,
+                                       const int32_t *seq_ids, const int32_t *in_tokens, int32_t n_reqs,
+                                       const int32_t *req_ids, const int32_t *chunk_lens, const int32_t *chunk_tokens,
+                                       const int32_t *emit_last, const mars_sampling_t *sampling, int32_t *out_tokens,
+                                       float *out_logprobs, const mars_debug_t *debug);
+
 /* mars_score_chunk: teacher-forced scoring of tokens that are already known -- the pass that gives
  * log pi_theta(o_t | q, o_<t) for every position of a response, i.e. the numerator of the importance
  * ratio (Eq. 3) under the current weights, or the behaviour-policy term when it is recomputed.

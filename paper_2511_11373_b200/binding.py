@@ -88,6 +88,9 @@ SIGNATURES = {
     "mars_prefill_chunk": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), POINTER(c_int32), c_void_p,
                                      POINTER(c_int32), POINTER(mars_sampling_t), c_void_p, c_void_p,
                                      POINTER(mars_debug_t)]),
+    "mars_mixed_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), c_void_p, c_int32,
+                                  POINTER(c_int32), POINTER(c_int32), c_void_p, POINTER(c_int32), POINTER(mars_sampling_t),
+                                  c_void_p, c_void_p, POINTER(mars_debug_t)]),
     "mars_score_chunk": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), POINTER(c_int32), c_void_p,
                                    c_void_p, ctypes.c_float, c_void_p, POINTER(mars_debug_t)]),
     "mars_decode_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), c_void_p,
@@ -331,6 +334,19 @@ def mars_prefill_chunk(model: Model, kv: KvCache, seq_ids, chunk_lens, tokens: t
     return lib().mars_prefill_chunk(model.handle, kv.handle, _stream_handle(stream), n, ids, lens, _ptr(tokens), emit,
                                     byref(sampling), _ptr(out_tokens), _ptr(out_logprobs),
                                     byref(debug) if debug is not None else None)
+
+
+def mars_mixed_step(model: Model, kv: KvCache, seq_ids, in_tokens: torch.Tensor, req_ids, chunk_lens,
+                    chunk_tokens: torch.Tensor, emit_last, sampling: mars_sampling_t, out_tokens: torch.Tensor,
+                    out_logprobs: torch.Tensor, debug: mars_debug_t | None = None, stream=None) -> int:
+    """Decode rows and prompt chunks in one pass; outputs: decode rows first, then the emitting requests."""
+    ids, n = _i32_array(seq_ids)
+    rids, nr = _i32_array(req_ids)
+    lens, _ = _i32_array(chunk_lens)
+    emit, _ = _i32_array(emit_last) if emit_last is not None else (None, 0)
+    return lib().mars_mixed_step(model.handle, kv.handle, _stream_handle(stream), n, ids, _ptr(in_tokens), nr, rids, lens,
+                                 _ptr(chunk_tokens), emit, byref(sampling), _ptr(out_tokens), _ptr(out_logprobs),
+                                 byref(debug) if debug is not None else None)
 
 
 def mars_score_chunk(model: Model, kv: KvCache, seq_ids, chunk_lens, tokens: torch.Tensor, targets: torch.Tensor,

@@ -377,8 +377,8 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     }
     __syncthreads();
 
-    const int n_units = p.step[H_NITEMS] * p.nkv;
-    const int4* items = reinterpret_cast<const int4*>(p.step + p.lay.items);
+    const int n_units = p.step[H_PF_ITEMS] * p.nkv;
+    const int4* items = reinterpret_cast<const int4*>(p.step + p.lay.items) + p.step[H_PF_FIRST];
     const uint64_t pol = l2_evict_first_policy();
     uint32_t gs = 0;
 

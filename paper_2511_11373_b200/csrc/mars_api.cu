@@ -658,7 +658,9 @@ struct StepPlan {
     std::vector<int32_t> tok_seq, tok_pos, emit_rows, emit_slot, updates;
     const int32_t* tokens_dev;
     int span;   // cached tokens per attention item (decode)
-    bool prefill = false;   // attention items are blocks of consecutive prompt tokens (causal kernel)
+    bool prefill = false;   // the call has prompt rows (blocks of consecutive tokens for the causal kernel)
+    int n_decode = 0;       // rows [0, n_decode) are decode rows (one new token attending over its cache in
+                            // spans); rows after them are prompt rows.  Set by the entry points.
     const int32_t* score_targets = nullptr;   // scoring pass: device [n_tok] target token per row (< 0: none)
     float score_temperature = 1.f;
 };
@@ -673,23 +675,24 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     int span = plan.span;
     int64_t n_items = 0;
     constexpr int kPrefillBlock = 4;   // consecutive prompt tokens per item of the causal prefill kernel
-    if (plan.prefill) {
-        for (int t = 0; t < n_tok;) {
-            int e = t + 1;
-            while (e < n_tok && e - t < kPrefillBlock && plan.tok_seq[e] == plan.tok_seq[t]) ++e;
-            t = e;
-            ++n_items;
-        }
-        if (n_items > m->caps.n_items) return MARS_ERR_INVALID_ARG;
-    } else {
-        for (;;) {
-            n_items = 0;
-            for (int t = 0; t < n_tok; ++t) n_items += ((int64_t)plan.tok_pos[t] + 1 + span - 1) / span;
-            if (n_items <= m->caps.n_items) break;
-            if (span > (1 << 28)) return MARS_ERR_INVALID_ARG;
-            span *= 2;
-        }
+    const int n_dec = plan.n_decode;
+    int64_t pf_items = 0;
+    for (int t = n_dec; t < n_tok;) {
+        int e = t + 1;
+        while (e < n_tok && e - t < kPrefillBlock && plan.tok_seq[e] == plan.tok_seq[t]) ++e;
+        t = e;
+        ++pf_items;
     }
+    if (pf_items > m->caps.n_items) return MARS_ERR_INVALID_ARG;
+    int64_t dec_items = 0;
+    for (;;) {
+        dec_items = 0;
+        for (int t = 0; t < n_dec; ++t) dec_items += ((int64_t)plan.tok_pos[t] + 1 + span - 1) / span;
+        if (dec_items + pf_items <= m->caps.n_items) break;
+        if (span > (1 << 28)) return MARS_ERR_INVALID_ARG;
+        span *= 2;
+    }
+    n_items = dec_items + pf_items;
 
     const int slot = m->next_slot;
     m->next_slot = (slot + 1) % kStagingSlots;
@@ -697,7 +700,9 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     int32_t* blk = m->staging[slot];
     std::memset(blk, 0, H_WORDS * 4);
     blk[H_NTOK] = n_tok;
-    blk[H_NITEMS] = (int32_t)n_items;
+    blk[H_NITEMS] = (int32_t)dec_items;
+    blk[H_PF_FIRST] = (int32_t)dec_items;
+    blk[H_PF_ITEMS] = (int32_t)pf_items;
     blk[H_NUPDATES] = (int32_t)(plan.updates.size() / 3);
     blk[H_NEMIT] = n_emit;
     blk[H_GREEDY] = smp.greedy ? 1 : 0;
@@ -719,32 +724,29 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         int32_t* items = blk + lay.items;
         int32_t* off = blk + lay.tok_item_off;
         int at = 0;
-        if (plan.prefill) {
-            // blocks of consecutive tokens of one request: (first row, 0, keys visible to the last one, count)
-            for (int t = 0; t < n_tok;) {
-                int e = t + 1;
-                while (e < n_tok && e - t < kPrefillBlock && plan.tok_seq[e] == plan.tok_seq[t]) ++e;
+        for (int t = 0; t < n_dec; ++t) {
+            off[t] = at;
+            const int len = plan.tok_pos[t] + 1;
+            kv_tokens += len;
+            for (int s0 = 0; s0 < len; s0 += span) {
                 items[4 * at + 0] = t;
-                items[4 * at + 1] = 0;
-                items[4 * at + 2] = plan.tok_pos[e - 1] + 1;
-                items[4 * at + 3] = e - t;
-                for (int q = t; q < e; ++q) { off[q] = at; kv_tokens += plan.tok_pos[q] + 1; }
+                items[4 * at + 1] = s0;
+                items[4 * at + 2] = std::min(span, len - s0);
+                items[4 * at + 3] = 0;
                 ++at;
-                t = e;
             }
-        } else {
-            for (int t = 0; t < n_tok; ++t) {
-                off[t] = at;
-                const int len = plan.tok_pos[t] + 1;
-                kv_tokens += len;
-                for (int s0 = 0; s0 < len; s0 += span) {
-                    items[4 * at + 0] = t;
-                    items[4 * at + 1] = s0;
-                    items[4 * at + 2] = std::min(span, len - s0);
-                    items[4 * at + 3] = 0;
-                    ++at;
-                }
-            }
+        }
+        // blocks of consecutive tokens of one request: (first row, 0, keys visible to the last one, count)
+        for (int t = n_dec; t < n_tok;) {
+            int e = t + 1;
+            while (e < n_tok && e - t < kPrefillBlock && plan.tok_seq[e] == plan.tok_seq[t]) ++e;
+            items[4 * at + 0] = t;
+            items[4 * at + 1] = 0;
+            items[4 * at + 2] = plan.tok_pos[e - 1] + 1;
+            items[4 * at + 3] = e - t;
+            for (int q = t; q < e; ++q) { off[q] = at; kv_tokens += plan.tok_pos[q] + 1; }
+            ++at;
+            t = e;
         }
         off[n_tok] = at;
     }
@@ -802,13 +804,14 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
                 return n + launch_qkv_post(s, b, lay, w, kv->view, l, n_tok, ksplit, st);
             });
         }
-        if (plan.prefill) {   // causal kernel over blocks of prompt tokens; writes the merged output itself
+        if (n_dec > 0) {      // decode rows: spans of cached tokens, then the merge of each row's spans
+            run(MARS_K_ATTN, [&] { return launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st); });
+            run(MARS_K_ATTN_MERGE, [&] { return launch_attn_merge(s, b, lay, n_dec, st); });
+        }
+        if (n_dec < n_tok) {  // prompt rows: causal kernel over blocks of tokens; writes the merged output itself
             run(MARS_K_ATTN, [&] {
                 return launch_attention_prefill(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st);
             });
-        } else {
-            run(MARS_K_ATTN, [&] { return launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st); });
-            run(MARS_K_ATTN_MERGE, [&] { return launch_attn_merge(s, b, lay, n_tok, st); });
         }
         if (umma) {
             run(MARS_K_OPROJ, [&] {
@@ -883,6 +886,7 @@ mars_status_t mars_decode_step(mars_model_t* m, mars_kv_t* kv, void* cuda_stream
     StepPlan plan;
     plan.tokens_dev = in_tokens;
     plan.span = kSpanTokens;
+    plan.n_decode = n_seqs;
     std::vector<uint8_t> seen(kv->max_seqs, 0);
     int new_pages = 0;
     for (int i = 0; i < n_seqs; ++i) {
@@ -931,21 +935,36 @@ mars_status_t mars_decode_step(mars_model_t* m, mars_kv_t* kv, void* cuda_stream
     return MARS_OK;
 }
 
-// Chunks of prompt tokens appended to their sequences: with score_targets == null the prefill call
-// (sampling from the last position where asked), otherwise the scoring pass (a log-prob per row).
-static mars_status_t feed_chunks(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_reqs,
-                                 const int32_t* seq_ids, const int32_t* chunk_lens, const int32_t* tokens,
-                                 const int32_t* emit_last, const mars_sampling_t* sampling, int32_t* out_tokens,
-                                 float* out_logprobs, const mars_debug_t* debug, const int32_t* score_targets,
-                                 float score_temperature) {
+// Chunks of prompt tokens appended to their sequences, optionally together with decode rows (one new
+// token per listed sequence) that travel through the same pass.  With score_targets == null this is
+// the prefill / mixed call (sampling from the decode rows and from the last position of the chunks
+// that ask for it), otherwise the scoring pass (a log-prob per row, chunks only).
+static mars_status_t feed_chunks(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_dec, const int32_t* dec_ids,
+                                 const int32_t* dec_tokens, int32_t n_reqs, const int32_t* seq_ids,
+                                 const int32_t* chunk_lens, const int32_t* tokens, const int32_t* emit_last,
+                                 const mars_sampling_t* sampling, int32_t* out_tokens, float* out_logprobs,
+                                 const mars_debug_t* debug, const int32_t* score_targets, float score_temperature) {
     if (!m || !kv || kv->model != m) return MARS_ERR_BAD_HANDLE;
-    if (!seq_ids || !chunk_lens || !tokens || !sampling || n_reqs < 1) return MARS_ERR_INVALID_ARG;
+    if (!seq_ids || !chunk_lens || !tokens || !sampling || n_reqs < 1 || n_dec < 0) return MARS_ERR_INVALID_ARG;
+    if (n_dec > 0 && (!dec_ids || !dec_tokens)) return MARS_ERR_INVALID_ARG;
     if (!sampling->greedy && (!(sampling->temperature > 0.f) || !(sampling->top_p > 0.f) || sampling->top_p > 1.f))
         return MARS_ERR_INVALID_ARG;
     const int ps = kv->view.page_size;
     int64_t total = 0, new_pages = 0;
-    int n_emit = 0;
+    int n_emit = n_dec;
     std::vector<uint8_t> seen(kv->max_seqs, 0);
+    for (int i = 0; i < n_dec; ++i) {
+        const int sq = dec_ids[i];
+        if (sq < 0 || sq >= kv->max_seqs || !kv->seqs[sq].used || seen[sq]) return MARS_ERR_BAD_HANDLE;
+        seen[sq] = 1;
+        const SeqState& s = kv->seqs[sq];
+        if (s.len + 1 > m->cfg.max_pos) return MARS_ERR_INVALID_ARG;
+        if (!next_write_is_private(kv, s, s.len)) return MARS_ERR_BAD_HANDLE;
+        if (s.len / ps >= (int)s.pages.size()) {
+            if ((int)s.pages.size() + 1 > kv->view.max_pages_per_seq) return MARS_ERR_KV_FULL;
+            ++new_pages;
+        }
+    }
     for (int r = 0; r < n_reqs; ++r) {
         const int sq = seq_ids[r];
         if (sq < 0 || sq >= kv->max_seqs || !kv->seqs[sq].used || seen[sq]) return MARS_ERR_BAD_HANDLE;
@@ -961,34 +980,46 @@ static mars_status_t feed_chunks(mars_model_t* m, mars_kv_t* kv, void* cuda_stre
         total += chunk_lens[r];
         if (emit_last && emit_last[r]) ++n_emit;
     }
-    if (total > m->max_prefill) return MARS_ERR_INVALID_ARG;
+    if (n_dec == 0 && total > m->max_prefill) return MARS_ERR_INVALID_ARG;
+    if (n_dec + total > m->caps.n_tok) return MARS_ERR_INVALID_ARG;
     if (n_emit > m->caps.n_emit) return MARS_ERR_INVALID_ARG;
     if (n_emit && (!out_tokens || !out_logprobs)) return MARS_ERR_INVALID_ARG;
     if (new_pages > (int64_t)kv->free_list.size()) return MARS_ERR_KV_FULL;
 
     StepPlan plan;
     plan.tokens_dev = tokens;
-    plan.span = 1 << 30;
-    plan.prefill = true;   // attention items are blocks of consecutive prompt tokens
+    plan.span = kSpanTokens;
+    plan.prefill = true;
+    plan.n_decode = n_dec;
     plan.score_targets = score_targets;
     plan.score_temperature = score_temperature;
     std::vector<std::pair<int, int32_t>> taken;
-    int row = 0;
+    auto take_page = [&](int sq) {
+        SeqState& s = kv->seqs[sq];
+        const int32_t p = kv->free_list.back();
+        kv->free_list.pop_back();
+        kv->refs[p] = 1;
+        plan.updates.push_back(sq);
+        plan.updates.push_back((int32_t)s.pages.size());
+        plan.updates.push_back(p);
+        s.pages.push_back(p);
+        taken.emplace_back(sq, p);
+    };
+    for (int i = 0; i < n_dec; ++i) {
+        const int sq = dec_ids[i];
+        SeqState& s = kv->seqs[sq];
+        if (s.len / ps >= (int)s.pages.size()) take_page(sq);
+        plan.tok_seq.push_back(sq);
+        plan.tok_pos.push_back(s.len);
+        plan.emit_rows.push_back(i);
+        plan.emit_slot.push_back(sq);
+    }
+    int row = n_dec;
     for (int r = 0; r < n_reqs; ++r) {
         const int sq = seq_ids[r];
         SeqState& s = kv->seqs[sq];
-        const int end = s.len + chunk_lens[r];
-        const int need = (end + ps - 1) / ps;
-        while ((int)s.pages.size() < need) {
-            const int32_t p = kv->free_list.back();
-            kv->free_list.pop_back();
-            kv->refs[p] = 1;
-            plan.updates.push_back(sq);
-            plan.updates.push_back((int32_t)s.pages.size());
-            plan.updates.push_back(p);
-            s.pages.push_back(p);
-            taken.emplace_back(sq, p);
-        }
+        const int need = (s.len + chunk_lens[r] + ps - 1) / ps;
+        while ((int)s.pages.size() < need) take_page(sq);
         for (int i = 0; i < chunk_lens[r]; ++i) {
             plan.tok_seq.push_back(sq);
             plan.tok_pos.push_back(s.len + i);
@@ -999,15 +1030,33 @@ static mars_status_t feed_chunks(mars_model_t* m, mars_kv_t* kv, void* cuda_stre
             plan.emit_slot.push_back(sq);
         }
     }
-    mars_status_t st = run_step(m, kv, (cudaStream_t)cuda_stream, plan, *sampling, out_tokens, out_logprobs, debug);
-    if (st != MARS_OK) {
+    auto undo = [&] {
         for (auto it = taken.rbegin(); it != taken.rend(); ++it) {
             kv->seqs[it->first].pages.pop_back();
             kv->refs[it->second] = 0;
             kv->free_list.push_back(it->second);
         }
+    };
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (n_dec > 0) {
+        // one token array for the embedding: decode tokens, then the chunks.  The routing-index buffer is
+        // free until the first layer's router runs, which is after the embedding has read the tokens.
+        int32_t* cat = m->buf.route_idx;
+        cudaError_t e = cudaMemcpyAsync(cat, dec_tokens, (size_t)n_dec * 4, cudaMemcpyDeviceToDevice, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(cat + n_dec, tokens, (size_t)total * 4, cudaMemcpyDeviceToDevice, stream);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int32_t)e;
+            undo();
+            return MARS_ERR_CUDA;
+        }
+        plan.tokens_dev = cat;
+    }
+    mars_status_t st = run_step(m, kv, stream, plan, *sampling, out_tokens, out_logprobs, debug);
+    if (st != MARS_OK) {
+        undo();
         return st;
     }
+    for (int i = 0; i < n_dec; ++i) kv->seqs[dec_ids[i]].len += 1;
     for (int r = 0; r < n_reqs; ++r) kv->seqs[seq_ids[r]].len += chunk_lens[r];
     return MARS_OK;
 }
@@ -1016,8 +1065,17 @@ mars_status_t mars_prefill_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stre
                                  const int32_t* seq_ids, const int32_t* chunk_lens, const int32_t* tokens,
                                  const int32_t* emit_last, const mars_sampling_t* sampling, int32_t* out_tokens,
                                  float* out_logprobs, const mars_debug_t* debug) {
-    return feed_chunks(m, kv, cuda_stream, n_reqs, seq_ids, chunk_lens, tokens, emit_last, sampling, out_tokens,
-                       out_logprobs, debug, nullptr, 1.f);
+    return feed_chunks(m, kv, cuda_stream, 0, nullptr, nullptr, n_reqs, seq_ids, chunk_lens, tokens, emit_last, sampling,
+                       out_tokens, out_logprobs, debug, nullptr, 1.f);
+}
+
+mars_status_t mars_mixed_step(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_seqs, const int32_t* seq_ids,
+                              const int32_t* in_tokens, int32_t n_reqs, const int32_t* req_ids, const int32_t* chunk_lens,
+                              const int32_t* chunk_tokens, const int32_t* emit_last, const mars_sampling_t* sampling,
+                              int32_t* out_tokens, float* out_logprobs, const mars_debug_t* debug) {
+    if (n_seqs < 1) return MARS_ERR_INVALID_ARG;
+    return feed_chunks(m, kv, cuda_stream, n_seqs, seq_ids, in_tokens, n_reqs, req_ids, chunk_lens, chunk_tokens, emit_last,
+                       sampling, out_tokens, out_logprobs, debug, nullptr, 1.f);
 }
 
 mars_status_t mars_score_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_reqs, const int32_t* seq_ids,
@@ -1030,8 +1088,8 @@ mars_status_t mars_score_chunk(mars_model_t* m, mars_kv_t* kv, void* cuda_stream
     mars_sampling_t none;
     std::memset(&none, 0, sizeof(none));
     none.greedy = 1; none.temperature = 1.f; none.top_p = 1.f;
-    return feed_chunks(m, kv, cuda_stream, n_reqs, seq_ids, chunk_lens, tokens, nullptr, &none, nullptr, out_logprobs,
-                       debug, targets, temperature);
+    return feed_chunks(m, kv, cuda_stream, 0, nullptr, nullptr, n_reqs, seq_ids, chunk_lens, tokens, nullptr, &none, nullptr,
+                       out_logprobs, debug, targets, temperature);
 }
 
 mars_status_t mars_decode_step_host(mars_model_t* m, mars_kv_t* kv, void* cuda_stream, int32_t n_seqs,

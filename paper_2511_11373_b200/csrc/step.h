@@ -13,13 +13,15 @@ constexpr int kErrTimeout = 2;
 // Header words of the step block (int32 each).
 enum StepHdr {
     H_NTOK = 0,       // token rows in this call
-    H_NITEMS = 1,     // attention work items
+    H_NITEMS = 1,     // attention work items of the decode kernel (spans of cached tokens), items [0, H_NITEMS)
     H_NUPDATES = 2,   // block-table entries to write before the step
     H_NEMIT = 3,      // rows that sample a token
     H_GREEDY = 4,
     H_TEMPERATURE = 5,  // float bits
     H_TOP_P = 6,        // float bits
     H_SEED_LO = 7, H_SEED_HI = 8, H_STEP_LO = 9, H_STEP_HI = 10,
+    H_PF_FIRST = 11,  // first work item of the causal (prompt) attention kernel; decode spans come before it
+    H_PF_ITEMS = 12,  // number of such items
     H_WORDS = 16
 };
 
