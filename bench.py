@@ -1,7 +1,7 @@
 """Benchmark of the rollout step: decode tokens/s on a Qwen3-30B-A3B-shaped MoE and the fraction of
 the HBM roofline it reaches.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 2|3|5] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 2|3|4|5|6|7|8] [--impl reference]
 
 One "step" is one pass of the whole hot path (embedding, 48 x {QKV+RoPE+append, paged attention,
 output projection, router, experts, combine}, lm_head, sampling) over the batch.  Inputs are
@@ -330,6 +330,80 @@ def run_mixed(args):
     print(json.dumps(line))
 
 
+def run_grouped(args):
+    """Grouped rollouts: G groups of M sequences, every group forked from one cached prompt (its pages
+    are held once).  Times the decode step with the shared prompt read once per block of rows and,
+    on the same state, with every row reading its whole context."""
+    from paper_2511_11373_b200 import binding
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    cfg = wl.CONFIGS[args.workload]
+    model, ps = cfg["model"], cfg["page_size"]
+    G, M, P = cfg["groups"], cfg["members"], cfg["prompt"]
+    own = wl.make_group_lengths(cfg)
+    total_steps = 2 * (args.warmup + args.steps) + 2
+    B = G * M
+    n_pages = G * wl.pages_needed(P, ps) + sum(wl.pages_needed(o + total_steps + 1, ps) + 1 for g in own for o in g) + 8
+    max_pages = wl.pages_needed(P + cfg["own_range"][1] + total_steps + 1, ps) + 2
+    weights = wl.make_weights(model, seed=0, device=device, gains="ones")
+    k_pool, v_pool = wl.make_kv_pools(model, n_pages, ps, seed=0, device=device)
+    m = binding.Model(model, weights, max_decode_seqs=B, max_prefill_tokens=0, max_pos=P + cfg["own_range"][1] + total_steps + 8)
+    kv = binding.KvCache(m, k_pool, v_pool, ps, B, max_pages)
+    for g in range(G):                                   # the prompt, then M - 1 forks, then everyone's own tokens
+        kv.seq_reserve(g * M, P)
+        kv.seq_set_len(g * M, P)
+        for j in range(1, M):
+            assert kv.seq_fork(g * M, g * M + j) == 0
+        for j in range(M):
+            kv.seq_reserve(g * M + j, P + own[g][j])
+            kv.seq_set_len(g * M + j, P + own[g][j])
+    ids = list(range(B))
+    tok_a = wl.make_tokens(B, model["vocab"], seed=0).to(device)
+    tok_b = torch.empty_like(tok_a)
+    logp = torch.empty(B, dtype=torch.float32, device=device)
+    stream = torch.cuda.current_stream()
+    step_no = 0
+    out = {}
+    peaks = load_peaks()
+    for label, share in (("shared", True), ("per_row", False)):
+        kv.share_reads(share)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler = None
+        for it in range(args.warmup + args.steps):
+            if it == args.warmup:
+                torch.cuda.synchronize()
+                sampler = ClockSampler(0)
+                e0.record(stream)
+            smp = binding.make_sampling(seed=2025, step=step_no, **cfg["sampling"])
+            st = binding.mars_decode_step(m, kv, ids, tok_a, smp, tok_b, logp)
+            assert st == 0, binding.STATUS_NAMES.get(st, st)
+            tok_a, tok_b = tok_b, tok_a
+            step_no += 1
+        e1.record(stream)
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        assert m.poll_status() == 0
+        info = m.last_step_info()
+        ms = e0.elapsed_time(e1) / args.steps
+        active = m.active_experts().tolist()
+        logical = algorithmic_bytes(model, info["kv_tokens_read"], active)
+        streamed = algorithmic_bytes(model, info["kv_tokens_streamed"], active)
+        out[label] = dict(ms_per_step=ms, tokens_per_s=B / (ms / 1e3), kv_tokens_read=info["kv_tokens_read"],
+                          kv_tokens_streamed=info["kv_tokens_streamed"], bytes_streamed=streamed["total"],
+                          frac_of_measured_hbm_streamed=streamed["total"] / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                          frac_of_measured_hbm_logical=logical["total"] / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                          launches=info["kernel_launches"], clocks=clocks)
+    line = dict(metric=METRIC, value=out["shared"]["tokens_per_s"], unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
+                ms_per_step=out["shared"]["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16", data="synthetic",
+                config=dict(workload=cfg["name"], groups=G, members=M, prompt_tokens=P, own_range=cfg["own_range"],
+                            l2="inputs larger than L2"),
+                clocks=out["shared"]["clocks"], gpu_launches=int(out["shared"]["launches"]) * args.steps,
+                shared_prefix_read_once=out["shared"], every_row_reads_its_context=out["per_row"],
+                speedup=out["per_row"]["ms_per_step"] / out["shared"]["ms_per_step"])
+    print(json.dumps(line))
+
+
 def run_cuda(args):
     rank, local_rank, world = dist_env()
     if world > 1:
@@ -442,7 +516,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", type=int, default=3, choices=[2, 3, 4, 5, 6])
+    ap.add_argument("--workload", type=int, default=3, choices=[2, 3, 4, 5, 6, 7, 8])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     args = ap.parse_args()
     if args.impl == "reference":
@@ -452,6 +526,8 @@ def main():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
         if args.workload in (4, 6):
             run_mixed(args)
+        elif args.workload in (7, 8):
+            run_grouped(args)
         else:
             run_cuda(args)
 

@@ -183,6 +183,17 @@ MARS_API mars_status_t mars_kv_seq_import(mars_kv_t *kv, int32_t seq, const void
 MARS_API mars_status_t mars_kv_seq_fork(mars_kv_t *kv, int32_t src, int32_t dst, void *cuda_stream);
 MARS_API int32_t mars_kv_page_refs(const mars_kv_t *kv, int32_t page);
 
+/* Reading a shared prefix once (on by default).  When several DECODE rows of one call list the same
+ * pages from position 0 on -- the members of a rollout group after mars_kv_seq_fork (Section 3.3:
+ * the outputs of a group continue one common input) -- the decode step reads the common whole pages
+ * once per block of 4 such rows instead of once per row: every K/V tile of the prefix is fetched
+ * into shared memory once and scored against the queries of all rows of the block, each row keeps
+ * its own online softmax, and the per-row partial results join the row's own spans in the usual
+ * log-sum-exp merge.  Results equal those of the per-row reading up to fp32 summation order.
+ * Prefixes shorter than 128 tokens, prompt rows, and the allocation-free entry point read per row.
+ * enable == 0 switches the grouping off (every row reads its whole context), e.g. to compare. */
+MARS_API mars_status_t mars_kv_share_reads(mars_kv_t *kv, int32_t enable);
+
 /* ---- the step ---------------------------------------------------------------------------------
  * mars_decode_step: for each listed sequence slot b (context length c_b), feed in_tokens[b] at
  * position c_b, append its key/value to the cache (a new page is taken from the free list when
@@ -294,6 +305,8 @@ typedef struct {
     int64_t kernel_launches;
     int64_t attn_items;
     int64_t kv_tokens_read; /* sum over token rows of (position + 1) */
+    int64_t kv_tokens_streamed; /* cached tokens actually fetched per layer and KV head: a shared prefix
+                                   counts once per block of rows, a prompt block once per block */
 } mars_step_info_t;
 MARS_API mars_status_t mars_last_step_info(const mars_model_t *model, mars_step_info_t *out);
 

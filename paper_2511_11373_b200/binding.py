@@ -57,7 +57,8 @@ class mars_debug_t(ctypes.Structure):
 
 
 class mars_step_info_t(ctypes.Structure):
-    _fields_ = [("kernel_launches", c_int64), ("attn_items", c_int64), ("kv_tokens_read", c_int64)]
+    _fields_ = [("kernel_launches", c_int64), ("attn_items", c_int64), ("kv_tokens_read", c_int64),
+                ("kv_tokens_streamed", c_int64)]
 
 
 # name -> (restype, argtypes); mirrors include/mars.h one to one
@@ -83,6 +84,7 @@ SIGNATURES = {
     "mars_kv_seq_import": (c_int32, [c_void_p, c_int32, c_void_p, c_size_t, c_int32, c_void_p]),
     "mars_kv_seq_fork": (c_int32, [c_void_p, c_int32, c_int32, c_void_p]),
     "mars_kv_page_refs": (c_int32, [c_void_p, c_int32]),
+    "mars_kv_share_reads": (c_int32, [c_void_p, c_int32]),
     "mars_decode_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), c_void_p,
                                    POINTER(mars_sampling_t), c_void_p, c_void_p, POINTER(mars_debug_t)]),
     "mars_prefill_chunk": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_int32), POINTER(c_int32), c_void_p,
@@ -200,7 +202,7 @@ class Model:
         info = mars_step_info_t()
         _check(lib().mars_last_step_info(self.handle, byref(info)), "mars_last_step_info")
         return dict(kernel_launches=info.kernel_launches, attn_items=info.attn_items,
-                    kv_tokens_read=info.kv_tokens_read)
+                    kv_tokens_read=info.kv_tokens_read, kv_tokens_streamed=info.kv_tokens_streamed)
 
     def profile_enable(self, on: bool = True):
         _check(lib().mars_profile_enable(self.handle, int(on)), "mars_profile_enable")
@@ -302,6 +304,9 @@ class KvCache:
 
     def page_refs(self, page: int) -> int:
         return lib().mars_kv_page_refs(self.handle, page)
+
+    def share_reads(self, enable: bool) -> None:
+        _check(lib().mars_kv_share_reads(self.handle, 1 if enable else 0), "mars_kv_share_reads")
 
     def close(self):
         if getattr(self, "handle", None):

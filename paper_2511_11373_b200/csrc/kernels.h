@@ -43,6 +43,11 @@ int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, co
 // Causal attention of a prefill chunk: items are blocks of up to 4 consecutive prompt tokens; writes b.o.
 int launch_attention_prefill(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv,
                              const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int sm_count, cudaStream_t st);
+// Spans of cached tokens that several decode rows share (same pages): read once per block of up to 4 rows;
+// every row gets its partial result in its own slot.
+int launch_attention_shared(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv,
+                            const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
+                            cudaStream_t st);
 int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st);
 
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,

@@ -114,7 +114,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
         const int item = u / p.nkv, hk = u - item * p.nkv;
         const int4 it = items[item];
-        const int row = it.x, start = it.y, len = it.z;
+        const int row = it.x, start = it.y, len = it.z, slot_out = it.w;
         const int seq = p.step[p.lay.tok_seq + row];
         const int n_st = (len + kStageTok - 1) / kStageTok;
         const int32_t* bt = p.block_table + (size_t)seq * p.max_pages_per_seq;
@@ -280,7 +280,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 L += ml[w * 8 + hh] * sc;
                 o += mo[(w * 8 + hh) * D + d] * sc;
             }
-            const size_t ph = (size_t)item * p.nq + hk * p.g + hh;
+            const size_t ph = (size_t)slot_out * p.nq + hk * p.g + hh;
             p.part_o[ph * D + d] = o;
             if (d == 0) p.part_ml[ph] = make_float2(M, L);
         }
@@ -291,13 +291,19 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 }
 
 // ---------------------------------------------------------------------------------------------
-// Causal attention of chunked prefill.  A work item is a block of up to kPfQueries consecutive
-// prompt tokens of one request (items: first token row, 0, keys visible to the LAST query of the
-// block, number of queries); a unit is (item, KV head).  The K/V tiles of positions 0 .. last are
-// streamed once per unit through the same TMA ring as in the decode kernel, and warp w owns query
-// w of the block: it scores all 64 tokens of every stage (four 16-token blocks), masks by its own
-// causal length, and keeps its own online softmax and output accumulator.  Nothing is split along
-// the keys, so the normalised output goes straight to b.o as (hi, lo) pairs.
+// Attention of a BLOCK of up to kPfQueries query rows that read the same cached tokens, so that every
+// K/V tile is fetched once for the block.  A unit is (item, KV head); the tiles stream through the
+// same TMA ring as in the decode kernel, and warp w owns query w of the block: it scores all 64
+// tokens of every stage (four 16-token blocks) and keeps its own online softmax and accumulator.
+//
+// SHARED == false: causal attention of chunked prefill.  An item is a run of consecutive prompt
+//   tokens of one request (items: first token row, 0, keys visible to the LAST query, number of
+//   queries); every warp masks by its own causal length.  Nothing is split along the keys, so the
+//   normalised output goes straight to b.o as (hi, lo) pairs.
+// SHARED == true: decode rows of DIFFERENT sequences whose block tables list the same pages for a
+//   span of cached tokens (members of a rollout group forked from one prompt).  An item is (first
+//   cached token, tokens, rows, 0, token row x 4, partial slot x 4); all rows see the whole span, and
+//   each writes (max, sum, unnormalised O) to its own partial slot for the span merge.
 constexpr int kPfQueries = 4;
 
 template <int D>
@@ -354,9 +360,9 @@ __device__ __forceinline__ void attend16(uint32_t kbase, uint32_t vbase, int w0,
     }
 }
 
-template <int D>
+template <int D, bool SHARED>
 __global__ void __launch_bounds__(kPfQueries * 32, 2)
-attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, AttnParams p,
+attn_block_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, AttnParams p,
                     __nv_bfloat16* o_out) {
     constexpr int TILE_BYTES = kStageTok * D * 2;
     constexpr int STAGE_BYTES = 2 * TILE_BYTES;
@@ -377,20 +383,29 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     }
     __syncthreads();
 
-    const int n_units = p.step[H_PF_ITEMS] * p.nkv;
+    const int n_units = p.step[SHARED ? H_SH_ITEMS : H_PF_ITEMS] * p.nkv;
     const int4* items = reinterpret_cast<const int4*>(p.step + p.lay.items) + p.step[H_PF_FIRST];
     const uint64_t pol = l2_evict_first_policy();
     uint32_t gs = 0;
 
     for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
         const int item = u / p.nkv, hk = u - item * p.nkv;
-        const int4 it = items[item];
-        const int row0 = it.x, len = it.z, nq_blk = it.w;          // len: keys visible to the last query
+        int row0, start, len, nq_blk, my_row, my_slot = 0;
+        if (SHARED) {
+            const int32_t* it = p.step + p.lay.sh_items + 12 * item;
+            start = it[0]; len = it[1]; nq_blk = it[2];
+            const int w = min(warp, nq_blk - 1);
+            row0 = it[4]; my_row = it[4 + w]; my_slot = it[8 + w];
+        } else {
+            const int4 it = items[item];
+            row0 = it.x; start = 0; len = it.z; nq_blk = it.w;    // len: keys visible to the last query
+            my_row = row0 + min(warp, nq_blk - 1);
+        }
         const int seq = p.step[p.lay.tok_seq + row0];
         const int n_st = (len + kStageTok - 1) / kStageTok;
         const int32_t* bt = p.block_table + (size_t)seq * p.max_pages_per_seq;
         const bool has_q = warp < nq_blk;
-        const int my_len = len - (nq_blk - 1 - warp);              // keys visible to this warp's query
+        const int my_len = SHARED ? len : len - (nq_blk - 1 - warp);   // keys visible to this warp's query
 
         auto issue = [&](int j, uint32_t g_stage) {
             const int slot = g_stage % kAttnStages;
@@ -400,7 +415,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             const int n_boxes = (n_valid + p.box_rows - 1) / p.box_rows;
             mbar_expect_tx(&full_bar[slot], (uint32_t)(n_boxes * p.box_rows * D * 2 * 2));
             for (int bi = 0; bi < n_boxes; ++bi) {
-                const int tok = j * kStageTok + bi * p.box_rows;
+                const int tok = start + j * kStageTok + bi * p.box_rows;
                 const int page = bt[tok / p.page_size];
                 const int y = (((p.layer * p.n_pages + page) * p.nkv + hk) * p.page_size) + tok % p.page_size;
 #pragma unroll
@@ -418,8 +433,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 
         uint32_t qa[KSTEPS][4];
         {
-            const int qrow_i = row0 + (has_q ? warp : 0);
-            const __nv_bfloat16* qhi = p.q + (size_t)qrow_i * 2 * p.nq * D + (size_t)(hk * p.g + gid) * D;
+            const __nv_bfloat16* qhi = p.q + (size_t)my_row * 2 * p.nq * D + (size_t)(hk * p.g + gid) * D;
             const __nv_bfloat16* qlo = qhi + (size_t)p.nq * D;
 #pragma unroll
             for (int ks = 0; ks < KSTEPS; ++ks) {
@@ -475,9 +489,19 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-        if (has_q && gid < p.g) {
+        if (SHARED) {
+            if (has_q && gid < p.g) {
+                const size_t ph = (size_t)my_slot * p.nq + hk * p.g + gid;
+                float* dst = p.part_o + ph * D;
+#pragma unroll
+                for (int c = 0; c < NTILES; ++c)
+                    *reinterpret_cast<float2*>(dst + c * 8 + 2 * tig) =
+                        make_float2(oacc[c][0] + oacc[c][2], oacc[c][1] + oacc[c][3]);      // hi rows + lo rows
+                if (tig == 0) p.part_ml[ph] = make_float2(m_run, l_run);
+            }
+        } else if (has_q && gid < p.g) {
             const float inv = 1.f / l_run;
-            __nv_bfloat16* dst = o_out + (size_t)(row0 + warp) * 2 * p.nq * D + (size_t)(hk * p.g + gid) * D;
+            __nv_bfloat16* dst = o_out + (size_t)my_row * 2 * p.nq * D + (size_t)(hk * p.g + gid) * D;
 #pragma unroll
             for (int c = 0; c < NTILES; ++c)
 #pragma unroll
@@ -556,8 +580,25 @@ int launch_attention_prefill(const Shape& s, const Buffers& b, const StepLayout&
     p.nkv = s.nkv; p.nq = s.nq; p.g = s.nq / s.nkv; p.layer = layer;
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
     const int grid = sm_count * 2;
-    if (s.D == 128) attn_prefill_kernel<128><<<grid, kPfQueries * 32, attn_smem_bytes<128>(), st>>>(tm_k, tm_v, p, b.o);
-    else attn_prefill_kernel<64><<<grid, kPfQueries * 32, attn_smem_bytes<64>(), st>>>(tm_k, tm_v, p, b.o);
+    if (s.D == 128) attn_block_kernel<128, false><<<grid, kPfQueries * 32, attn_smem_bytes<128>(), st>>>(tm_k, tm_v, p, b.o);
+    else attn_block_kernel<64, false><<<grid, kPfQueries * 32, attn_smem_bytes<64>(), st>>>(tm_k, tm_v, p, b.o);
+    return 1;
+}
+
+int launch_attention_shared(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv,
+                            const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
+                            cudaStream_t st) {
+    AttnParams p;
+    p.q = b.q; p.part_o = b.part_o; p.part_ml = b.part_ml; p.step = b.step; p.lay = lay;
+    p.block_table = kv.block_table; p.err = b.err;
+    p.max_pages_per_seq = kv.max_pages_per_seq; p.n_pages = kv.n_pages; p.page_size = kv.page_size;
+    p.box_rows = kv.page_size < kStageTok ? kv.page_size : kStageTok;
+    p.nkv = s.nkv; p.nq = s.nq; p.g = s.nq / s.nkv; p.layer = layer;
+    p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
+    int grid = n_items * s.nkv;
+    if (grid > sm_count * 2) grid = sm_count * 2;
+    if (s.D == 128) attn_block_kernel<128, true><<<grid, kPfQueries * 32, attn_smem_bytes<128>(), st>>>(tm_k, tm_v, p, nullptr);
+    else attn_block_kernel<64, true><<<grid, kPfQueries * 32, attn_smem_bytes<64>(), st>>>(tm_k, tm_v, p, nullptr);
     return 1;
 }
 
@@ -574,10 +615,16 @@ cudaError_t init_attn_kernels() {
     e = cudaFuncSetAttribute(attn_decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)attn_smem_bytes<64>());
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(attn_block_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)attn_smem_bytes<128>());
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attn_prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(attn_block_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes<64>());
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_block_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes<128>());
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attn_block_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)attn_smem_bytes<64>());
 }
 

@@ -37,6 +37,8 @@ namespace {
 constexpr int kSpanTokens = 1024;   // cached tokens per attention work item at decode
 constexpr int kStagingSlots = 4;
 constexpr int kUmmaMinTokens = 64;  // calls with more token rows take the tensor-core (tcgen05) contraction path
+constexpr int kSharedRows = 4;      // decode rows per work item of the shared-prefix attention kernel
+constexpr int kMinSharedTokens = 128;  // shorter common prefixes are read per row as usual
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -67,6 +69,7 @@ StepLayout make_layout(const Caps& k) {
     l.emit_slot = take(k.n_emit);
     l.updates = take(3 * k.n_updates);
     l.items = take(4 * k.n_items);
+    l.sh_items = take(12 * (k.n_items / 2 + 1));   // a shared item stands for the spans of at least two rows
     l.total_words = at;
     return l;
 }
@@ -207,6 +210,7 @@ struct mars_kv {
     std::vector<SeqState> seqs;
     std::vector<int32_t> free_list;   // stack of free page ids
     std::vector<int32_t> refs;        // number of sequence slots that list the page (0 = free)
+    bool share_reads = true;          // decode rows with a common page prefix read it once (mars_kv_share_reads)
 };
 
 extern "C" {
@@ -645,6 +649,12 @@ mars_status_t mars_kv_seq_fork(mars_kv_t* kv, int32_t src, int32_t dst, void* cu
     return rc;
 }
 
+mars_status_t mars_kv_share_reads(mars_kv_t* kv, int32_t enable) {
+    if (!kv) return MARS_ERR_BAD_HANDLE;
+    kv->share_reads = enable != 0;
+    return MARS_OK;
+}
+
 int32_t mars_kv_page_refs(const mars_kv_t* kv, int32_t page) {
     if (!kv || page < 0 || page >= kv->view.n_pages) return -1;
     return kv->refs[page];
@@ -671,11 +681,50 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     const int n_emit = (int)plan.emit_rows.size();
     const StepLayout& lay = m->lay;
 
+    // Decode rows whose sequences list the same pages from position 0 on (forked members of a rollout
+    // group): the common prefix, in whole pages strictly below every member's new position, is read
+    // once per block of kSharedRows rows by the shared-prefix kernel; the rest of each row as usual.
+    const int n_dec = plan.n_decode;
+    const int ps = kv->view.page_size;
+    struct SharedGroup { std::vector<int> rows; int tokens; };
+    std::vector<SharedGroup> shared;
+    std::vector<int> row_shared((size_t)n_dec, 0);   // tokens of the row that the shared kernel covers
+    if (kv->share_reads && n_dec > 1) {
+        std::vector<std::pair<int32_t, int>> first;   // (first page, index in `shared`), few entries
+        for (int t = 0; t < n_dec; ++t) {
+            const SeqState& q = kv->seqs[plan.tok_seq[t]];
+            if (q.pages.empty() || kv->refs[q.pages[0]] < 2) continue;
+            size_t gi = 0;
+            while (gi < first.size() && first[gi].first != q.pages[0]) ++gi;
+            if (gi == first.size()) {
+                first.emplace_back(q.pages[0], (int)shared.size());
+                shared.push_back(SharedGroup{{}, 0});
+            }
+            shared[first[gi].second].rows.push_back(t);
+        }
+        for (SharedGroup& g : shared) {
+            if (g.rows.size() < 2) continue;
+            const std::vector<int32_t>& p0 = kv->seqs[plan.tok_seq[g.rows[0]]].pages;
+            size_t common = p0.size();
+            int min_pos = plan.tok_pos[g.rows[0]];
+            for (size_t i = 1; i < g.rows.size(); ++i) {
+                const std::vector<int32_t>& pi = kv->seqs[plan.tok_seq[g.rows[i]]].pages;
+                size_t c = 0;
+                while (c < common && c < pi.size() && pi[c] == p0[c]) ++c;
+                common = c;
+                min_pos = std::min(min_pos, plan.tok_pos[g.rows[i]]);
+            }
+            const int tokens = (int)std::min<int64_t>((int64_t)common * ps, (int64_t)(min_pos / ps) * ps);
+            if (tokens < kMinSharedTokens) continue;
+            g.tokens = tokens;
+            for (int r : g.rows) row_shared[r] = tokens;
+        }
+    }
+
     // attention work items: spans of `span` cached tokens per token row (widened until they fit)
     int span = plan.span;
     int64_t n_items = 0;
     constexpr int kPrefillBlock = 4;   // consecutive prompt tokens per item of the causal prefill kernel
-    const int n_dec = plan.n_decode;
     int64_t pf_items = 0;
     for (int t = n_dec; t < n_tok;) {
         int e = t + 1;
@@ -684,15 +733,21 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         ++pf_items;
     }
     if (pf_items > m->caps.n_items) return MARS_ERR_INVALID_ARG;
-    int64_t dec_items = 0;
+    int64_t dec_items = 0, dec_slots = 0, sh_items = 0;
     for (;;) {
-        dec_items = 0;
-        for (int t = 0; t < n_dec; ++t) dec_items += ((int64_t)plan.tok_pos[t] + 1 + span - 1) / span;
-        if (dec_items + pf_items <= m->caps.n_items) break;
+        dec_items = dec_slots = sh_items = 0;
+        for (int t = 0; t < n_dec; ++t) {
+            const int64_t own = ((int64_t)plan.tok_pos[t] + 1 - row_shared[t] + span - 1) / span;
+            dec_items += own;
+            dec_slots += own + (row_shared[t] + span - 1) / span;
+        }
+        for (const SharedGroup& g : shared)
+            sh_items += (int64_t)((g.tokens + span - 1) / span) * (((int64_t)g.rows.size() + kSharedRows - 1) / kSharedRows);
+        if (dec_slots + pf_items <= m->caps.n_items && sh_items <= m->caps.n_items / 2 + 1) break;
         if (span > (1 << 28)) return MARS_ERR_INVALID_ARG;
         span *= 2;
     }
-    n_items = dec_items + pf_items;
+    n_items = dec_items + pf_items + sh_items;
 
     const int slot = m->next_slot;
     m->next_slot = (slot + 1) % kStagingSlots;
@@ -719,21 +774,47 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         std::memcpy(blk + lay.emit_slot, plan.emit_slot.data(), (size_t)n_emit * 4);
     }
     if (!plan.updates.empty()) std::memcpy(blk + lay.updates, plan.updates.data(), plan.updates.size() * 4);
-    int64_t kv_tokens = 0;
+    blk[H_SH_ITEMS] = (int32_t)sh_items;
+    int64_t kv_tokens = 0, kv_streamed = 0;
     {
         int32_t* items = blk + lay.items;
         int32_t* off = blk + lay.tok_item_off;
+        // partial slots of a decode row: its shared spans first, then its own spans
+        int slot_at = 0;
+        for (int t = 0; t < n_dec; ++t) {
+            off[t] = slot_at;
+            const int len = plan.tok_pos[t] + 1;
+            slot_at += (row_shared[t] + span - 1) / span + (len - row_shared[t] + span - 1) / span;
+        }
         int at = 0;
         for (int t = 0; t < n_dec; ++t) {
-            off[t] = at;
             const int len = plan.tok_pos[t] + 1;
             kv_tokens += len;
-            for (int s0 = 0; s0 < len; s0 += span) {
+            int slot_i = off[t] + (row_shared[t] + span - 1) / span;
+            for (int s0 = row_shared[t]; s0 < len; s0 += span) {
                 items[4 * at + 0] = t;
                 items[4 * at + 1] = s0;
                 items[4 * at + 2] = std::min(span, len - s0);
-                items[4 * at + 3] = 0;
+                items[4 * at + 3] = slot_i++;
+                kv_streamed += items[4 * at + 2];
                 ++at;
+            }
+        }
+        int32_t* sh = blk + lay.sh_items;
+        int sh_at = 0;
+        for (const SharedGroup& g : shared) {
+            for (int s0 = 0; s0 < g.tokens; s0 += span) {
+                for (size_t r0 = 0; r0 < g.rows.size(); r0 += kSharedRows) {
+                    const int nr = (int)std::min<size_t>(kSharedRows, g.rows.size() - r0);
+                    int32_t* it = sh + 12 * sh_at++;
+                    it[0] = s0; it[1] = std::min(span, g.tokens - s0); it[2] = nr; it[3] = 0;
+                    for (int i = 0; i < kSharedRows; ++i) {
+                        const int row = g.rows[r0 + (size_t)std::min(i, nr - 1)];
+                        it[4 + i] = row;
+                        it[8 + i] = off[row] + s0 / span;
+                    }
+                    kv_streamed += it[1];
+                }
             }
         }
         // blocks of consecutive tokens of one request: (first row, 0, keys visible to the last one, count)
@@ -744,15 +825,19 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             items[4 * at + 1] = 0;
             items[4 * at + 2] = plan.tok_pos[e - 1] + 1;
             items[4 * at + 3] = e - t;
-            for (int q = t; q < e; ++q) { off[q] = at; kv_tokens += plan.tok_pos[q] + 1; }
+            for (int q = t; q < e; ++q) { off[q] = slot_at; kv_tokens += plan.tok_pos[q] + 1; }
+            kv_streamed += plan.tok_pos[e - 1] + 1;
             ++at;
             t = e;
         }
-        off[n_tok] = at;
+        off[n_tok] = slot_at;
     }
     // one copy uploads the whole block up to the last item
-    const size_t used_words = (size_t)lay.items + 4 * (size_t)n_items;
+    const size_t used_words = (size_t)lay.items + 4 * (size_t)(dec_items + pf_items);
     CUDA_TRY(cudaMemcpyAsync(m->buf.step, blk, used_words * 4, cudaMemcpyHostToDevice, st));
+    if (sh_items)
+        CUDA_TRY(cudaMemcpyAsync(m->buf.step + lay.sh_items, blk + lay.sh_items, (size_t)sh_items * 12 * 4,
+                                 cudaMemcpyHostToDevice, st));
     CUDA_TRY(cudaEventRecord(m->staged[slot], st));
 
     const Shape& s = m->shape;
@@ -805,6 +890,10 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             });
         }
         if (n_dec > 0) {      // decode rows: spans of cached tokens, then the merge of each row's spans
+            if (sh_items)
+                run(MARS_K_ATTN, [&] {
+                    return launch_attention_shared(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, (int)sh_items, m->sm_count, st);
+                });
             run(MARS_K_ATTN, [&] { return launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st); });
             run(MARS_K_ATTN_MERGE, [&] { return launch_attn_merge(s, b, lay, n_dec, st); });
         }
@@ -869,6 +958,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     m->info.kernel_launches = launches;
     m->info.attn_items = n_items;
     m->info.kv_tokens_read = kv_tokens;
+    m->info.kv_tokens_streamed = kv_streamed;
     return MARS_OK;
 }
 
@@ -1219,6 +1309,7 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
             blk[lay.items + 4 * at + 0] = b;
             blk[lay.items + 4 * at + 1] = s0;
             blk[lay.items + 4 * at + 2] = std::min(kSpanTokens, len - s0);
+            blk[lay.items + 4 * at + 3] = at;      // partial slot = item index (nothing is shared here)
             ++at;
         }
     }

@@ -22,6 +22,7 @@ enum StepHdr {
     H_SEED_LO = 7, H_SEED_HI = 8, H_STEP_LO = 9, H_STEP_HI = 10,
     H_PF_FIRST = 11,  // first work item of the causal (prompt) attention kernel; decode spans come before it
     H_PF_ITEMS = 12,  // number of such items
+    H_SH_ITEMS = 13,  // work items of the shared-prefix kernel (a span of cached tokens read once for up to 4 rows)
     H_WORDS = 16
 };
 
@@ -29,11 +30,13 @@ enum StepHdr {
 struct StepLayout {
     int tok_seq;       // [n_tok] sequence slot (block-table row) of every token row
     int tok_pos;       // [n_tok] position of the token in its sequence
-    int tok_item_off;  // [n_tok + 1] first attention item of every token row
+    int tok_item_off;  // [n_tok + 1] first partial slot (span result) of every token row
     int emit_rows;     // [n_emit] token row whose hidden state is sampled
     int emit_slot;     // [n_emit] sequence slot of that row (random-number counter)
     int updates;       // [n_updates][3] (slot, page index, page id)
-    int items;         // [n_items][4] (token row, first cached token, number of tokens, 0)
+    int items;         // [n_items][4] decode spans: (token row, first cached token, number of tokens, partial slot);
+                       // prompt blocks after them: (first row, 0, keys visible to the last row, rows)
+    int sh_items;      // [n_sh][12] (first cached token, tokens, rows <= 4, 0, token row x 4, partial slot x 4)
     int total_words;
 };
 
@@ -55,8 +58,8 @@ struct Buffers {
     __nv_bfloat16* o;       // [n_tok, 2, nq D] attention output, (hi, lo) rows
     float2* rope;           // [n_tok, D/2] (cos, sin) of pos * theta_i
     double* inv_freq;       // [D/2] theta^(-2i/D)
-    float* part_o;          // [items, nq, D] unnormalised partial outputs
-    float2* part_ml;        // [items, nq] (running max in log2 units, sum)
+    float* part_o;          // [slots, nq, D] unnormalised partial outputs, one slot per (token row, span)
+    float2* part_ml;        // [slots, nq] (running max in log2 units, sum)
     float* rlogits;         // [n_tok, E] gate logits (prefill path: computed by one contraction for all rows)
     int32_t* route_idx;     // [n_tok, k]
     float* route_w;         // [n_tok, k]

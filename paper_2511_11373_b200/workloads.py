@@ -58,6 +58,13 @@ CONFIGS = {
             sampling=dict(greedy=0, temperature=1.0, top_p=0.95)),
     5: dict(name="qwen3-30b-a3b-48layer-decode-b16-64k", model=MODEL_FULL, page_size=64, batch=16,
             ctx=[65536] * 16, steps=64, sampling=dict(greedy=1, temperature=1.0, top_p=1.0)),
+    # grouped agentic rollouts: 8 groups of 8 responses, each group continuing one shared prompt
+    # (whole pages, held once in the cache); every member has its own response so far
+    7: dict(name="qwen3-30b-a3b-48layer-decode-8groups-of-8", model=MODEL_FULL, page_size=64, groups=8, members=8,
+            prompt=8192, own_range=(256, 4096), steps=32, sampling=dict(greedy=0, temperature=1.0, top_p=0.95)),
+    # one-layer stand-in of the same for quick checks
+    8: dict(name="qwen3-30b-a3b-1layer-decode-8groups-of-8", model=MODEL_LAYER, page_size=64, groups=8, members=8,
+            prompt=8192, own_range=(256, 4096), steps=8, sampling=dict(greedy=0, temperature=1.0, top_p=0.95)),
 }
 
 STAGES = ("solver", "verifier", "corrector")
@@ -132,6 +139,13 @@ def make_context_lengths(cfg: dict, seed: int = 0):
         c = int(round(spec["medians"][STAGES[t]] * math.exp(spec["sigma"] * zi)))
         ctx.append(max(lo, min(hi, c)))
     return ctx, [STAGES[t] for t in tags]
+
+
+def make_group_lengths(cfg: dict, seed: int = 0):
+    """Tokens of its own response that every member of every group has cached: [groups][members]."""
+    g = _gen("cpu", seed, cfg["name"] + ".own")
+    lo, hi = cfg["own_range"]
+    return torch.randint(lo, hi + 1, (cfg["groups"], cfg["members"]), generator=g).tolist()
 
 
 def pages_needed(n_tokens: int, page_size: int) -> int:
