@@ -73,6 +73,20 @@ __device__ __forceinline__ float block_sum(float v, float* scratch) {
     return t;
 }
 
+// Programmatic dependent launch.  Every kernel of the step is launched with the stream-serialisation
+// attribute relaxed (launch_chained in kernels.h): its blocks are scheduled as soon as all blocks of
+// the previous kernel of the stream have exited, without waiting for that grid's completion to be
+// signalled, and pdl_wait() returns once the previous kernel has completed and its writes are visible.
+// Rule kept by every kernel here: nothing produced by an earlier kernel is read, and no global memory
+// is written, before pdl_wait(); only weights (constant during a step), shared memory, barriers and
+// tensor memory are touched ahead of it.  Every kernel has at least one thread that executes
+// pdl_wait() before the grid can end, so completion of a kernel implies completion of all kernels
+// before it.  No kernel issues griddepcontrol.launch_dependents: measured on the 48-layer decode step
+// (22.04 ms with plain launches), letting the next grid's blocks become resident early cost time
+// (23.7 ms with the trigger at the top of every kernel, 21.6 ms with it in the small kernels only),
+// while the implicit trigger at block exit gives 21.2 ms.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {

@@ -26,6 +26,24 @@ struct DebugTaps {
     float* nucleus_mass;      // [n_emit] or null
 };
 
+// Launch with programmatic stream serialisation: the kernel's blocks may start while the previous kernel
+// of the stream drains (see pdl_wait in common.cuh for the rule the kernels keep).
+template <typename... Params, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
+}
+
 // Each wrapper enqueues its kernel(s) on `st` and returns the number of kernels it launched.
 int launch_prep(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, int n_tok, cudaStream_t st);
 int launch_embed(const Shape& s, const Buffers& b, const StepLayout& lay, const __nv_bfloat16* embed,
@@ -48,6 +66,7 @@ int launch_attention_prefill(const Shape& s, const Buffers& b, const StepLayout&
 int launch_attention_shared(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv,
                             const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
                             cudaStream_t st);
+
 int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st);
 
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,

@@ -104,6 +104,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    pdl_wait();
 
     const int32_t* hdr = p.step;
     const int n_units = hdr[H_NITEMS] * p.nkv;
@@ -111,38 +112,52 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     const uint64_t pol = l2_evict_first_policy();
     uint32_t gs = 0;  // stages consumed so far by this CTA (ring position and parity)
 
-    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-        const int item = u / p.nkv, hk = u - item * p.nkv;
+    // A unit's first ring stages are requested while the previous unit is still in its epilogue
+    // (warp merge, partial store, span merge), so the stream into the SM does not pause between units.
+    struct Unit { int row, start, len, slot_out, hk, n_st; const int32_t* bt; };
+    auto load_unit = [&](int u) {
+        Unit c;
+        const int item = u / p.nkv;
+        c.hk = u - item * p.nkv;
         const int4 it = items[item];
-        const int row = it.x, start = it.y, len = it.z, slot_out = it.w;
-        const int seq = p.step[p.lay.tok_seq + row];
-        const int n_st = (len + kStageTok - 1) / kStageTok;
-        const int32_t* bt = p.block_table + (size_t)seq * p.max_pages_per_seq;
-
-        auto issue = [&](int j, uint32_t g_stage) {
-            const int slot = g_stage % kAttnStages;
-            unsigned char* kdst = smem + (size_t)slot * STAGE_BYTES;
-            unsigned char* vdst = kdst + TILE_BYTES;
-            const int n_valid = min(kStageTok, len - j * kStageTok);
-            const int n_boxes = (n_valid + p.box_rows - 1) / p.box_rows;
-            mbar_expect_tx(&full_bar[slot], (uint32_t)(n_boxes * p.box_rows * D * 2 * 2));
-            for (int bi = 0; bi < n_boxes; ++bi) {
-                const int tok = start + j * kStageTok + bi * p.box_rows;
-                const int page = bt[tok / p.page_size];
-                const int y = (((p.layer * p.n_pages + page) * p.nkv + hk) * p.page_size) + tok % p.page_size;
+        c.row = it.x; c.start = it.y; c.len = it.z; c.slot_out = it.w;
+        c.n_st = (c.len + kStageTok - 1) / kStageTok;
+        c.bt = p.block_table + (size_t)p.step[p.lay.tok_seq + c.row] * p.max_pages_per_seq;
+        return c;
+    };
+    auto issue = [&](const Unit& c, int j, uint32_t g_stage) {
+        const int slot = g_stage % kAttnStages;
+        unsigned char* kdst = smem + (size_t)slot * STAGE_BYTES;
+        unsigned char* vdst = kdst + TILE_BYTES;
+        const int n_valid = min(kStageTok, c.len - j * kStageTok);
+        const int n_boxes = (n_valid + p.box_rows - 1) / p.box_rows;
+        mbar_expect_tx(&full_bar[slot], (uint32_t)(n_boxes * p.box_rows * D * 2 * 2));
+        for (int bi = 0; bi < n_boxes; ++bi) {
+            const int tok = c.start + j * kStageTok + bi * p.box_rows;
+            const int page = c.bt[tok / p.page_size];
+            const int y = (((p.layer * p.n_pages + page) * p.nkv + c.hk) * p.page_size) + tok % p.page_size;
 #pragma unroll
-                for (int hf = 0; hf < HALVES; ++hf) {
-                    const int off = hf * (kStageTok * 128) + bi * p.box_rows * 128;
-                    tma_load_2d(kdst + off, &tm_k, hf * 64, y, &full_bar[slot], pol);
-                    tma_load_2d(vdst + off, &tm_v, hf * 64, y, &full_bar[slot], pol);
-                }
+            for (int hf = 0; hf < HALVES; ++hf) {
+                const int off = hf * (kStageTok * 128) + bi * p.box_rows * 128;
+                tma_load_2d(kdst + off, &tm_k, hf * 64, y, &full_bar[slot], pol);
+                tma_load_2d(vdst + off, &tm_v, hf * 64, y, &full_bar[slot], pol);
             }
-        };
-
-        if (tid == 0 && !dead) {
-            const int pre = min(kAttnStages - 1, n_st);
-            for (int j = 0; j < pre; ++j) issue(j, gs + j);
         }
+    };
+    auto prefetch = [&](const Unit& c, uint32_t g0) {
+        const int pre = min(kAttnStages - 1, c.n_st);
+        for (int j = 0; j < pre; ++j) issue(c, j, g0 + j);
+    };
+
+    int u = blockIdx.x;
+    bool have = u < n_units;
+    Unit cur;
+    if (have) {
+        cur = load_unit(u);
+        if (tid == 0) prefetch(cur, gs);
+    }
+    while (have) {
+        const int row = cur.row, len = cur.len, slot_out = cur.slot_out, hk = cur.hk, n_st = cur.n_st;
 
         // Query fragments.  The group has at most 8 heads, so MMA rows 0..7 carry the hi part of head
         // gid and rows 8..15 its lo part: S = d0 + d2 (d1 + d3) costs no extra tensor work.
@@ -168,7 +183,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         float m_run = -INFINITY, l_run = 0.f;
 
         for (int j = 0; j < n_st; ++j) {
-            if (tid == 0 && !dead && j + kAttnStages - 1 < n_st) issue(j + kAttnStages - 1, gs + j + kAttnStages - 1);
+            if (tid == 0 && !dead && j + kAttnStages - 1 < n_st) issue(cur, j + kAttnStages - 1, gs + j + kAttnStages - 1);
             const uint32_t g_stage = gs + j;
             const int slot = g_stage % kAttnStages;
             // Every lane polls; the outcome is made warp-uniform before any .sync instruction.
@@ -255,10 +270,21 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         }
         gs += n_st;
 
-        // merge the four warps (stage memory is idle: every issued tile has been consumed)
+        // the next unit's first stages go into ring slots gs, gs + 1; the slot after them stays free
+        // until that unit's main loop, and serves as scratch for the epilogue below
+        const int un = u + gridDim.x;
+        const bool have_next = un < n_units;
+        Unit nxt = cur;
+        if (have_next) {
+            nxt = load_unit(un);
+            if (tid == 0 && !dead) prefetch(nxt, gs);
+        }
+        unsigned char* scratch = smem + (size_t)((gs + kAttnStages - 1) % kAttnStages) * STAGE_BYTES;
+
+        // merge the four warps
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-        float* mo = reinterpret_cast<float*>(smem);                 // [warps][8][D]
+        float* mo = reinterpret_cast<float*>(scratch);              // [warps][8][D]
         float* mm = mo + kAttnWarps * 8 * D;                        // [warps][8]
         float* ml = mm + kAttnWarps * 8;                            // [warps][8]
 #pragma unroll
@@ -287,6 +313,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         // the generic-proxy writes above must be ordered before the next TMA write to this memory
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncthreads();
+        cur = nxt; u = un; have = have_next;
     }
 }
 
@@ -382,6 +409,7 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    pdl_wait();
 
     const int n_units = p.step[SHARED ? H_SH_ITEMS : H_PF_ITEMS] * p.nkv;
     const int4* items = reinterpret_cast<const int4*>(p.step + p.lay.items) + p.step[H_PF_FIRST];
@@ -519,6 +547,7 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 template <int D>
 __global__ void __launch_bounds__(D) attn_combine_kernel(Buffers b, StepLayout lay, int nq) {
     __shared__ float2 sml[D];
+    pdl_wait();
     const int t = blockIdx.x, j = blockIdx.y, d = threadIdx.x;
     const int i0 = b.step[lay.tok_item_off + t], i1 = b.step[lay.tok_item_off + t + 1];
     float den = 0.f, o = 0.f;
@@ -565,8 +594,8 @@ int launch_attention(const Shape& s, const Buffers& b, const StepLayout& lay, co
     p.nkv = s.nkv; p.nq = s.nq; p.g = s.nq / s.nkv; p.layer = layer;
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
     const int grid = sm_count * 2;
-    if (s.D == 128) attn_decode_kernel<128><<<grid, kAttnWarps * 32, attn_smem_bytes<128>(), st>>>(tm_k, tm_v, p);
-    else attn_decode_kernel<64><<<grid, kAttnWarps * 32, attn_smem_bytes<64>(), st>>>(tm_k, tm_v, p);
+    if (s.D == 128) launch_chained(attn_decode_kernel<128>, dim3(grid), dim3(kAttnWarps * 32), attn_smem_bytes<128>(), st, tm_k, tm_v, p);
+    else launch_chained(attn_decode_kernel<64>, dim3(grid), dim3(kAttnWarps * 32), attn_smem_bytes<64>(), st, tm_k, tm_v, p);
     return 1;
 }
 
@@ -580,8 +609,8 @@ int launch_attention_prefill(const Shape& s, const Buffers& b, const StepLayout&
     p.nkv = s.nkv; p.nq = s.nq; p.g = s.nq / s.nkv; p.layer = layer;
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
     const int grid = sm_count * 2;
-    if (s.D == 128) attn_block_kernel<128, false><<<grid, kPfQueries * 32, attn_smem_bytes<128>(), st>>>(tm_k, tm_v, p, b.o);
-    else attn_block_kernel<64, false><<<grid, kPfQueries * 32, attn_smem_bytes<64>(), st>>>(tm_k, tm_v, p, b.o);
+    if (s.D == 128) launch_chained(attn_block_kernel<128, false>, dim3(grid), dim3(kPfQueries * 32), attn_smem_bytes<128>(), st, tm_k, tm_v, p, b.o);
+    else launch_chained(attn_block_kernel<64, false>, dim3(grid), dim3(kPfQueries * 32), attn_smem_bytes<64>(), st, tm_k, tm_v, p, b.o);
     return 1;
 }
 
@@ -597,14 +626,14 @@ int launch_attention_shared(const Shape& s, const Buffers& b, const StepLayout& 
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
     int grid = n_items * s.nkv;
     if (grid > sm_count * 2) grid = sm_count * 2;
-    if (s.D == 128) attn_block_kernel<128, true><<<grid, kPfQueries * 32, attn_smem_bytes<128>(), st>>>(tm_k, tm_v, p, nullptr);
-    else attn_block_kernel<64, true><<<grid, kPfQueries * 32, attn_smem_bytes<64>(), st>>>(tm_k, tm_v, p, nullptr);
+    if (s.D == 128) launch_chained(attn_block_kernel<128, true>, dim3(grid), dim3(kPfQueries * 32), attn_smem_bytes<128>(), st, tm_k, tm_v, p, nullptr);
+    else launch_chained(attn_block_kernel<64, true>, dim3(grid), dim3(kPfQueries * 32), attn_smem_bytes<64>(), st, tm_k, tm_v, p, nullptr);
     return 1;
 }
 
 int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st) {
-    if (s.D == 128) attn_combine_kernel<128><<<dim3(n_tok, s.nq), 128, 0, st>>>(b, lay, s.nq);
-    else attn_combine_kernel<64><<<dim3(n_tok, s.nq), 64, 0, st>>>(b, lay, s.nq);
+    if (s.D == 128) launch_chained(attn_combine_kernel<128>, dim3(n_tok, s.nq), dim3(128), 0, st, b, lay, s.nq);
+    else launch_chained(attn_combine_kernel<64>, dim3(n_tok, s.nq), dim3(64), 0, st, b, lay, s.nq);
     return 1;
 }
 

@@ -10,6 +10,7 @@ namespace mars {
 // (cos, sin)(pos * theta_i) for every token row (fp64 angles: pos reaches 64k and beyond, where an
 // fp32 product pos * theta_0 is already off by milliradians).
 __global__ void prep_kernel(Buffers b, StepLayout lay, KvView kv, int half_d) {
+    pdl_wait();
     const int32_t* hdr = b.step;
     const int n_tok = hdr[H_NTOK];
     if (blockIdx.x == 0) {
@@ -32,7 +33,7 @@ int launch_prep(const Shape& s, const Buffers& b, const StepLayout& lay, const K
     int grid = (total + 255) / 256;
     if (grid < 1) grid = 1;
     if (grid > 1024) grid = 1024;
-    prep_kernel<<<grid, 256, 0, st>>>(b, lay, kv, s.D / 2);
+    launch_chained(prep_kernel, dim3(grid), dim3(256), 0, st, b, lay, kv, s.D / 2);
     return 1;
 }
 
@@ -66,6 +67,7 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(Shape s, Buffers b, 
                                                             const int32_t* tokens, const __nv_bfloat16* gain,
                                                             float* hidden_tap) {
     __shared__ float scratch[32];
+    pdl_wait();
     const int t = blockIdx.x;
     int tok = tokens[t];
     if (tok < 0 || tok >= s.V) {
@@ -91,7 +93,7 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(Shape s, Buffers b, 
 
 int launch_embed(const Shape& s, const Buffers& b, const StepLayout&, const __nv_bfloat16* embed, const int32_t* tokens,
                  const __nv_bfloat16* first_gain, float* hidden_tap, int n_tok, cudaStream_t st) {
-    embed_kernel<<<n_tok, kRowThreads, 0, st>>>(s, b, embed, tokens, first_gain, hidden_tap);
+    launch_chained(embed_kernel, dim3(n_tok), dim3(kRowThreads), 0, st, s, b, embed, tokens, first_gain, hidden_tap);
     return 1;
 }
 
@@ -150,6 +152,8 @@ __global__ void __launch_bounds__(kGemmMaxWarps * 32, 1) stream_gemm_kernel(Gemm
 #pragma unroll
     for (int n = 0; n < kGemmNT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
 
+    // the weight ring above reads constants only; the activations come from the previous kernel
+    pdl_wait();
     const int pieces = p.ks / 8;   // 16-byte pieces per activation row
     for (int ph = 0; ph < p.phases; ++ph) {
         if (ph > 0) __syncthreads();             // every warp is done with the previous phase's activations
@@ -212,7 +216,7 @@ static int launch_gemm(GemmParams p, bool many_rows, int sm_count, cudaStream_t 
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_w = w; }
     }
     dim3 grid((p.rows + best_w * 16 - 1) / (best_w * 16), ksplit, tok_tiles);
-    stream_gemm_kernel<<<grid, best_w * 32, gemm_smem_bytes(p.ks, best_w), st>>>(p);
+    launch_chained(stream_gemm_kernel, dim3(grid), dim3(best_w * 32), gemm_smem_bytes(p.ks, best_w), st, p);
     return 1;
 }
 
@@ -225,6 +229,7 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepL
                                                        const __nv_bfloat16* q_gain, const __nv_bfloat16* k_gain,
                                                        int layer, int ksplit, int n_tok) {
     constexpr int HALF = D / 2, PER = HALF / 32;
+    pdl_wait();
     const int t = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_heads = s.nq + 2 * s.nkv;
     const int pos = b.step[lay.tok_pos + t], seq = b.step[lay.tok_seq + t];
@@ -298,9 +303,9 @@ int launch_qkv_post(const Shape& s, const Buffers& b, const StepLayout& lay, con
                     int n_tok, int ksplit, cudaStream_t st) {
     const dim3 grid(n_tok, (s.nq + 2 * s.nkv + 3) / 4);
     if (s.D == 128)
-        qkv_post_kernel<128><<<grid, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
+        launch_chained(qkv_post_kernel<128>, dim3(grid), dim3(128), 0, st, s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
     else
-        qkv_post_kernel<64><<<grid, 128, 0, st>>>(s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
+        launch_chained(qkv_post_kernel<64>, dim3(grid), dim3(128), 0, st, s, b, lay, kv, w.q_norm, w.k_norm, layer, ksplit, n_tok);
     return 1;
 }
 

@@ -79,6 +79,7 @@ __global__ void __launch_bounds__(kRouterCta) router_kernel(Shape s, Buffers b, 
     __shared__ float scratch[32];
     __shared__ float z[kMaxExperts];
     __shared__ float zp[kMaxExperts];     // partial logits of the K quarters: [quarter][expert]
+    pdl_wait();
     const int t = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tig = lane & 3;
     const int H = s.H, E = s.E, k = s.k;
     const int xrow = x_row_bytes(H);
@@ -168,6 +169,7 @@ __global__ void __launch_bounds__(kRouterCta) router_kernel(Shape s, Buffers b, 
 __global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int layer, int n_pairs, int tok_cap) {
     __shared__ int cnt[kMaxExperts];
     __shared__ int off[kMaxExperts + 1];
+    pdl_wait();
     const int tid = threadIdx.x, E = s.E;
     for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
     __syncthreads();
@@ -260,6 +262,7 @@ __device__ __forceinline__ void gate_up_epilogue(const float (&acc)[NT][4], int 
 __global__ void __launch_bounds__(kGuMaxWarps * 32, 1) expert_gate_up_kernel(Shape s, Buffers b, const __nv_bfloat16* Wgu,
                                                                           int tok_cap) {
     extern __shared__ __align__(128) unsigned char smem[];
+    pdl_wait();      // the group list comes from the permute kernel
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tig = lane & 3;
     const int H = s.H, I = s.I;
     const int n_warps = blockDim.x >> 5;
@@ -393,6 +396,7 @@ __device__ __forceinline__ void down_tile(const __nv_bfloat16* Wd, int H, int I,
 __global__ void __launch_bounds__(kExpMaxWarps * 32) expert_down_kernel(Shape s, Buffers b, const __nv_bfloat16* Wdn,
                                                                      int tok_cap) {
     extern __shared__ __align__(128) unsigned char smem[];
+    pdl_wait();
     const int e = blockIdx.y;
     const int o0 = b.expert_off[e], m = b.expert_off[e + 1] - o0;
     if (m == 0) return;
@@ -434,6 +438,7 @@ __global__ void __launch_bounds__(kRouterThreads) combine_kernel(Shape s, Buffer
     __shared__ float scratch[32];
     __shared__ int slots[kMaxTopK];
     __shared__ float ws[kMaxTopK];
+    pdl_wait();
     const int t = blockIdx.x, tid = threadIdx.x, H = s.H, k = s.k;
     if (tid < k) { slots[tid] = b.slot_of[(size_t)t * k + tid]; ws[tid] = b.route_w[(size_t)t * k + tid]; }
     __syncthreads();
@@ -487,6 +492,7 @@ __global__ void __launch_bounds__(kRouterThreads) combine_kernel(Shape s, Buffer
 __global__ void __launch_bounds__(kRouterThreads) resid_norm_kernel(Shape s, Buffers b, const __nv_bfloat16* gain, int n_tok,
                                                                    int o_ksplit) {
     __shared__ float scratch[32];
+    pdl_wait();
     const int t = blockIdx.x, tid = threadIdx.x, H = s.H;
     float v[kRowMaxPer];
     const float* __restrict__ xin = b.x + (size_t)t * H;
@@ -521,6 +527,7 @@ __global__ void __launch_bounds__(kRouterThreads) resid_norm_kernel(Shape s, Buf
 // One warp per token row: logits [n_tok][E] (fp32, from the contraction) -> routing.
 __global__ void __launch_bounds__(128) route_select_kernel(Shape s, Buffers b, DebugTaps dbg, int layer, int n_tok) {
     extern __shared__ float zs[];     // [4][E]
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * 4 + warp;
     if (t >= n_tok) return;
@@ -531,14 +538,14 @@ __global__ void __launch_bounds__(128) route_select_kernel(Shape s, Buffers b, D
 }
 
 int launch_resid_norm(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int o_ksplit, cudaStream_t st) {
-    resid_norm_kernel<<<n_tok, kRouterThreads, 0, st>>>(s, b, w.mlp_norm, n_tok, o_ksplit);
+    launch_chained(resid_norm_kernel, dim3(n_tok), dim3(kRouterThreads), 0, st, s, b, w.mlp_norm, n_tok, o_ksplit);
     return 1;
 }
 
 int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int group_cap,
                         cudaStream_t st) {
-    route_select_kernel<<<(n_tok + 3) / 4, 128, 4 * s.E * sizeof(float), st>>>(s, b, dbg, layer, n_tok);
-    permute_kernel<<<1, 1024, 0, st>>>(s, b, layer, n_tok * s.k, group_cap);
+    launch_chained(route_select_kernel, dim3((n_tok + 3) / 4), dim3(128), 4 * s.E * sizeof(float), st, s, b, dbg, layer, n_tok);
+    launch_chained(permute_kernel, dim3(1), dim3(1024), 0, st, s, b, layer, n_tok * s.k, group_cap);
     return 2;
 }
 
@@ -559,12 +566,12 @@ int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const Debug
                   int group_cap, cudaStream_t st) {
     int ks, o_ksplit, phases;
     gemm_plan(s.nq * s.D, n_tok, false, &ks, &o_ksplit, &phases);
-    router_kernel<<<n_tok, kRouterCta, 8 * x_row_bytes(s.H), st>>>(s, b, w.mlp_norm, w.router, dbg, layer, n_tok,
+    launch_chained(router_kernel, dim3(n_tok), dim3(kRouterCta), 8 * x_row_bytes(s.H), st, s, b, w.mlp_norm, w.router, dbg, layer, n_tok,
                                                                        o_ksplit);
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
     if (group_cap > 0) cap = group_cap;          // the tensor-core expert path wants one 128-row tile per group
-    permute_kernel<<<1, 1024, 0, st>>>(s, b, layer, n_tok * s.k, cap);
+    launch_chained(permute_kernel, dim3(1), dim3(1024), 0, st, s, b, layer, n_tok * s.k, cap);
     return 2;
 }
 
@@ -572,7 +579,7 @@ int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok,
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
     const size_t smem = (size_t)cap * 2 * x_row_bytes(s.H) + (size_t)warps * kRingWarpBytes;
-    expert_gate_up_kernel<<<sm_count, warps * 32, smem, st>>>(s, b, w.w_gate_up, cap);
+    launch_chained(expert_gate_up_kernel, dim3(sm_count), dim3(warps * 32), smem, st, s, b, w.w_gate_up, cap);
     return 1;
 }
 
@@ -581,13 +588,13 @@ int launch_down(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cu
     expert_plan(s, n_tok, &cap, &warps);
     const int w2 = cap > 8 ? 8 : 4;
     dim3 g2((s.H / 32 + w2 - 1) / w2, s.E);
-    expert_down_kernel<<<g2, w2 * 32, (size_t)cap * 2 * x_row_bytes(s.I), st>>>(s, b, w.w_down, cap);
+    launch_chained(expert_down_kernel, dim3(g2), dim3(w2 * 32), (size_t)cap * 2 * x_row_bytes(s.I), st, s, b, w.w_down, cap);
     return 1;
 }
 
 int launch_combine(const Shape& s, const Buffers& b, const __nv_bfloat16* next_gain, float* hidden_tap, int n_tok,
                    cudaStream_t st) {
-    combine_kernel<<<n_tok, kRouterThreads, 0, st>>>(s, b, next_gain, hidden_tap);
+    launch_chained(combine_kernel, dim3(n_tok), dim3(kRouterThreads), 0, st, s, b, next_gain, hidden_tap);
     return 1;
 }
 

@@ -66,6 +66,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(Shape s, Buffers
     __shared__ unsigned int sel_prefix;
     __shared__ unsigned long long sel_above;
     __shared__ int sel_token;
+    pdl_wait();
 
     const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int V = s.V;
@@ -232,7 +233,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(Shape s, Buffers
 
 int launch_sample(const Shape& s, const Buffers& b, const StepLayout& lay, int n_emit, int32_t* out_tokens,
                   float* out_logprobs, float* nucleus_mass, cudaStream_t st) {
-    sample_kernel<<<n_emit, kSampleThreads, 0, st>>>(s, b, lay, out_tokens, out_logprobs, nucleus_mass);
+    launch_chained(sample_kernel, dim3(n_emit), dim3(kSampleThreads), 0, st, s, b, lay, out_tokens, out_logprobs, nucleus_mass);
     return 1;
 }
 

@@ -135,6 +135,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int dead;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_wait();      // the group list and the activations come from earlier kernels
 
     // which rows of A and B this tile contracts
     int m0, m_valid, b_row0, b_row1, col0;     // b_row0 / b_row1: first weight row of each 128-column half
@@ -346,9 +347,26 @@ umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int ks = 0; ks < nk && !dead; ++ks) {
+            // The weights are constants of the step: the first ring-full of weight tiles is requested
+            // before the previous kernel has finished; the activations it produces only after pdl_wait().
+            const int pre = nk < kSwStages ? nk : kSwStages;
+            for (int ks = 0; ks < pre; ++ks) {
+                unsigned char* st = smem + (size_t)ks * kSwStageBytes;
+                const int k = k0 + ks * kUmStageK;
+                um_expect_tx(&full_bar[ks], kSwStageBytes);
+                um_tma_2d(st, &tm_w, k, row0, &full_bar[ks]);
+                um_tma_2d(st + 8192, &tm_w, k, row0 + 64, &full_bar[ks]);
+            }
+            pdl_wait();
+            for (int ks = 0; ks < pre; ++ks) {
+                unsigned char* st = smem + (size_t)ks * kSwStageBytes;
+                const int k = k0 + ks * kUmStageK;
+                um_tma_3d(st + kSwABytes, &tm_x, k, 0, 0, &full_bar[ks]);
+                um_tma_3d(st + kSwABytes + kSwBBytes, &tm_x, k, 1, 0, &full_bar[ks]);
+            }
+            for (int ks = pre; ks < nk && !dead; ++ks) {
                 const int s = ks % kSwStages;
-                if (ks >= kSwStages && !um_wait(&empty_bar[s], ((ks / kSwStages) - 1) & 1)) {
+                if (!um_wait(&empty_bar[s], ((ks / kSwStages) - 1) & 1)) {
                     dead = 1; atomicOr(p.err, kErrTimeout); break;
                 }
                 unsigned char* st = smem + (size_t)s * kSwStageBytes;
@@ -414,13 +432,14 @@ static size_t swap_smem_bytes() { return (size_t)kSwStages * kSwStageBytes + 102
 int launch_umma_swap(const CUtensorMap& tm_w, const CUtensorMap& tm_x, int rows, int n_tok, int K, int splits, float* out,
                      int32_t* err, cudaStream_t st) {
     SwapParams p{rows, n_tok, K / splits, out, err};
-    umma_swap_kernel<<<dim3((rows + 127) / 128, splits), kUmThreads, swap_smem_bytes(), st>>>(tm_w, tm_x, p);
+    launch_chained(umma_swap_kernel, dim3((rows + 127) / 128, splits), dim3(kUmThreads), swap_smem_bytes(), st, tm_w, tm_x, p);
     return 1;
 }
 
 // Rows of the normalised activations gathered into expert-slot order: xperm[slot] = h[slot_token[slot]]
 // (both planes), so that a group's rows are one contiguous TMA box.
 __global__ void __launch_bounds__(256) gather_rows_kernel(Buffers b, int H, int n_slots) {
+    pdl_wait();
     const int slot = blockIdx.x;
     if (slot >= n_slots) return;
     const uint4* src = reinterpret_cast<const uint4*>(b.h + (size_t)b.slot_token[slot] * 2 * H);
@@ -434,7 +453,7 @@ int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_ro
                       int32_t* err, cudaStream_t st) {
     UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err, nullptr, 0.f, nullptr, nullptr};
     dim3 grid((n_cols + kUmTileN - 1) / kUmTileN, (m_rows + kUmTileM - 1) / kUmTileM);
-    umma_gemm_kernel<<<grid, kUmThreads, umma_smem_bytes(), st>>>(tm_a, tm_b, p);
+    launch_chained(umma_gemm_kernel, dim3(grid), dim3(kUmThreads), umma_smem_bytes(), st, tm_a, tm_b, p);
     return 1;
 }
 
@@ -442,11 +461,11 @@ int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_
                         const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, cudaStream_t st) {
     const int n_slots = n_tok * s.k;
     const int max_groups = s.E + (n_slots + kUmTileM - 1) / kUmTileM;
-    gather_rows_kernel<<<n_slots, 256, 0, st>>>(b, s.H, n_slots);
+    launch_chained(gather_rows_kernel, dim3(n_slots), dim3(256), 0, st, b, s.H, n_slots);
     UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err, nullptr, 0.f, nullptr, nullptr};
-    umma_gemm_kernel<<<dim3((s.I + 127) / 128, max_groups), kUmThreads, umma_smem_bytes(), st>>>(tm_xperm, tm_wgu, gu);
+    launch_chained(umma_gemm_kernel, dim3((s.I + 127) / 128, max_groups), dim3(kUmThreads), umma_smem_bytes(), st, tm_xperm, tm_wgu, gu);
     UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err, nullptr, 0.f, nullptr, nullptr};
-    umma_gemm_kernel<<<dim3((s.H + kUmTileN - 1) / kUmTileN, max_groups), kUmThreads, umma_smem_bytes(), st>>>(
+    launch_chained(umma_gemm_kernel, dim3((s.H + kUmTileN - 1) / kUmTileN, max_groups), dim3(kUmThreads), umma_smem_bytes(), st, 
         tm_act, tm_wdown, dn);
     return 3;
 }
@@ -458,6 +477,7 @@ int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_
 __global__ void __launch_bounds__(256) score_combine_kernel(const float2* __restrict__ ml, const float* __restrict__ zt,
                                                             const int32_t* __restrict__ targets, int n_rows, int n_tiles,
                                                             int vocab, float* __restrict__ out, int32_t* err) {
+    pdl_wait();
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (row >= n_rows) return;
     const int tgt = targets[row];
@@ -486,8 +506,8 @@ int launch_umma_score(const CUtensorMap& tm_h, const CUtensorMap& tm_lm, int n_r
     UmmaParams p{K, n_rows, nullptr, nullptr, 0, vocab, 2, logits_tap, nullptr, err, targets, inv_temp, score_ml, score_tgt};
     const int n_tiles = (vocab + kUmTileN - 1) / kUmTileN;
     dim3 grid(n_tiles, (n_rows + kUmTileM - 1) / kUmTileM);
-    umma_gemm_kernel<<<grid, kUmThreads, umma_smem_bytes(), st>>>(tm_h, tm_lm, p);
-    score_combine_kernel<<<(n_rows + 7) / 8, 256, 0, st>>>(score_ml, score_tgt, targets, n_rows, n_tiles, vocab,
+    launch_chained(umma_gemm_kernel, dim3(grid), dim3(kUmThreads), umma_smem_bytes(), st, tm_h, tm_lm, p);
+    launch_chained(score_combine_kernel, dim3((n_rows + 7) / 8), dim3(256), 0, st, score_ml, score_tgt, targets, n_rows, n_tiles, vocab,
                                                             out_logprobs, err);
     return 2;
 }
