@@ -259,6 +259,51 @@ __device__ __forceinline__ void gate_up_epilogue(const float (&acc)[NT][4], int 
     }
 }
 
+// cp.async.wait_group wants an immediate; after unrolling `pending` is a constant.
+__device__ __forceinline__ void cp_async_wait_n(int pending) {
+    switch (pending) {
+        case 0: cp_async_wait<0>(); break;
+        case 1: cp_async_wait<1>(); break;
+        case 2: cp_async_wait<2>(); break;
+        case 3: cp_async_wait<3>(); break;
+        case 4: cp_async_wait<4>(); break;
+        case 5: cp_async_wait<5>(); break;
+        case 6: cp_async_wait<6>(); break;
+        case 7: cp_async_wait<7>(); break;
+        case 8: cp_async_wait<8>(); break;
+        case 9: cp_async_wait<9>(); break;
+        case 10: cp_async_wait<10>(); break;
+        case 11: cp_async_wait<11>(); break;
+        case 12: cp_async_wait<12>(); break;
+        case 13: cp_async_wait<13>(); break;
+        case 14: cp_async_wait<14>(); break;
+        default: cp_async_wait<15>(); break;
+    }
+}
+
+// One unit's K loop: kGuBatch slices are consumed, then kGuBatch slices are requested back to back, so
+// that every weight row is asked for in runs of kGuBatch x 64 contiguous bytes (measured per launch on
+// the 48-layer decode step: one slice at a time 156 us, two 153 us, four 142-145 us, eight 145 us; a
+// deeper ring with fewer warps was slower).  n_slices = H / 32 is a multiple of 8.
+constexpr int kGuBatch = 4;
+constexpr int kGuRing = kRing;                                // slices in flight per warp
+constexpr int kGuRingWarpBytes = kGuRing * kRingStageBytes;
+static_assert(kGuBatch <= kGuRing && 8 % kGuBatch == 0, "the batch must divide the slice count");
+template <int NT, typename Issue>
+__device__ __forceinline__ void gu_stream(const unsigned char* ring, int& ccount, int lane, const unsigned char* xs, int xrow,
+                                          int n_slices, float (&acc)[NT][4], Issue& issue_next) {
+    for (int sl = 0; sl < n_slices; sl += kGuBatch) {
+#pragma unroll
+        for (int b = 0; b < kGuBatch; ++b) {
+            cp_async_wait_n(kGuRing - 1 - b);
+            ring_consume<NT>(ring, ccount % kGuRing, lane, xs + (size_t)(sl + b) * 64, 8 * xrow, acc);
+            ++ccount;
+        }
+#pragma unroll
+        for (int b = 0; b < kGuBatch; ++b) issue_next();
+    }
+}
+
 __global__ void __launch_bounds__(kGuMaxWarps * 32, 1) expert_gate_up_kernel(Shape s, Buffers b, const __nv_bfloat16* Wgu,
                                                                           int tok_cap) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -268,7 +313,7 @@ __global__ void __launch_bounds__(kGuMaxWarps * 32, 1) expert_gate_up_kernel(Sha
     const int n_warps = blockDim.x >> 5;
     const int xrow = x_row_bytes(H);
     unsigned char* xt = smem;
-    unsigned char* ring = smem + (size_t)2 * tok_cap * xrow + (size_t)warp * kRingWarpBytes;
+    unsigned char* ring = smem + (size_t)2 * tok_cap * xrow + (size_t)warp * kGuRingWarpBytes;
     const int4* groups = reinterpret_cast<const int4*>(b.groups);
     const int n_groups = *b.n_groups;
     const int upe = I / 8;                                   // units per group
@@ -299,7 +344,7 @@ __global__ void __launch_bounds__(kGuMaxWarps * 32, 1) expert_gate_up_kernel(Sha
     int icount = 0, ccount = 0;
     auto issue_next = [&]() {                                // one slice (or nothing) and one commit group
         if (ic.g <= g_last) {
-            ring_issue(ring, icount % kRing, lane, ic.p0 + (size_t)ic.sl * 32, ic.p1 + (size_t)ic.sl * 32);
+            ring_issue(ring, icount % kGuRing, lane, ic.p0 + (size_t)ic.sl * 32, ic.p1 + (size_t)ic.sl * 32);
             if (++ic.sl == n_slices) {
                 ic.sl = 0;
                 ic.u += n_warps;
@@ -310,7 +355,7 @@ __global__ void __launch_bounds__(kGuMaxWarps * 32, 1) expert_gate_up_kernel(Sha
         ++icount;
     };
 #pragma unroll 1
-    for (int i = 0; i < kRing; ++i) issue_next();
+    for (int i = 0; i < kGuRing; ++i) issue_next();
 
     const int pieces = H / 8;
     for (int g = g_first; g <= g_last; ++g) {
@@ -334,32 +379,17 @@ __global__ void __launch_bounds__(kGuMaxWarps * 32, 1) expert_gate_up_kernel(Sha
             const int row = (u - g * upe) * 8 + gid;
             if (nt == 1) {
                 float acc[1][4] = {{0.f, 0.f, 0.f, 0.f}};
-                for (int sl = 0; sl < n_slices; ++sl) {
-                    cp_async_wait<kRing - 1>();
-                    ring_consume<1>(ring, ccount % kRing, lane, xs + (size_t)sl * 64, 8 * xrow, acc);
-                    ++ccount;
-                    issue_next();
-                }
+                gu_stream<1>(ring, ccount, lane, xs, xrow, n_slices, acc, issue_next);
                 gate_up_epilogue<1>(acc, m_here, row, I, act_out, tig);
             } else if (nt == 2) {
                 float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                for (int sl = 0; sl < n_slices; ++sl) {
-                    cp_async_wait<kRing - 1>();
-                    ring_consume<2>(ring, ccount % kRing, lane, xs + (size_t)sl * 64, 8 * xrow, acc);
-                    ++ccount;
-                    issue_next();
-                }
+                gu_stream<2>(ring, ccount, lane, xs, xrow, n_slices, acc, issue_next);
                 gate_up_epilogue<2>(acc, m_here, row, I, act_out, tig);
             } else {
                 float acc[4][4];
 #pragma unroll
                 for (int n = 0; n < 4; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-                for (int sl = 0; sl < n_slices; ++sl) {
-                    cp_async_wait<kRing - 1>();
-                    ring_consume<4>(ring, ccount % kRing, lane, xs + (size_t)sl * 64, 8 * xrow, acc);
-                    ++ccount;
-                    issue_next();
-                }
+                gu_stream<4>(ring, ccount, lane, xs, xrow, n_slices, acc, issue_next);
                 gate_up_epilogue<4>(acc, m_here, row, I, act_out, tig);
             }
         }
@@ -557,7 +587,7 @@ static void expert_plan(const Shape& s, int n_tok, int* cap, int* warps) {
     *cap = avg <= 5.0 ? 8 : 16;
     while ((size_t)*cap * 2 * x_row_bytes(s.H) > 140u * 1024u && *cap > 4) *cap /= 2;
     const size_t left = 227u * 1024u - 1024u - (size_t)*cap * 2 * x_row_bytes(s.H);
-    int w = (int)(left / kRingWarpBytes);
+    int w = (int)(left / kGuRingWarpBytes);
     *warps = w > kGuMaxWarps ? kGuMaxWarps : (w < 1 ? 1 : w);
 }
 
@@ -578,7 +608,7 @@ int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const Debug
 int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st) {
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
-    const size_t smem = (size_t)cap * 2 * x_row_bytes(s.H) + (size_t)warps * kRingWarpBytes;
+    const size_t smem = (size_t)cap * 2 * x_row_bytes(s.H) + (size_t)warps * kGuRingWarpBytes;
     launch_chained(expert_gate_up_kernel, dim3(sm_count), dim3(warps * 32), smem, st, s, b, w.w_gate_up, cap);
     return 1;
 }
