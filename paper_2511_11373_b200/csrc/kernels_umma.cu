@@ -1,16 +1,18 @@
 // Dense contractions of chunked prefill on the 5th-generation tensor cores (tcgen05 + TMEM).
 //
 // C[m, n] = sum_k X[m, k] W[n, k] for hundreds to thousands of token rows m: a real dense
-// contraction, unlike the decode-sized streams.  One CTA computes a 128 x 256 output tile:
+// contraction, unlike the decode-sized streams.  A persistent CTA per SM walks 128 x 256 output tiles:
 //   warp 0 (one lane)  TMA producer: per 64-wide K stage the hi plane and the lo plane of 128
 //                      activation rows and four 64-row boxes of weights, 128-byte swizzle, into a
-//                      3-stage ring (mbarrier full/empty pairs);
+//                      3-stage ring (mbarrier full/empty pairs) that runs on across tile boundaries;
 //   warp 1 (one lane)  issues tcgen05.mma (M 128, N 256, K 16, bf16 x bf16 -> fp32 in TMEM): per
 //                      stage four K steps for the hi plane and four for the lo plane, all into the
-//                      same accumulator, then tcgen05.commit to release the stage;
-//   warps 2..5         epilogue: wait for the accumulator, tcgen05.ld (each warp its 32-lane
+//                      same accumulator, then tcgen05.commit to release the stage; tiles alternate
+//                      between two accumulators (2 x 256 TMEM columns);
+//   warps 2..5         epilogue: wait for an accumulator, tcgen05.ld (each warp its 32-lane
 //                      quarter of TMEM), then either store fp32 rows or apply SwiGLU to the
-//                      (gate, up) column halves and store (hi, lo) bf16 pairs.
+//                      (gate, up) column halves and store (hi, lo) bf16 pairs, and hand the
+//                      accumulator back -- all while the next tile's MMAs run.
 // Activations are (hi, lo) bf16 pairs stored [row][2][K]; a 3-D tensor map (K, plane, row) picks a
 // plane of 128 rows as one box.  For the experts the rows are expert slots (tokens gathered in
 // expert order) and a tile is one entry of the permute kernel's group list.
@@ -125,98 +127,131 @@ struct UmmaParams {
     float inv_temp;
     float2* score_ml;
     float* score_tgt;
+    int tiles_x;              // column tiles per row tile (mode 1: 128 output columns each, else 256)
 };
+
+// The kernel is persistent: CTA c computes tiles c, c + gridDim.x, ... (column tile fastest, so that
+// CTAs running side by side share the row tile's activations and, for grouped calls, an expert's
+// weights through the L2).  Tensor memory holds TWO accumulators (2 x 256 columns): while the four
+// epilogue warps drain tile t, the MMA lane already accumulates tile t + 1, and the TMA producer runs
+// ahead through the ring across tile boundaries, so the tensor pipe only idles at the very start.
+struct UmTile { int m0, m_valid, b_row0, b_row1, col0, x; };
+
+__device__ __forceinline__ UmTile um_tile(const UmmaParams& p, int tile) {
+    UmTile t;
+    const int y = tile / p.tiles_x;
+    t.x = tile - y * p.tiles_x;
+    if (p.groups) {
+        const int4 g = reinterpret_cast<const int4*>(p.groups)[y];
+        t.m0 = g.y; t.m_valid = g.z;
+        const int base = g.x * p.b_rows_per_expert;
+        if (p.swiglu) { t.col0 = t.x * 128; t.b_row0 = base + t.col0; t.b_row1 = base + p.n_cols + t.col0; }
+        else { t.col0 = t.x * kUmTileN; t.b_row0 = base + t.col0; t.b_row1 = t.b_row0 + 128; }
+    } else {
+        t.m0 = y * kUmTileM; t.m_valid = min(kUmTileM, p.m_rows - t.m0);
+        t.col0 = t.x * kUmTileN; t.b_row0 = t.col0; t.b_row1 = t.col0 + 128;
+    }
+    return t;
+}
+
+__device__ __forceinline__ void um_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 
 __global__ void __launch_bounds__(kUmThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, UmmaParams p) {
     extern __shared__ unsigned char um_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)um_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t full_bar[kUmStages], empty_bar[kUmStages], accum_bar;
+    __shared__ __align__(8) uint64_t full_bar[kUmStages], empty_bar[kUmStages], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int dead;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    pdl_wait();      // the group list and the activations come from earlier kernels
-
-    // which rows of A and B this tile contracts
-    int m0, m_valid, b_row0, b_row1, col0;     // b_row0 / b_row1: first weight row of each 128-column half
-    if (p.groups) {
-        if ((int)blockIdx.y >= *p.n_groups) return;                 // uniform for the CTA
-        const int4 g = reinterpret_cast<const int4*>(p.groups)[blockIdx.y];
-        m0 = g.y; m_valid = g.z;
-        const int base = g.x * p.b_rows_per_expert;
-        if (p.swiglu) { col0 = blockIdx.x * 128; b_row0 = base + col0; b_row1 = base + p.n_cols + col0; }
-        else { col0 = blockIdx.x * kUmTileN; b_row0 = base + col0; b_row1 = b_row0 + 128; }
-    } else {
-        m0 = blockIdx.y * kUmTileM; m_valid = min(kUmTileM, p.m_rows - m0);
-        col0 = blockIdx.x * kUmTileN; b_row0 = col0; b_row1 = col0 + 128;
-    }
-    const int nk = p.K / kUmStageK;
 
     if (tid == 0) {
         for (int i = 0; i < kUmStages; ++i) { um_mbar_init(&full_bar[i], 1); um_mbar_init(&empty_bar[i], 1); }
-        um_mbar_init(&accum_bar, 1);
+        for (int i = 0; i < 2; ++i) { um_mbar_init(&acc_full[i], 1); um_mbar_init(&acc_empty[i], 4); }
         dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 2) {   // one warp allocates the TMEM columns (fp32 accumulator: 128 lanes x 256 columns)
+    if (warp == 2) {   // one warp allocates the TMEM columns: two fp32 accumulators of 128 lanes x 256 columns
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
-                     "r"(kUmTileN));
+                     "r"(2 * kUmTileN));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_d = tmem_slot;
+    pdl_wait();      // the group list and the activations come from earlier kernels
+
+    const int nk = p.K / kUmStageK;
+    const int n_y = p.groups ? *p.n_groups : (p.m_rows + kUmTileM - 1) / kUmTileM;
+    const int n_tiles = n_y * p.tiles_x;
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int ks = 0; ks < nk && !dead; ++ks) {
-                const int s = ks % kUmStages;
-                if (ks >= kUmStages && !um_wait(&empty_bar[s], ((ks / kUmStages) - 1) & 1)) {
-                    dead = 1; atomicOr(p.err, kErrTimeout); break;
+            uint32_t it = 0;                                         // ring stages produced so far
+            for (int tile = blockIdx.x; tile < n_tiles && !dead; tile += gridDim.x) {
+                const UmTile t = um_tile(p, tile);
+                for (int ks = 0; ks < nk && !dead; ++ks, ++it) {
+                    const int s = it % kUmStages;
+                    if (!um_wait(&empty_bar[s], ((it / kUmStages) & 1) ^ 1)) {   // passes at once in the first round
+                        dead = 1; atomicOr(p.err, kErrTimeout); break;
+                    }
+                    unsigned char* st = smem + (size_t)s * kUmStageBytes;
+                    um_expect_tx(&full_bar[s], kUmStageBytes);
+                    um_tma_3d(st, &tm_a, ks * kUmStageK, 0, t.m0, &full_bar[s]);
+                    um_tma_3d(st + kUmTileBytes, &tm_a, ks * kUmStageK, 1, t.m0, &full_bar[s]);
+                    unsigned char* sb = st + 2 * kUmTileBytes;        // four boxes of 64 weight rows (8 KB each)
+                    um_tma_2d(sb, &tm_b, ks * kUmStageK, t.b_row0, &full_bar[s]);
+                    um_tma_2d(sb + 8192, &tm_b, ks * kUmStageK, t.b_row0 + 64, &full_bar[s]);
+                    um_tma_2d(sb + 16384, &tm_b, ks * kUmStageK, t.b_row1, &full_bar[s]);
+                    um_tma_2d(sb + 24576, &tm_b, ks * kUmStageK, t.b_row1 + 64, &full_bar[s]);
                 }
-                unsigned char* st = smem + (size_t)s * kUmStageBytes;
-                um_expect_tx(&full_bar[s], kUmStageBytes);
-                um_tma_3d(st, &tm_a, ks * kUmStageK, 0, m0, &full_bar[s]);
-                um_tma_3d(st + kUmTileBytes, &tm_a, ks * kUmStageK, 1, m0, &full_bar[s]);
-                unsigned char* sb = st + 2 * kUmTileBytes;            // four boxes of 64 weight rows (8 KB each)
-                um_tma_2d(sb, &tm_b, ks * kUmStageK, b_row0, &full_bar[s]);
-                um_tma_2d(sb + 8192, &tm_b, ks * kUmStageK, b_row0 + 64, &full_bar[s]);
-                um_tma_2d(sb + 16384, &tm_b, ks * kUmStageK, b_row1, &full_bar[s]);
-                um_tma_2d(sb + 24576, &tm_b, ks * kUmStageK, b_row1 + 64, &full_bar[s]);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            for (int ks = 0; ks < nk && !dead; ++ks) {
-                const int s = ks % kUmStages;
-                if (!um_wait(&full_bar[s], (ks / kUmStages) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); break; }
+            uint32_t it = 0;
+            int local = 0;                                           // tiles of this CTA so far
+            for (int tile = blockIdx.x; tile < n_tiles && !dead; tile += gridDim.x, ++local) {
+                const int buf = local & 1;
+                // the epilogue must have drained this accumulator (two tiles ago)
+                if (!um_wait(&acc_empty[buf], ((local >> 1) & 1) ^ 1)) { dead = 1; atomicOr(p.err, kErrTimeout); break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_hi = smem_u32(smem + (size_t)s * kUmStageBytes);
-                const uint64_t d_hi = um_smem_desc(a_hi), d_lo = um_smem_desc(a_hi + kUmTileBytes),
-                               d_b = um_smem_desc(a_hi + 2 * kUmTileBytes);
+                const uint32_t acc = tmem_d + (uint32_t)(buf * kUmTileN);
+                for (int ks = 0; ks < nk && !dead; ++ks, ++it) {
+                    const int s = it % kUmStages;
+                    if (!um_wait(&full_bar[s], (it / kUmStages) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_hi = smem_u32(smem + (size_t)s * kUmStageBytes);
+                    const uint64_t d_hi = um_smem_desc(a_hi), d_lo = um_smem_desc(a_hi + kUmTileBytes),
+                                   d_b = um_smem_desc(a_hi + 2 * kUmTileBytes);
 #pragma unroll
-                for (int kk = 0; kk < kUmStageK / 16; ++kk) {       // 32 bytes along K per step: +2 in the address field
-                    um_mma(tmem_d, d_hi + 2 * kk, d_b + 2 * kk, (ks | kk) != 0);
-                    um_mma(tmem_d, d_lo + 2 * kk, d_b + 2 * kk, 1u);
+                    for (int kk = 0; kk < kUmStageK / 16; ++kk) {   // 32 bytes along K per step: +2 in the address field
+                        um_mma(acc, d_hi + 2 * kk, d_b + 2 * kk, (ks | kk) != 0);
+                        um_mma(acc, d_lo + 2 * kk, d_b + 2 * kk, 1u);
+                    }
+                    um_commit(&empty_bar[s]);                        // the stage is free once these MMAs retire
                 }
-                um_commit(&empty_bar[s]);                            // the stage is free once these MMAs retire
+                um_commit(&acc_full[buf]);
             }
-            um_commit(&accum_bar);
         }
     } else {
         // epilogue: a warp may touch the TMEM lanes 32 (warp % 4) .. +31
         const int quarter = warp & 3;
         const int r = quarter * 32 + lane;                           // row of the tile = TMEM lane
-        bool ok = true;
-        if (lane == 0 && !um_wait(&accum_bar, 0)) { dead = 1; atomicOr(p.err, kErrTimeout); }
-        __syncwarp();
-        ok = !dead;
-        ok = __all_sync(0xffffffffu, ok);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {
-            const uint32_t lane_base = tmem_d + ((uint32_t)(quarter * 32) << 16);
+        int local = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++local) {
+            const int buf = local & 1;
+            const UmTile t = um_tile(p, tile);
+            const int m0 = t.m0, m_valid = t.m_valid, col0 = t.col0;
+            if (lane == 0 && !dead && !um_wait(&acc_full[buf], (local >> 1) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); }
+            __syncwarp();
+            if (!__all_sync(0xffffffffu, !dead)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t lane_base = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kUmTileN);
             if (!p.swiglu) {
 #pragma unroll 1
                 for (int c = 0; c < kUmTileN; c += 32) {
@@ -266,7 +301,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                     }
                 }
                 if (live) {
-                    p.score_ml[(size_t)blockIdx.x * p.m_rows + m0 + r] = make_float2(mx, sum);
+                    p.score_ml[(size_t)t.x * p.m_rows + m0 + r] = make_float2(mx, sum);
                     if (tgt >= col0 && tgt < col0 + kUmTileN && tgt < p.n_cols) p.score_tgt[m0 + r] = zt;
                 }
             } else {
@@ -276,23 +311,40 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                     um_ld32(lane_base + c, gt);
                     um_ld32(lane_base + 128 + c, up);
                     if (r < m_valid) {
+                        // expert_inter is a multiple of 64: a run of 8 columns is inside or outside as a whole
                         __nv_bfloat16* dst = p.act + (size_t)(m0 + r) * 2 * p.n_cols + col0 + c;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
+                        for (int j = 0; j < 32; j += 8)
                             if (col0 + c + j < p.n_cols) {
-                                const float gte = __uint_as_float(gt[j]);
-                                split_bf16(gte / (1.f + expf(-gte)) * __uint_as_float(up[j]), dst[j], dst[p.n_cols + j]);
+                                uint32_t hi[4], lo[4];
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    float a[2];
+#pragma unroll
+                                    for (int e = 0; e < 2; ++e) {
+                                        const float gte = __uint_as_float(gt[j + 2 * q + e]);
+                                        a[e] = gte / (1.f + expf(-gte)) * __uint_as_float(up[j + 2 * q + e]);
+                                    }
+                                    hi[q] = pack_bf16(a[0], a[1]);
+                                    lo[q] = pack_bf16(a[0] - bf16_lo(hi[q]), a[1] - bf16_hi(hi[q]));
+                                }
+                                *reinterpret_cast<uint4*>(dst + j) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                                *reinterpret_cast<uint4*>(dst + p.n_cols + j) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                             }
                     }
                 }
             }
+            // this warp has read its lanes of the accumulator: hand it back to the MMA lane
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) um_arrive(&acc_empty[buf]);
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
     __syncthreads();
     if (warp == 2) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kUmTileN));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(2 * kUmTileN));
     }
 }
 
@@ -449,11 +501,15 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(Buffers b, int H, int 
 
 static size_t umma_smem_bytes() { return (size_t)kUmStages * kUmStageBytes + 1024; }
 
+// Persistent grid: one CTA per SM, or fewer when there are fewer tiles.
+static int g_umma_sms = 0;
+static int umma_grid(int tiles) { return tiles < g_umma_sms ? (tiles < 1 ? 1 : tiles) : g_umma_sms; }
+
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
                       int32_t* err, cudaStream_t st) {
-    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err, nullptr, 0.f, nullptr, nullptr};
-    dim3 grid((n_cols + kUmTileN - 1) / kUmTileN, (m_rows + kUmTileM - 1) / kUmTileM);
-    launch_chained(umma_gemm_kernel, dim3(grid), dim3(kUmThreads), umma_smem_bytes(), st, tm_a, tm_b, p);
+    const int tx = (n_cols + kUmTileN - 1) / kUmTileN, ty = (m_rows + kUmTileM - 1) / kUmTileM;
+    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err, nullptr, 0.f, nullptr, nullptr, tx};
+    launch_chained(umma_gemm_kernel, dim3(umma_grid(tx * ty)), dim3(kUmThreads), umma_smem_bytes(), st, tm_a, tm_b, p);
     return 1;
 }
 
@@ -462,11 +518,13 @@ int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_
     const int n_slots = n_tok * s.k;
     const int max_groups = s.E + (n_slots + kUmTileM - 1) / kUmTileM;
     launch_chained(gather_rows_kernel, dim3(n_slots), dim3(256), 0, st, b, s.H, n_slots);
-    UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err, nullptr, 0.f, nullptr, nullptr};
-    launch_chained(umma_gemm_kernel, dim3((s.I + 127) / 128, max_groups), dim3(kUmThreads), umma_smem_bytes(), st, tm_xperm, tm_wgu, gu);
-    UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err, nullptr, 0.f, nullptr, nullptr};
-    launch_chained(umma_gemm_kernel, dim3((s.H + kUmTileN - 1) / kUmTileN, max_groups), dim3(kUmThreads), umma_smem_bytes(), st, 
-        tm_act, tm_wdown, dn);
+    const int gx = (s.I + 127) / 128, dx = (s.H + kUmTileN - 1) / kUmTileN;
+    UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err, nullptr, 0.f, nullptr, nullptr, gx};
+    launch_chained(umma_gemm_kernel, dim3(umma_grid(gx * max_groups)), dim3(kUmThreads), umma_smem_bytes(), st, tm_xperm,
+                   tm_wgu, gu);
+    UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err, nullptr, 0.f, nullptr, nullptr, dx};
+    launch_chained(umma_gemm_kernel, dim3(umma_grid(dx * max_groups)), dim3(kUmThreads), umma_smem_bytes(), st, tm_act,
+                   tm_wdown, dn);
     return 3;
 }
 
@@ -503,10 +561,11 @@ __global__ void __launch_bounds__(256) score_combine_kernel(const float2* __rest
 int launch_umma_score(const CUtensorMap& tm_h, const CUtensorMap& tm_lm, int n_rows, int vocab, int K,
                       const int32_t* targets, float inv_temp, float2* score_ml, float* score_tgt, float* logits_tap,
                       float* out_logprobs, int32_t* err, cudaStream_t st) {
-    UmmaParams p{K, n_rows, nullptr, nullptr, 0, vocab, 2, logits_tap, nullptr, err, targets, inv_temp, score_ml, score_tgt};
     const int n_tiles = (vocab + kUmTileN - 1) / kUmTileN;
-    dim3 grid(n_tiles, (n_rows + kUmTileM - 1) / kUmTileM);
-    launch_chained(umma_gemm_kernel, dim3(grid), dim3(kUmThreads), umma_smem_bytes(), st, tm_h, tm_lm, p);
+    UmmaParams p{K, n_rows, nullptr, nullptr, 0, vocab, 2, logits_tap, nullptr, err, targets, inv_temp, score_ml, score_tgt,
+                 n_tiles};
+    launch_chained(umma_gemm_kernel, dim3(umma_grid(n_tiles * ((n_rows + kUmTileM - 1) / kUmTileM))), dim3(kUmThreads),
+                   umma_smem_bytes(), st, tm_h, tm_lm, p);
     launch_chained(score_combine_kernel, dim3((n_rows + 7) / 8), dim3(256), 0, st, score_ml, score_tgt, targets, n_rows, n_tiles, vocab,
                                                             out_logprobs, err);
     return 2;
@@ -515,7 +574,12 @@ int launch_umma_score(const CUtensorMap& tm_h, const CUtensorMap& tm_lm, int n_r
 int score_vocab_tiles(int vocab) { return (vocab + kUmTileN - 1) / kUmTileN; }
 
 cudaError_t init_umma_kernels() {
-    cudaError_t e = cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes());
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&g_umma_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes());
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(umma_swap_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)swap_smem_bytes());
 }
