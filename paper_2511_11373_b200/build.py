@@ -15,7 +15,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "libmars.so")
-SOURCES = ["kernels_dense.cu", "kernels_attn.cu", "kernels_moe.cu", "kernels_sample.cu", "kernels_umma.cu", "kernels_kv.cu",
+SOURCES = ["kernels_dense.cu", "kernels_attn.cu", "kernels_moe.cu", "kernels_sample.cu", "kernels_umma.cu", "kernels_fattn.cu", "kernels_kv.cu",
            "mars_api.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-I", os.path.join(ROOT, "include")]

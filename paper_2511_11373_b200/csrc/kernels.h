@@ -67,6 +67,13 @@ int launch_attention_shared(const Shape& s, const Buffers& b, const StepLayout& 
                             const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
                             cudaStream_t st);
 
+// Causal prefill attention on tcgen05 (head_dim 128, 8 query heads per KV head): items are blocks of up to
+// fattn_block_tokens() consecutive prompt tokens; tm_q is the 4-D map (d, head, plane, token) over b.q.
+bool fattn_supported(const Shape& s);
+int fattn_block_tokens();
+int launch_fattn_prefill(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_q,
+                         const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
+                         cudaStream_t st);
 int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st);
 
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,

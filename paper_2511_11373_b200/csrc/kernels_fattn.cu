@@ -1,0 +1,421 @@
+// Causal attention of chunked prefill on the 5th-generation tensor cores (tcgen05 + TMEM), for the
+// head shape head_dim 128 with 8 query heads per KV head.
+//
+// A work item is a block of up to 16 consecutive prompt tokens of one request; a unit is (item, KV
+// head).  The 16 tokens x 8 query heads of the KV head are the 128 rows of one MMA tile (row =
+// 8 * token + head), so one pass over the keys serves 128 query rows and the diagonal block of the
+// causal mask is only 16 tokens wide.  A persistent CTA per SM walks units; per unit
+//   warp 4 (one lane)   TMA producer: the Q tile (hi and lo planes, two 64-wide halves of head_dim,
+//                       through a 4-D tensor map (d, head, plane, token)), then the K and V page
+//                       tiles of 64 cached tokens each through a 3-stage ring;
+//   warp 5 (one lane)   MMA issuer: S = Q K^T (M 128, N 64, K 128; hi and lo planes of Q accumulate
+//                       into the same fp32 tile in TMEM, two S buffers), and, once the softmax warps
+//                       have written P, O_tile = P V (M 128, N 128, K 64; hi and lo planes of P), with V
+//                       read as an MN-major operand straight from the [token][d] page tile;
+//   warps 0..3          softmax: thread r owns row r (TMEM lane r): it reads its 64 scores with
+//                       tcgen05.ld, masks by its own causal length, keeps the running max and sum,
+//                       writes P = exp2(s - m) as (hi, lo) bf16 pairs into a swizzled K-major shared
+//                       tile, and adds O_tile into its 128 fp32 output registers after rescaling
+//                       them (the output accumulator lives in registers, so no TMEM round trip is
+//                       needed when the running max moves).
+// While the softmax warps work on tile j the tensor pipe already computes S of tile j + 1.
+// Every wait is bounded: a wait that gives up sets the device status word, all roles stop, the CTA
+// frees its TMEM columns and returns.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace mars {
+
+constexpr int kFaQ = 16;                   // query tokens per block
+constexpr int kFaHeads = 8;                // query heads per KV head
+constexpr int kFaRows = kFaQ * kFaHeads;   // 128 rows of the MMA tile
+constexpr int kFaD = 128;
+constexpr int kFaKv = 64;                  // cached tokens per tile
+constexpr int kFaStages = 3;
+constexpr int kFaQTile = kFaRows * 128;    // one (plane, half) tile of Q: 128 rows x 128 B = 16 KB
+constexpr int kFaQBytes = 4 * kFaQTile;    // hi/lo x two halves of head_dim
+constexpr int kFaPTile = kFaRows * 128;    // one plane of P: 128 rows x 64 tokens bf16
+constexpr int kFaHalf = kFaKv * 128;       // one 64-wide half of a K or V tile: 64 tokens x 128 B = 8 KB
+constexpr int kFaStageBytes = 4 * kFaHalf; // K halves, V halves
+constexpr int kFaSmem = kFaQBytes + 2 * kFaPTile + kFaStages * kFaStageBytes;
+constexpr int kFaThreads = 192;
+constexpr int kFaTmemCols = 256;           // S buffers at columns 0 and 64, O_tile at 128..255
+constexpr uint32_t kFaSpin = 1u << 22;
+
+struct FaParams {
+    const int32_t* step;
+    StepLayout lay;
+    const int32_t* block_table;
+    __nv_bfloat16* o_out;      // [n_tok][2][nq * D]
+    int32_t* err;
+    int max_pages_per_seq, n_pages, page_size, box_rows, nkv, nq, layer;
+    float scale_log2;
+};
+
+__device__ __forceinline__ void fa_mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void fa_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void fa_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool fa_wait(uint64_t* bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kFaSpin; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void fa_tma_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"((uint64_t)tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void fa_tma_4d(void* dst, const CUtensorMap* tm, int x, int y, int z, int w, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(smem_u32(dst)), "l"((uint64_t)tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar)) : "memory");
+}
+
+// Shared-memory matrix descriptors (descriptor version 1, 128-byte swizzle), see the PTX ISA.
+// K-major tile (rows of 128 B, 8-row groups 1024 B apart): Q, K and P.
+__device__ __forceinline__ uint64_t fa_desc_kmajor(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// MN-major tile: a row of 128 B holds 64 consecutive N elements (head_dim) of one K index (token);
+// 8-token groups are 1024 B apart (stride offset), the next 64 N elements `lbo` bytes further
+// (leading offset): the V page tile exactly as TMA writes it.
+__device__ __forceinline__ uint64_t fa_desc_mnmajor(uint32_t addr, uint32_t lbo) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3fffu);
+    d |= (uint64_t)((lbo >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptors: fp32 accumulator, bf16 operands; bit 16 = B is MN-major.
+constexpr uint32_t kFaIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kFaKv >> 3) << 17) | ((uint32_t)(kFaRows >> 4) << 24);
+constexpr uint32_t kFaIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(kFaD >> 3) << 17) |
+                               ((uint32_t)(kFaRows >> 4) << 24);
+
+__device__ __forceinline__ void fa_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void fa_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void fa_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct FaUnit { int row0, len, nq_blk, hk, n_tiles; const int32_t* bt; };
+
+__device__ __forceinline__ FaUnit fa_unit(const FaParams& p, int u) {
+    FaUnit c;
+    const int item = u / p.nkv;
+    c.hk = u - item * p.nkv;
+    const int4 it = reinterpret_cast<const int4*>(p.step + p.lay.items)[p.step[H_PF_FIRST] + item];
+    c.row0 = it.x; c.len = it.z; c.nq_blk = it.w;                  // len: keys visible to the LAST query of the block
+    c.n_tiles = (c.len + kFaKv - 1) / kFaKv;
+    c.bt = p.block_table + (size_t)p.step[p.lay.tok_seq + c.row0] * p.max_pages_per_seq;
+    return c;
+}
+
+__global__ void __launch_bounds__(kFaThreads, 1)
+fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                     const __grid_constant__ CUtensorMap tm_v, FaParams p) {
+    extern __shared__ unsigned char fa_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)fa_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char* q_smem = smem;                                   // [plane][half][128 rows][128 B]
+    unsigned char* p_smem = smem + kFaQBytes;                       // [plane][128 rows][128 B]
+    unsigned char* kv_smem = p_smem + 2 * kFaPTile;                 // [stage][K half 0, K half 1, V half 0, V half 1]
+    __shared__ __align__(8) uint64_t q_full, q_free, kv_full[kFaStages], kv_empty[kFaStages], s_ready[2], p_ready, o_ready;
+    __shared__ uint32_t tmem_slot;
+    __shared__ volatile int dead;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        fa_mbar_init(&q_full, 1); fa_mbar_init(&q_free, 1);
+        for (int i = 0; i < kFaStages; ++i) { fa_mbar_init(&kv_full[i], 1); fa_mbar_init(&kv_empty[i], 1); }
+        fa_mbar_init(&s_ready[0], 1); fa_mbar_init(&s_ready[1], 1);
+        fa_mbar_init(&p_ready, 4); fa_mbar_init(&o_ready, 1);
+        dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 4) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                     "r"(kFaTmemCols));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_slot;
+    pdl_wait();
+
+    const int n_units = p.step[H_PF_ITEMS] * p.nkv;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t g = 0;                                          // K/V tiles requested so far (ring position)
+            int local = 0;
+            for (int u = blockIdx.x; u < n_units && !dead; u += gridDim.x, ++local) {
+                const FaUnit c = fa_unit(p, u);
+                auto load_kv = [&](int j) -> bool {
+                    const int s = g % kFaStages;
+                    if (!fa_wait(&kv_empty[s], ((g / kFaStages) & 1) ^ 1)) return false;
+                    unsigned char* st = kv_smem + (size_t)s * kFaStageBytes;
+                    const int n_valid = min(kFaKv, c.len - j * kFaKv);
+                    const int n_boxes = (n_valid + p.box_rows - 1) / p.box_rows;
+                    fa_expect_tx(&kv_full[s], (uint32_t)(n_boxes * p.box_rows * 128 * 4));
+                    for (int bi = 0; bi < n_boxes; ++bi) {
+                        const int tok = j * kFaKv + bi * p.box_rows;
+                        const int page = c.bt[tok / p.page_size];
+                        const int y = (((p.layer * p.n_pages + page) * p.nkv + c.hk) * p.page_size) + tok % p.page_size;
+                        const int off = bi * p.box_rows * 128;
+#pragma unroll
+                        for (int hf = 0; hf < 2; ++hf) {
+                            fa_tma_2d(st + hf * kFaHalf + off, &tm_k, hf * 64, y, &kv_full[s]);
+                            fa_tma_2d(st + (2 + hf) * kFaHalf + off, &tm_v, hf * 64, y, &kv_full[s]);
+                        }
+                    }
+                    ++g;
+                    return true;
+                };
+                // the first K/V tiles may be requested while the previous unit still uses the Q tile
+                const int early = min(c.n_tiles, kFaStages - 1);
+                bool ok = true;
+                for (int j = 0; j < early && ok; ++j) ok = load_kv(j);
+                if (ok) ok = fa_wait(&q_free, (local & 1) ^ 1);
+                if (ok) {
+                    fa_expect_tx(&q_full, kFaQBytes);
+#pragma unroll
+                    for (int pl = 0; pl < 2; ++pl)
+#pragma unroll
+                        for (int hf = 0; hf < 2; ++hf)
+                            fa_tma_4d(q_smem + (pl * 2 + hf) * kFaQTile, &tm_q, hf * 64, c.hk * kFaHeads, pl, c.row0, &q_full);
+                }
+                for (int j = early; j < c.n_tiles && ok; ++j) ok = load_kv(j);
+                if (!ok) { dead = 1; atomicOr(p.err, kErrTimeout); }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t g = 0;                                          // K/V tiles consumed so far
+            int local = 0;
+            const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem);
+            auto issue_s = [&](uint32_t gi) -> bool {                // S(gi) = Q K^T into S buffer gi & 1
+                const int s = gi % kFaStages;
+                if (!fa_wait(&kv_full[s], (gi / kFaStages) & 1)) return false;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t k_addr = smem_u32(kv_smem + (size_t)s * kFaStageBytes);
+                const uint32_t acc = tmem + (gi & 1) * kFaKv;
+#pragma unroll
+                for (int pl = 0; pl < 2; ++pl)
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf) {
+                        const uint64_t da = fa_desc_kmajor(q_addr + (pl * 2 + hf) * kFaQTile);
+                        const uint64_t db = fa_desc_kmajor(k_addr + hf * kFaHalf);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) fa_mma(acc, da + 2 * kk, db + 2 * kk, kFaIdescS, (pl | hf | kk) != 0);
+                    }
+                fa_commit(&s_ready[gi & 1]);
+                return true;
+            };
+            for (int u = blockIdx.x; u < n_units && !dead; u += gridDim.x, ++local) {
+                const FaUnit c = fa_unit(p, u);
+                bool ok = fa_wait(&q_full, local & 1);
+                if (ok) ok = issue_s(g);
+                for (int j = 0; j < c.n_tiles && ok; ++j, ++g) {
+                    ok = fa_wait(&p_ready, g & 1);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const int s = g % kFaStages;
+                    const uint32_t v_addr = smem_u32(kv_smem + (size_t)s * kFaStageBytes + 2 * kFaHalf);
+                    const uint64_t dv = fa_desc_mnmajor(v_addr, kFaHalf);
+#pragma unroll
+                    for (int pl = 0; pl < 2; ++pl) {
+                        const uint64_t dp = fa_desc_kmajor(p_addr + pl * kFaPTile);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)     // 16 tokens per step: 32 B along a P row, 2048 B down the V tile
+                            fa_mma(tmem + 128, dp + 2 * kk, dv + 128 * kk, kFaIdescO, (pl | kk) != 0);
+                    }
+                    fa_commit(&o_ready);
+                    fa_commit(&kv_empty[s]);
+                    if (j + 1 < c.n_tiles) ok = issue_s(g + 1);
+                }
+                if (!ok) { dead = 1; atomicOr(p.err, kErrTimeout); break; }
+                fa_commit(&q_free);                                  // every MMA that reads this unit's Q has been issued
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax warps
+        const int r = warp * 32 + lane;                              // row of the tile = TMEM lane
+        const int q_tok = r >> 3, head = r & 7;
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        uint32_t g = 0;
+        for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+            const FaUnit c = fa_unit(p, u);
+            // keys visible to this row's query; rows past the block's last token are computed but never stored
+            const int my_len = min(c.len, c.len - (c.nq_blk - 1 - q_tok));
+            float o[kFaD];
+#pragma unroll
+            for (int i = 0; i < kFaD; ++i) o[i] = 0.f;
+            float m_run = -INFINITY, l_run = 0.f;
+            bool alive = true;
+            for (int j = 0; j < c.n_tiles; ++j, ++g) {
+                if (lane == 0 && !dead && !fa_wait(&s_ready[g & 1], (g >> 1) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); }
+                __syncwarp();
+                alive = __all_sync(0xffffffffu, !dead);
+                if (!alive) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                // scores of this row: 64 columns of the S buffer
+                const int kv0 = j * kFaKv;
+                float sv[kFaKv];
+                float mx = -INFINITY;
+#pragma unroll
+                for (int cb = 0; cb < kFaKv; cb += 32) {
+                    uint32_t v[32];
+                    fa_ld32(lane_base + (g & 1) * kFaKv + cb, v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float s = kv0 + cb + i < my_len ? __uint_as_float(v[i]) * p.scale_log2 : -INFINITY;
+                        sv[cb + i] = s;
+                        mx = fmaxf(mx, s);
+                    }
+                }
+                const float m_new = fmaxf(m_run, mx);
+                const float m_use = m_new == -INFINITY ? 0.f : m_new;     // rows past the block see nothing at all
+                const float alpha = exp2f(m_run - m_use);
+                float sum = 0.f;
+                // P as (hi, lo) bf16 planes, K-major with the 128-byte swizzle: 16-byte chunk c of row r
+                // sits at r * 128 + ((c ^ (r & 7)) << 4)
+                unsigned char* prow = p_smem + r * 128;
+#pragma unroll
+                for (int ch = 0; ch < kFaKv / 8; ++ch) {
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float a = exp2f(sv[ch * 8 + 2 * q] - m_use), b2 = exp2f(sv[ch * 8 + 2 * q + 1] - m_use);
+                        sum += a + b2;
+                        hi[q] = pack_bf16(a, b2);
+                        lo[q] = pack_bf16(a - bf16_lo(hi[q]), b2 - bf16_hi(hi[q]));
+                    }
+                    const int sw = (ch ^ (r & 7)) << 4;
+                    *reinterpret_cast<uint4*>(prow + sw) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4*>(prow + kFaPTile + sw) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                }
+                l_run = l_run * alpha + sum;
+                m_run = m_new;
+                // the last tile may reach past the request's tokens: those value rows hold whatever the page
+                // holds, and 0 * NaN is NaN, so they are cleared (whole rows: the swizzle permutes within a row)
+                const int n_valid = min(kFaKv, c.len - kv0);
+                if (n_valid < kFaKv) {
+                    unsigned char* vt = kv_smem + (size_t)(g % kFaStages) * kFaStageBytes + 2 * kFaHalf;
+                    for (int i = r; i < (kFaKv - n_valid) * 16; i += kFaRows) {
+                        const int row = n_valid + (i >> 4), piece = i & 15;
+                        *reinterpret_cast<uint4*>(vt + (piece >> 3) * kFaHalf + row * 128 + (piece & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+                // P (and the cleared rows) must be visible to the tensor core's reads; the S buffer and
+                // the previous O_tile have been read: hand over to the MMA lane
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) fa_arrive(&p_ready);
+                // O_tile = P V of this tile
+                if (lane == 0 && !dead && !fa_wait(&o_ready, g & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); }
+                __syncwarp();
+                alive = __all_sync(0xffffffffu, !dead);
+                if (!alive) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                for (int cb = 0; cb < kFaD; cb += 32) {
+                    uint32_t v[32];
+                    fa_ld32(lane_base + 128 + cb, v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[cb + i] = fmaf(o[cb + i], alpha, __uint_as_float(v[i]));
+                }
+            }
+            if (!alive) break;
+            if (q_tok < c.nq_blk) {
+                const float inv = 1.f / l_run;
+                __nv_bfloat16* dst = p.o_out + (size_t)(c.row0 + q_tok) * 2 * p.nq * kFaD + (size_t)(c.hk * kFaHeads + head) * kFaD;
+#pragma unroll
+                for (int i = 0; i < kFaD; i += 8) {
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float a = o[i + 2 * q] * inv, b2 = o[i + 2 * q + 1] * inv;
+                        hi[q] = pack_bf16(a, b2);
+                        lo[q] = pack_bf16(a - bf16_lo(hi[q]), b2 - bf16_hi(hi[q]));
+                    }
+                    *reinterpret_cast<uint4*>(dst + i) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4*>(dst + (size_t)p.nq * kFaD + i) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 4) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kFaTmemCols));
+    }
+}
+
+bool fattn_supported(const Shape& s) { return s.D == kFaD && s.nq / s.nkv == kFaHeads; }
+int fattn_block_tokens() { return kFaQ; }
+
+int launch_fattn_prefill(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_q,
+                         const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
+                         cudaStream_t st) {
+    FaParams p;
+    p.step = b.step; p.lay = lay; p.block_table = kv.block_table; p.o_out = b.o; p.err = b.err;
+    p.max_pages_per_seq = kv.max_pages_per_seq; p.n_pages = kv.n_pages; p.page_size = kv.page_size;
+    p.box_rows = kv.page_size < kFaKv ? kv.page_size : kFaKv;
+    p.nkv = s.nkv; p.nq = s.nq; p.layer = layer;
+    p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
+    int grid = n_items * s.nkv;
+    if (grid > sm_count) grid = sm_count;
+    if (grid < 1) grid = 1;
+    launch_chained(fattn_prefill_kernel, dim3(grid), dim3(kFaThreads), (size_t)kFaSmem + 1024, st, tm_q, tm_k, tm_v, p);
+    return 1;
+}
+
+cudaError_t init_fattn_kernels() {
+    return cudaFuncSetAttribute(fattn_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmem + 1024);
+}
+
+}  // namespace mars

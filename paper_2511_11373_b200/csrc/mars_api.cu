@@ -17,6 +17,7 @@ cudaError_t init_dense_kernels();
 cudaError_t init_attn_kernels();
 cudaError_t init_moe_kernels();
 cudaError_t init_umma_kernels();
+cudaError_t init_fattn_kernels();
 }  // namespace mars
 
 using namespace mars;
@@ -143,7 +144,7 @@ static mars_status_t make_tiled_map(CUtensorMap* tm, const void* base, int rank,
     cudaDriverEntryPointQueryResult qres;
     CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
     if (!fn || qres != cudaDriverEntryPointSuccess) return MARS_ERR_UNSUPPORTED;
-    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
     CUresult r = ((EncodeTiledFn)fn)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims,
                                      strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -153,6 +154,12 @@ static mars_status_t make_tiled_map(CUtensorMap* tm, const void* base, int rank,
         return MARS_ERR_CUDA;
     }
     return MARS_OK;
+}
+// queries [token][2][nq][D] as a 4-D tensor (d, head, plane, token): boxes of 64 elements x 8 heads x 16 tokens
+static mars_status_t make_query_map(CUtensorMap* tm, const void* q, uint64_t tokens, uint64_t nq, uint64_t D) {
+    const cuuint64_t dims[4] = {D, nq, 2, tokens}, strides[3] = {D * 2, nq * D * 2, 2 * nq * D * 2};
+    const cuuint32_t box[4] = {64u, 8u, 1u, 16u};
+    return make_tiled_map(tm, q, 4, dims, strides, box);
 }
 // weights [rows][K]: boxes of 64 rows x 64 elements
 static mars_status_t make_weight_map(CUtensorMap* tm, const void* w, uint64_t rows, uint64_t K) {
@@ -178,6 +185,8 @@ struct mars_model {
     std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown, tm_router;
     CUtensorMap tm_h, tm_o, tm_xperm, tm_act;
     CUtensorMap tm_h64, tm_o64, tm_lm;      // decode-sized (64 token rows per box) and the lm_head
+    CUtensorMap tm_q;                       // queries for the tcgen05 prefill attention: (d, head, plane, token)
+    bool fattn_ready;
     bool umma_ready;
     const __nv_bfloat16 *embed, *final_norm, *lm_head;
     int32_t *io_in, *io_out;
@@ -268,6 +277,7 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
     CUDA_TRY(init_attn_kernels());
     CUDA_TRY(init_moe_kernels());
     CUDA_TRY(init_umma_kernels());
+    CUDA_TRY(init_fattn_kernels());
 
     mars_model* m = new (std::nothrow) mars_model();
     if (!m) return MARS_ERR_INVALID_ARG;
@@ -345,6 +355,11 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
             if (rc == MARS_OK) rc = make_pair_map(&m->tm_o, m->buf.o, n, QD);
             if (rc == MARS_OK) rc = make_pair_map(&m->tm_xperm, m->buf.xperm, slots, H);
             if (rc == MARS_OK) rc = make_pair_map(&m->tm_act, m->buf.act, slots, I);
+        }
+        m->fattn_ready = false;
+        if (rc == MARS_OK && big && fattn_supported(m->shape)) {
+            rc = make_query_map(&m->tm_q, m->buf.q, n, (uint64_t)cfg->n_q_heads, (uint64_t)cfg->head_dim);
+            m->fattn_ready = rc == MARS_OK;
         }
         if (rc != MARS_OK) {
             mars_model_free(m);
@@ -724,7 +739,10 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     // attention work items: spans of `span` cached tokens per token row (widened until they fit)
     int span = plan.span;
     int64_t n_items = 0;
-    constexpr int kPrefillBlock = 4;   // consecutive prompt tokens per item of the causal prefill kernel
+    // consecutive prompt tokens per item of the causal prefill kernel: 16 (x 8 heads = 128 tensor-core rows)
+    // where the tcgen05 kernel applies, else 4 (one per warp of the mma.sync kernel)
+    const bool fattn = m->fattn_ready && n_tok > n_dec;
+    const int kPrefillBlock = fattn ? fattn_block_tokens() : 4;
     int64_t pf_items = 0;
     for (int t = n_dec; t < n_tok;) {
         int e = t + 1;
@@ -899,6 +917,9 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         }
         if (n_dec < n_tok) {  // prompt rows: causal kernel over blocks of tokens; writes the merged output itself
             run(MARS_K_ATTN, [&] {
+                if (fattn)
+                    return launch_fattn_prefill(s, b, lay, kv->view, m->tm_q, kv->tm_k, kv->tm_v, l, (int)pf_items,
+                                                m->sm_count, st);
                 return launch_attention_prefill(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st);
             });
         }

@@ -308,6 +308,21 @@ def test_prefill_many_tokens_tensor_core_path():
     run_and_compare(case, toks, label="decode after large prefill")
 
 
+MODEL_GQA8 = dict(n_layers=2, hidden=512, n_q_heads=16, n_kv_heads=2, head_dim=128, n_experts=8, top_k=2, expert_inter=128,
+                  vocab=1024, qk_norm=1, rope_theta=1e6, rms_eps=1e-6)
+
+
+@pytest.mark.parametrize("ps", [16, 64, 128])
+def test_prefill_attention_on_tensor_cores(ps):
+    """head_dim 128 with 8 query heads per KV head: the causal attention of a prefill-sized call runs
+    on tcgen05 (blocks of 16 prompt tokens x 8 heads = 128 accumulator rows, 64-token key tiles).
+    Chunks start at position 0, inside a page and on a page boundary; lengths leave ragged last
+    blocks (70 = 4 x 16 + 6) and ragged last key tiles; one chunk is a single token."""
+    case, toks = prefill_and_compare(MODEL_GQA8, ps, [0, 21, 128, 300, 64], [70, 33, 150, 1, 64], seed=24 + ps,
+                                     label=f"prefill-tcgen05-attention ps={ps}")
+    run_and_compare(case, toks, label="decode after tcgen05 prefill attention")
+
+
 def test_prefill_in_two_calls_equals_one_call():
     model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=0)
     V = model["vocab"]
