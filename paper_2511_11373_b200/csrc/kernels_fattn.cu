@@ -5,19 +5,22 @@
 // head).  The 16 tokens x 8 query heads of the KV head are the 128 rows of one MMA tile (row =
 // 8 * token + head), so one pass over the keys serves 128 query rows and the diagonal block of the
 // causal mask is only 16 tokens wide.  A persistent CTA per SM walks units; per unit
-//   warp 4 (one lane)   TMA producer: the Q tile (hi and lo planes, two 64-wide halves of head_dim,
+//   warp 8 (one lane)   TMA producer: the Q tile (hi and lo planes, two 64-wide halves of head_dim,
 //                       through a 4-D tensor map (d, head, plane, token)), then the K and V page
 //                       tiles of 64 cached tokens each through a 3-stage ring;
-//   warp 5 (one lane)   MMA issuer: S = Q K^T (M 128, N 64, K 128; hi and lo planes of Q accumulate
+//   warp 9 (one lane)   MMA issuer: S = Q K^T (M 128, N 64, K 128; hi and lo planes of Q accumulate
 //                       into the same fp32 tile in TMEM, two S buffers), and, once the softmax warps
 //                       have written P, O_tile = P V (M 128, N 128, K 64; hi and lo planes of P), with V
 //                       read as an MN-major operand straight from the [token][d] page tile;
-//   warps 0..3          softmax: thread r owns row r (TMEM lane r): it reads its 64 scores with
-//                       tcgen05.ld, masks by its own causal length, keeps the running max and sum,
-//                       writes P = exp2(s - m) as (hi, lo) bf16 pairs into a swizzled K-major shared
-//                       tile, and adds O_tile into its 128 fp32 output registers after rescaling
-//                       them (the output accumulator lives in registers, so no TMEM round trip is
-//                       needed when the running max moves).
+//   warps 0..7          softmax: two threads share row r (TMEM lane r; warp w reads lanes 32 (w % 4) ..,
+//                       warps 0..3 the first half of the columns, warps 4..7 the second): each reads
+//                       its 32 scores with tcgen05.ld, masks by the row's causal length, the two
+//                       exchange their maxima through shared memory, each writes its part of
+//                       P = exp2(s - m) as (hi, lo) bf16 pairs into a swizzled K-major shared tile and
+//                       adds its 64 columns of O_tile into fp32 output registers after rescaling them
+//                       (the output accumulator lives in registers, so no TMEM round trip is needed
+//                       when the running max moves).  Eight warps, two per scheduler, hide each
+//                       other's instruction latencies; with four the kernel ran at half the speed.
 // While the softmax warps work on tile j the tensor pipe already computes S of tile j + 1.
 // Every wait is bounded: a wait that gives up sets the device status word, all roles stop, the CTA
 // frees its TMEM columns and returns.
@@ -38,7 +41,8 @@ constexpr int kFaPTile = kFaRows * 128;    // one plane of P: 128 rows x 64 toke
 constexpr int kFaHalf = kFaKv * 128;       // one 64-wide half of a K or V tile: 64 tokens x 128 B = 8 KB
 constexpr int kFaStageBytes = 4 * kFaHalf; // K halves, V halves
 constexpr int kFaSmem = kFaQBytes + 2 * kFaPTile + kFaStages * kFaStageBytes;
-constexpr int kFaThreads = 192;
+constexpr int kFaThreads = 320;             // 8 softmax warps, producer warp, MMA warp
+constexpr int kFaSoftmaxThreads = 256;
 constexpr int kFaTmemCols = 256;           // S buffers at columns 0 and 64, O_tile at 128..255
 constexpr uint32_t kFaSpin = 1u << 22;
 
@@ -136,6 +140,12 @@ __device__ __forceinline__ void fa_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ float fa_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 struct FaUnit { int row0, len, nq_blk, hk, n_tiles; const int32_t* bt; };
 
 __device__ __forceinline__ FaUnit fa_unit(const FaParams& p, int u) {
@@ -160,18 +170,20 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     __shared__ __align__(8) uint64_t q_full, q_free, kv_full[kFaStages], kv_empty[kFaStages], s_ready[2], p_ready, o_ready;
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int dead;
+    __shared__ float xmax[2][2][kFaRows];                            // [tile parity][column half][row]
+    __shared__ float xsum[2][kFaRows];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
         fa_mbar_init(&q_full, 1); fa_mbar_init(&q_free, 1);
         for (int i = 0; i < kFaStages; ++i) { fa_mbar_init(&kv_full[i], 1); fa_mbar_init(&kv_empty[i], 1); }
         fa_mbar_init(&s_ready[0], 1); fa_mbar_init(&s_ready[1], 1);
-        fa_mbar_init(&p_ready, 4); fa_mbar_init(&o_ready, 1);
+        fa_mbar_init(&p_ready, 8); fa_mbar_init(&o_ready, 1);
         dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 4) {
+    if (warp == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
                      "r"(kFaTmemCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
@@ -184,7 +196,7 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
     const int n_units = p.step[H_PF_ITEMS] * p.nkv;
 
-    if (warp == 4) {
+    if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t g = 0;                                          // K/V tiles requested so far (ring position)
@@ -229,7 +241,7 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (!ok) { dead = 1; atomicOr(p.err, kErrTimeout); }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             uint32_t g = 0;                                          // K/V tiles consumed so far
@@ -281,58 +293,61 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         }
     } else {
         // ------------------------------------------------------------------ softmax warps
-        const int r = warp * 32 + lane;                              // row of the tile = TMEM lane
+        const int quarter = warp & 3, half = warp >> 2;
+        const int r = quarter * 32 + lane;                           // row of the tile = TMEM lane
         const int q_tok = r >> 3, head = r & 7;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+        constexpr int SC = kFaKv / 2, OC = kFaD / 2;                 // score and output columns of this thread
         uint32_t g = 0;
         for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
             const FaUnit c = fa_unit(p, u);
             // keys visible to this row's query; rows past the block's last token are computed but never stored
             const int my_len = min(c.len, c.len - (c.nq_blk - 1 - q_tok));
-            float o[kFaD];
+            float o[OC];
 #pragma unroll
-            for (int i = 0; i < kFaD; ++i) o[i] = 0.f;
-            float m_run = -INFINITY, l_run = 0.f;
-            bool alive = true;
+            for (int i = 0; i < OC; ++i) o[i] = 0.f;
+            float m_run = -INFINITY, l_run = 0.f;                    // l_run: sum over this thread's columns only
+            // No early exit from these loops: the eight warps meet at a named barrier in every tile, so a
+            // warp must never leave while others still go there.  After a wait has given up (`dead`),
+            // the remaining iterations run without waiting (their results are garbage and the status
+            // word says so).
             for (int j = 0; j < c.n_tiles; ++j, ++g) {
                 if (lane == 0 && !dead && !fa_wait(&s_ready[g & 1], (g >> 1) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); }
                 __syncwarp();
-                alive = __all_sync(0xffffffffu, !dead);
-                if (!alive) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                // scores of this row: 64 columns of the S buffer
-                const int kv0 = j * kFaKv;
-                float sv[kFaKv];
+                // this thread's 32 scores of the row
+                const int kv0 = j * kFaKv + half * SC;
+                float sv[SC];
                 float mx = -INFINITY;
-#pragma unroll
-                for (int cb = 0; cb < kFaKv; cb += 32) {
+                {
                     uint32_t v[32];
-                    fa_ld32(lane_base + (g & 1) * kFaKv + cb, v);
+                    fa_ld32(lane_base + (g & 1) * kFaKv + half * SC, v);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float s = kv0 + cb + i < my_len ? __uint_as_float(v[i]) * p.scale_log2 : -INFINITY;
-                        sv[cb + i] = s;
-                        mx = fmaxf(mx, s);
+                    for (int i = 0; i < SC; ++i) {
+                        sv[i] = kv0 + i < my_len ? __uint_as_float(v[i]) * p.scale_log2 : -INFINITY;
+                        mx = fmaxf(mx, sv[i]);
                     }
                 }
-                const float m_new = fmaxf(m_run, mx);
-                const float m_use = m_new == -INFINITY ? 0.f : m_new;     // rows past the block see nothing at all
-                const float alpha = exp2f(m_run - m_use);
+                xmax[g & 1][half][r] = mx;
+                asm volatile("bar.sync 1, %0;" ::"n"(kFaSoftmaxThreads) : "memory");
+                const float m_new = fmaxf(m_run, fmaxf(mx, xmax[g & 1][half ^ 1][r]));
+                const float m_use = m_new == -INFINITY ? 0.f : m_new;
+                const float alpha = fa_exp2(m_run - m_use);
                 float sum = 0.f;
                 // P as (hi, lo) bf16 planes, K-major with the 128-byte swizzle: 16-byte chunk c of row r
                 // sits at r * 128 + ((c ^ (r & 7)) << 4)
                 unsigned char* prow = p_smem + r * 128;
 #pragma unroll
-                for (int ch = 0; ch < kFaKv / 8; ++ch) {
+                for (int ch = 0; ch < SC / 8; ++ch) {
                     uint32_t hi[4], lo[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        const float a = exp2f(sv[ch * 8 + 2 * q] - m_use), b2 = exp2f(sv[ch * 8 + 2 * q + 1] - m_use);
+                        const float a = fa_exp2(sv[ch * 8 + 2 * q] - m_use), b2 = fa_exp2(sv[ch * 8 + 2 * q + 1] - m_use);
                         sum += a + b2;
                         hi[q] = pack_bf16(a, b2);
                         lo[q] = pack_bf16(a - bf16_lo(hi[q]), b2 - bf16_hi(hi[q]));
                     }
-                    const int sw = (ch ^ (r & 7)) << 4;
+                    const int sw = ((half * (SC / 8) + ch) ^ (r & 7)) << 4;
                     *reinterpret_cast<uint4*>(prow + sw) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
                     *reinterpret_cast<uint4*>(prow + kFaPTile + sw) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 }
@@ -340,10 +355,10 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 m_run = m_new;
                 // the last tile may reach past the request's tokens: those value rows hold whatever the page
                 // holds, and 0 * NaN is NaN, so they are cleared (whole rows: the swizzle permutes within a row)
-                const int n_valid = min(kFaKv, c.len - kv0);
+                const int n_valid = min(kFaKv, c.len - j * kFaKv);
                 if (n_valid < kFaKv) {
                     unsigned char* vt = kv_smem + (size_t)(g % kFaStages) * kFaStageBytes + 2 * kFaHalf;
-                    for (int i = r; i < (kFaKv - n_valid) * 16; i += kFaRows) {
+                    for (int i = tid; i < (kFaKv - n_valid) * 16; i += kFaSoftmaxThreads) {
                         const int row = n_valid + (i >> 4), piece = i & 15;
                         *reinterpret_cast<uint4*>(vt + (piece >> 3) * kFaHalf + row * 128 + (piece & 7) * 16) = make_uint4(0, 0, 0, 0);
                     }
@@ -354,26 +369,28 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) fa_arrive(&p_ready);
-                // O_tile = P V of this tile
+                // O_tile = P V of this tile: this thread's 64 columns
                 if (lane == 0 && !dead && !fa_wait(&o_ready, g & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); }
                 __syncwarp();
-                alive = __all_sync(0xffffffffu, !dead);
-                if (!alive) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-                for (int cb = 0; cb < kFaD; cb += 32) {
+                for (int cb = 0; cb < OC; cb += 32) {
                     uint32_t v[32];
-                    fa_ld32(lane_base + 128 + cb, v);
+                    fa_ld32(lane_base + 128 + half * OC + cb, v);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) o[cb + i] = fmaf(o[cb + i], alpha, __uint_as_float(v[i]));
                 }
             }
-            if (!alive) break;
+            // the row's sum: both threads of the row saw the same sequence of maxima, so their sums add
+            xsum[half][r] = l_run;
+            asm volatile("bar.sync 1, %0;" ::"n"(kFaSoftmaxThreads) : "memory");
+            const float l_row = l_run + xsum[half ^ 1][r];
             if (q_tok < c.nq_blk) {
-                const float inv = 1.f / l_run;
-                __nv_bfloat16* dst = p.o_out + (size_t)(c.row0 + q_tok) * 2 * p.nq * kFaD + (size_t)(c.hk * kFaHeads + head) * kFaD;
+                const float inv = 1.f / l_row;
+                __nv_bfloat16* dst = p.o_out + (size_t)(c.row0 + q_tok) * 2 * p.nq * kFaD + (size_t)(c.hk * kFaHeads + head) * kFaD +
+                                     half * OC;
 #pragma unroll
-                for (int i = 0; i < kFaD; i += 8) {
+                for (int i = 0; i < OC; i += 8) {
                     uint32_t hi[4], lo[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
@@ -389,7 +406,7 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
     __syncthreads();
-    if (warp == 4) {
+    if (warp == 8) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kFaTmemCols));
     }
