@@ -34,16 +34,18 @@ constexpr int kFaHeads = 8;                // query heads per KV head
 constexpr int kFaRows = kFaQ * kFaHeads;   // 128 rows of the MMA tile
 constexpr int kFaD = 128;
 constexpr int kFaKv = 64;                  // cached tokens per tile
-constexpr int kFaStages = 3;
+constexpr int kFaKStages = 2;               // K tiles in flight (free as soon as S is computed)
+constexpr int kFaVStages = 3;               // V tiles in flight (free after P V)
 constexpr int kFaQTile = kFaRows * 128;    // one (plane, half) tile of Q: 128 rows x 128 B = 16 KB
 constexpr int kFaQBytes = 4 * kFaQTile;    // hi/lo x two halves of head_dim
 constexpr int kFaPTile = kFaRows * 128;    // one plane of P: 128 rows x 64 tokens bf16
 constexpr int kFaHalf = kFaKv * 128;       // one 64-wide half of a K or V tile: 64 tokens x 128 B = 8 KB
-constexpr int kFaStageBytes = 4 * kFaHalf; // K halves, V halves
-constexpr int kFaSmem = kFaQBytes + 2 * kFaPTile + kFaStages * kFaStageBytes;
+constexpr int kFaTile = 2 * kFaHalf;        // a K or a V tile: two halves
+constexpr int kFaPBuf = 2 * kFaPTile;       // hi and lo planes of P
+constexpr int kFaSmem = kFaQBytes + 2 * kFaPBuf + (kFaKStages + kFaVStages) * kFaTile;
 constexpr int kFaThreads = 320;             // 8 softmax warps, producer warp, MMA warp
 constexpr int kFaSoftmaxThreads = 256;
-constexpr int kFaTmemCols = 256;           // S buffers at columns 0 and 64, O_tile at 128..255
+constexpr int kFaTmemCols = 512;           // S buffers at columns 0 and 64, O_tile buffers at 128 and 256
 constexpr uint32_t kFaSpin = 1u << 22;
 
 struct FaParams {
@@ -165,9 +167,11 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     extern __shared__ unsigned char fa_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)fa_raw + 1023) & ~(uintptr_t)1023);
     unsigned char* q_smem = smem;                                   // [plane][half][128 rows][128 B]
-    unsigned char* p_smem = smem + kFaQBytes;                       // [plane][128 rows][128 B]
-    unsigned char* kv_smem = p_smem + 2 * kFaPTile;                 // [stage][K half 0, K half 1, V half 0, V half 1]
-    __shared__ __align__(8) uint64_t q_full, q_free, kv_full[kFaStages], kv_empty[kFaStages], s_ready[2], p_ready, o_ready;
+    unsigned char* p_smem = smem + kFaQBytes;                       // [buffer][plane][128 rows][128 B]
+    unsigned char* k_smem = p_smem + 2 * kFaPBuf;                   // [stage][half][64 tokens][128 B]
+    unsigned char* v_smem = k_smem + kFaKStages * kFaTile;          // [stage][half][64 tokens][128 B]
+    __shared__ __align__(8) uint64_t q_full, q_free, k_full[kFaKStages], k_empty[kFaKStages], v_full[kFaVStages],
+        v_empty[kFaVStages], s_ready[2], p_ready[2], o_ready[2];
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int dead;
     __shared__ float xmax[2][2][kFaRows];                            // [tile parity][column half][row]
@@ -176,9 +180,9 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
     if (tid == 0) {
         fa_mbar_init(&q_full, 1); fa_mbar_init(&q_free, 1);
-        for (int i = 0; i < kFaStages; ++i) { fa_mbar_init(&kv_full[i], 1); fa_mbar_init(&kv_empty[i], 1); }
-        fa_mbar_init(&s_ready[0], 1); fa_mbar_init(&s_ready[1], 1);
-        fa_mbar_init(&p_ready, 8); fa_mbar_init(&o_ready, 1);
+        for (int i = 0; i < kFaKStages; ++i) { fa_mbar_init(&k_full[i], 1); fa_mbar_init(&k_empty[i], 1); }
+        for (int i = 0; i < kFaVStages; ++i) { fa_mbar_init(&v_full[i], 1); fa_mbar_init(&v_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { fa_mbar_init(&s_ready[i], 1); fa_mbar_init(&p_ready[i], 8); fa_mbar_init(&o_ready[i], 1); }
         dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -199,35 +203,39 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t g = 0;                                          // K/V tiles requested so far (ring position)
+            uint32_t g = 0;                                          // tiles requested so far (ring positions)
             int local = 0;
             for (int u = blockIdx.x; u < n_units && !dead; u += gridDim.x, ++local) {
                 const FaUnit c = fa_unit(p, u);
-                auto load_kv = [&](int j) -> bool {
-                    const int s = g % kFaStages;
-                    if (!fa_wait(&kv_empty[s], ((g / kFaStages) & 1) ^ 1)) return false;
-                    unsigned char* st = kv_smem + (size_t)s * kFaStageBytes;
+                // tile j of this unit: K into its ring, V into its ring (separate lifetimes: K is free once
+                // S is computed, V only after P V)
+                auto load_tile = [&](int j) -> bool {
+                    const int ks = g % kFaKStages, vs = g % kFaVStages;
+                    if (!fa_wait(&k_empty[ks], ((g / kFaKStages) & 1) ^ 1)) return false;
+                    if (!fa_wait(&v_empty[vs], ((g / kFaVStages) & 1) ^ 1)) return false;
+                    unsigned char* kd = k_smem + (size_t)ks * kFaTile;
+                    unsigned char* vd = v_smem + (size_t)vs * kFaTile;
                     const int n_valid = min(kFaKv, c.len - j * kFaKv);
                     const int n_boxes = (n_valid + p.box_rows - 1) / p.box_rows;
-                    fa_expect_tx(&kv_full[s], (uint32_t)(n_boxes * p.box_rows * 128 * 4));
+                    fa_expect_tx(&k_full[ks], (uint32_t)(n_boxes * p.box_rows * 128 * 2));
+                    fa_expect_tx(&v_full[vs], (uint32_t)(n_boxes * p.box_rows * 128 * 2));
                     for (int bi = 0; bi < n_boxes; ++bi) {
                         const int tok = j * kFaKv + bi * p.box_rows;
                         const int page = c.bt[tok / p.page_size];
                         const int y = (((p.layer * p.n_pages + page) * p.nkv + c.hk) * p.page_size) + tok % p.page_size;
                         const int off = bi * p.box_rows * 128;
 #pragma unroll
-                        for (int hf = 0; hf < 2; ++hf) {
-                            fa_tma_2d(st + hf * kFaHalf + off, &tm_k, hf * 64, y, &kv_full[s]);
-                            fa_tma_2d(st + (2 + hf) * kFaHalf + off, &tm_v, hf * 64, y, &kv_full[s]);
-                        }
+                        for (int hf = 0; hf < 2; ++hf) fa_tma_2d(kd + hf * kFaHalf + off, &tm_k, hf * 64, y, &k_full[ks]);
+#pragma unroll
+                        for (int hf = 0; hf < 2; ++hf) fa_tma_2d(vd + hf * kFaHalf + off, &tm_v, hf * 64, y, &v_full[vs]);
                     }
                     ++g;
                     return true;
                 };
-                // the first K/V tiles may be requested while the previous unit still uses the Q tile
-                const int early = min(c.n_tiles, kFaStages - 1);
+                // the first tiles may be requested while the previous unit still uses the Q tile
+                const int early = min(c.n_tiles, kFaKStages);
                 bool ok = true;
-                for (int j = 0; j < early && ok; ++j) ok = load_kv(j);
+                for (int j = 0; j < early && ok; ++j) ok = load_tile(j);
                 if (ok) ok = fa_wait(&q_free, (local & 1) ^ 1);
                 if (ok) {
                     fa_expect_tx(&q_full, kFaQBytes);
@@ -237,21 +245,24 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         for (int hf = 0; hf < 2; ++hf)
                             fa_tma_4d(q_smem + (pl * 2 + hf) * kFaQTile, &tm_q, hf * 64, c.hk * kFaHeads, pl, c.row0, &q_full);
                 }
-                for (int j = early; j < c.n_tiles && ok; ++j) ok = load_kv(j);
+                for (int j = early; j < c.n_tiles && ok; ++j) ok = load_tile(j);
                 if (!ok) { dead = 1; atomicOr(p.err, kErrTimeout); }
             }
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------------ MMA issuer
+        // Order on the tensor pipe: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...: S runs one tile ahead of
+        // the softmax, so that the softmax warps never wait for scores, and P V of tile g overlaps the
+        // softmax of tile g + 1 (P and O_tile are double-buffered).
         if (lane == 0) {
-            uint32_t g = 0;                                          // K/V tiles consumed so far
+            uint32_t g = 0;                                          // tiles consumed so far
             int local = 0;
             const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem);
             auto issue_s = [&](uint32_t gi) -> bool {                // S(gi) = Q K^T into S buffer gi & 1
-                const int s = gi % kFaStages;
-                if (!fa_wait(&kv_full[s], (gi / kFaStages) & 1)) return false;
+                const int ks = gi % kFaKStages;
+                if (!fa_wait(&k_full[ks], (gi / kFaKStages) & 1)) return false;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t k_addr = smem_u32(kv_smem + (size_t)s * kFaStageBytes);
+                const uint32_t k_addr = smem_u32(k_smem + (size_t)ks * kFaTile);
                 const uint32_t acc = tmem + (gi & 1) * kFaKv;
 #pragma unroll
                 for (int pl = 0; pl < 2; ++pl)
@@ -263,29 +274,31 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         for (int kk = 0; kk < 4; ++kk) fa_mma(acc, da + 2 * kk, db + 2 * kk, kFaIdescS, (pl | hf | kk) != 0);
                     }
                 fa_commit(&s_ready[gi & 1]);
+                fa_commit(&k_empty[ks]);                             // the K tile is free once these MMAs retire
                 return true;
             };
             for (int u = blockIdx.x; u < n_units && !dead; u += gridDim.x, ++local) {
                 const FaUnit c = fa_unit(p, u);
                 bool ok = fa_wait(&q_full, local & 1);
                 if (ok) ok = issue_s(g);
+                if (ok && c.n_tiles > 1) ok = issue_s(g + 1);
                 for (int j = 0; j < c.n_tiles && ok; ++j, ++g) {
-                    ok = fa_wait(&p_ready, g & 1);
+                    const int vs = g % kFaVStages;
+                    ok = fa_wait(&p_ready[g & 1], (g >> 1) & 1) && fa_wait(&v_full[vs], (g / kFaVStages) & 1);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const int s = g % kFaStages;
-                    const uint32_t v_addr = smem_u32(kv_smem + (size_t)s * kFaStageBytes + 2 * kFaHalf);
-                    const uint64_t dv = fa_desc_mnmajor(v_addr, kFaHalf);
+                    const uint64_t dv = fa_desc_mnmajor(smem_u32(v_smem + (size_t)vs * kFaTile), kFaHalf);
+                    const uint32_t acc = tmem + 128 + (g & 1) * kFaD;
 #pragma unroll
                     for (int pl = 0; pl < 2; ++pl) {
-                        const uint64_t dp = fa_desc_kmajor(p_addr + pl * kFaPTile);
+                        const uint64_t dp = fa_desc_kmajor(p_addr + (g & 1) * kFaPBuf + pl * kFaPTile);
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)     // 16 tokens per step: 32 B along a P row, 2048 B down the V tile
-                            fa_mma(tmem + 128, dp + 2 * kk, dv + 128 * kk, kFaIdescO, (pl | kk) != 0);
+                            fa_mma(acc, dp + 2 * kk, dv + 128 * kk, kFaIdescO, (pl | kk) != 0);
                     }
-                    fa_commit(&o_ready);
-                    fa_commit(&kv_empty[s]);
-                    if (j + 1 < c.n_tiles) ok = issue_s(g + 1);
+                    fa_commit(&o_ready[g & 1]);
+                    fa_commit(&v_empty[vs]);
+                    if (j + 2 < c.n_tiles) ok = issue_s(g + 2);
                 }
                 if (!ok) { dead = 1; atomicOr(p.err, kErrTimeout); break; }
                 fa_commit(&q_free);                                  // every MMA that reads this unit's Q has been issued
@@ -307,6 +320,21 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
             for (int i = 0; i < OC; ++i) o[i] = 0.f;
             float m_run = -INFINITY, l_run = 0.f;                    // l_run: sum over this thread's columns only
+            float alpha_prev = 0.f;                                  // rescale factor of the tile whose O_tile is still to be added
+            // adds O_tile of tile gt (its P V has been issued) into the output registers
+            auto accumulate = [&](uint32_t gt, float alpha) {
+                if (lane == 0 && !dead && !fa_wait(&o_ready[gt & 1], (gt >> 1) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); }
+                __syncwarp();
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                for (int cb = 0; cb < OC; cb += 32) {
+                    uint32_t v[32];
+                    fa_ld32(lane_base + 128 + (gt & 1) * kFaD + half * OC + cb, v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[cb + i] = fmaf(o[cb + i], alpha, __uint_as_float(v[i]));
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            };
             // No early exit from these loops: the eight warps meet at a named barrier in every tile, so a
             // warp must never leave while others still go there.  After a wait has given up (`dead`),
             // the remaining iterations run without waiting (their results are garbage and the status
@@ -335,8 +363,9 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const float alpha = fa_exp2(m_run - m_use);
                 float sum = 0.f;
                 // P as (hi, lo) bf16 planes, K-major with the 128-byte swizzle: 16-byte chunk c of row r
-                // sits at r * 128 + ((c ^ (r & 7)) << 4)
-                unsigned char* prow = p_smem + r * 128;
+                // sits at r * 128 + ((c ^ (r & 7)) << 4).  Buffer g & 1: P V of tile g - 2, which read it
+                // last, was waited for before tile g - 1's softmax.
+                unsigned char* prow = p_smem + (g & 1) * kFaPBuf + r * 128;
 #pragma unroll
                 for (int ch = 0; ch < SC / 8; ++ch) {
                     uint32_t hi[4], lo[4];
@@ -357,30 +386,26 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 // holds, and 0 * NaN is NaN, so they are cleared (whole rows: the swizzle permutes within a row)
                 const int n_valid = min(kFaKv, c.len - j * kFaKv);
                 if (n_valid < kFaKv) {
-                    unsigned char* vt = kv_smem + (size_t)(g % kFaStages) * kFaStageBytes + 2 * kFaHalf;
+                    const int vs = g % kFaVStages;
+                    if (lane == 0 && !dead && !fa_wait(&v_full[vs], (g / kFaVStages) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); }
+                    __syncwarp();
+                    unsigned char* vt = v_smem + (size_t)vs * kFaTile;
                     for (int i = tid; i < (kFaKv - n_valid) * 16; i += kFaSoftmaxThreads) {
                         const int row = n_valid + (i >> 4), piece = i & 15;
                         *reinterpret_cast<uint4*>(vt + (piece >> 3) * kFaHalf + row * 128 + (piece & 7) * 16) = make_uint4(0, 0, 0, 0);
                     }
                 }
-                // P (and the cleared rows) must be visible to the tensor core's reads; the S buffer and
-                // the previous O_tile have been read: hand over to the MMA lane
+                // P (and the cleared rows) must be visible to the tensor core's reads; the S buffer has
+                // been read: hand over to the MMA lane
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
-                if (lane == 0) fa_arrive(&p_ready);
-                // O_tile = P V of this tile: this thread's 64 columns
-                if (lane == 0 && !dead && !fa_wait(&o_ready, g & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); }
-                __syncwarp();
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-                for (int cb = 0; cb < OC; cb += 32) {
-                    uint32_t v[32];
-                    fa_ld32(lane_base + 128 + half * OC + cb, v);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o[cb + i] = fmaf(o[cb + i], alpha, __uint_as_float(v[i]));
-                }
+                if (lane == 0) fa_arrive(&p_ready[g & 1]);
+                // while P V of this tile runs, add the previous tile's O_tile
+                if (j > 0) accumulate(g - 1, alpha_prev);
+                alpha_prev = alpha;
             }
+            accumulate(g - 1, alpha_prev);
             // the row's sum: both threads of the row saw the same sequence of maxima, so their sums add
             xsum[half][r] = l_run;
             asm volatile("bar.sync 1, %0;" ::"n"(kFaSoftmaxThreads) : "memory");
