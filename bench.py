@@ -38,9 +38,9 @@ UNIT = "tokens/s"
 PEAKS_FALLBACK = dict(hbm_gbs=6650.0, source="fallback")
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of the captured launch, per kernel class.
 # Set an entry to None (or delete it) when that kernel changes after the capture.
-NCU_TRAFFIC_RATIO = {"attn": (1206.095e6 + 8.407e6) / 1201.844e6,     # attn_decode_kernel<128>, 586 166 cached tokens
-                     "gate_up": (795.326e6 + 5.083e6) / 786.432e6,      # expert_gate_up_kernel, 125 experts
-                     "down": (397.982e6 + 5.032e6) / 393.216e6}         # expert_down_kernel
+NCU_TRAFFIC_RATIO = {"attn": (1206.248e6 + 7.596e6) / 1201.844e6,     # attn_decode_kernel<128>, 586 166 cached tokens
+                     "gate_up": (795.297e6 + 5.104e6) / 786.432e6,      # expert_gate_up_kernel, 125 experts
+                     "down": (397.981e6 + 5.244e6) / 393.216e6}         # expert_down_kernel
 
 
 def load_peaks() -> dict:
@@ -136,7 +136,9 @@ class DecodeWorkload:
         torch.cuda.synchronize(device)
         self.setup_s = time.time() - t0
         self.pages = wl.make_page_assignment(cap, ps, n_pages, seed=seed)
-        self.model = binding.Model(model, self.weights, max_decode_seqs=B, max_prefill_tokens=prefill_reqs * prefill_chunk,
+        # a fused mixed step carries the decode rows and the prompt rows in one call
+        self.model = binding.Model(model, self.weights, max_decode_seqs=B + prefill_reqs,
+                                   max_prefill_tokens=prefill_reqs * prefill_chunk + (B if prefill_reqs else 0),
                                    max_pos=max(cap + [prefill_chunk]) + 8)
         self.kv = binding.KvCache(self.model, self.k_pool, self.v_pool, ps, B + prefill_reqs, max_pages)
         for b in range(B):
@@ -264,7 +266,7 @@ def run_reference(args):
 def run_mixed(args):
     """Config 4: one chunked-prefill call (8 fresh prompts of 2048 tokens) followed by one decode step
     over 192 sequences = one mixed step.  Prints decode-only against the HBM roofline, prefill-only
-    against the bf16 tensor peak, and the pair."""
+    against the bf16 tensor peak, the pair, and the same work as one fused call (mars_mixed_step)."""
     from paper_2511_11373_b200 import binding
     device = torch.device("cuda", 0)
     torch.cuda.set_device(device)
@@ -297,6 +299,25 @@ def run_mixed(args):
             w.kv.seq_release(s_)
         if it >= args.warmup:
             t_pf.append(ev[0].elapsed_time(ev[1])); t_dec.append(ev[1].elapsed_time(ev[2]))
+    # the same work as ONE call: decode rows and prompt chunks share every projection and every expert pass
+    mix_t = torch.empty(w.B + pf["requests"], dtype=torch.int32, device=device)
+    mix_l = torch.empty(w.B + pf["requests"], dtype=torch.float32, device=device)
+    t_fused = []
+    for it in range(args.warmup + args.steps):
+        for s_ in ids:
+            w.kv.seq_reserve(s_, 0)
+        ev[0].record(stream)
+        st = binding.mars_mixed_step(w.model, w.kv, w.ids, w.tok_a, ids, [pf["chunk"]] * pf["requests"], toks,
+                                     [1] * pf["requests"], smp, mix_t, mix_l)
+        assert st == 0, binding.STATUS_NAMES.get(st, st)
+        ev[1].record(stream)
+        torch.cuda.synchronize()
+        assert w.model.poll_status() == 0
+        for s_ in ids:
+            w.kv.seq_release(s_)
+        if it >= args.warmup:
+            t_fused.append(ev[0].elapsed_time(ev[1]))
+    fused_ms = statistics.median(t_fused)
     # per-kernel-class device time of one more prefill call
     for s_ in ids:
         w.kv.seq_reserve(s_, 0)
@@ -326,7 +347,7 @@ def run_mixed(args):
                 prefill=dict(ms=pf_ms, tokens_per_s=n_pf / (pf_ms / 1e3), algorithmic_tflop=flops / 1e12,
                              achieved_tflops=flops / (pf_ms * 1e-3) / 1e12, frac_of_measured_bf16=flops / (pf_ms * 1e-3) / 1e12 / tflops_peak,
                              note="activations are (hi, lo) bf16 pairs: the tensor cores execute twice the algorithmic flops in the projections"),
-                mixed_ms=pf_ms + dec_ms, prefill_ms_by_class=pf_classes)
+                mixed_ms=pf_ms + dec_ms, fused_mixed_step_ms=fused_ms, prefill_ms_by_class=pf_classes)
     print(json.dumps(line))
 
 
