@@ -76,8 +76,9 @@ int launch_fattn_prefill(const Shape& s, const Buffers& b, const StepLayout& lay
                          cudaStream_t st);
 int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st);
 
+// o_ksplit: number of split-K partials of the output projection that the router kernel adds to the residual.
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,
-                  int group_cap, cudaStream_t st);
+                  int group_cap, int o_ksplit, cudaStream_t st);
 
 // Prefill-sized contractions on tcgen05: out[m][n_cols] = A[m][2][K] (hi + lo planes) . B[n_cols][K]^T, and
 // the grouped expert pair (gather rows to slot order, gate/up + SwiGLU, down) over the group list.
@@ -86,7 +87,9 @@ int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, 
                         cudaStream_t st);
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
                       int32_t* err, cudaStream_t st);
-// Decode-sized projection on tcgen05 with swapped operands: out[split][t][row], t < n_tok <= 64.
+// Decode-sized projection on tcgen05 with swapped operands: out[split][t][row], t < n_tok <= umma_swap_max_tokens().
+int umma_swap_max_tokens();
+int umma_swap_splits(int rows, int n_tok, int K);
 int launch_umma_swap(const CUtensorMap& tm_w, const CUtensorMap& tm_x, int rows, int n_tok, int K, int splits, float* out,
                      int32_t* err, cudaStream_t st);
 int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_xperm, const CUtensorMap& tm_wgu,

@@ -593,9 +593,7 @@ static void expert_plan(const Shape& s, int n_tok, int* cap, int* warps) {
 
 // ---------------------------------------------------------------------------------------------
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,
-                  int group_cap, cudaStream_t st) {
-    int ks, o_ksplit, phases;
-    gemm_plan(s.nq * s.D, n_tok, false, &ks, &o_ksplit, &phases);
+                  int group_cap, int o_ksplit, cudaStream_t st) {
     launch_chained(router_kernel, dim3(n_tok), dim3(kRouterCta), 8 * x_row_bytes(s.H), st, s, b, w.mlp_norm, w.router, dbg, layer, n_tok,
                                                                        o_ksplit);
     int cap, warps;

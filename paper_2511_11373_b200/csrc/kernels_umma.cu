@@ -23,6 +23,8 @@
 
 namespace mars {
 
+static int g_umma_sms = 0;     // SMs of the device (set by init_umma_kernels)
+
 constexpr int kUmStages = 3;
 constexpr int kUmTileM = 128, kUmTileN = 256, kUmStageK = 64;
 constexpr int kUmTileBytes = kUmTileM * kUmStageK * 2;              // 16 KB: 128 rows x 128 B
@@ -350,18 +352,26 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 
 // ---------------------------------------------------------------------------------------------
 // Decode-sized dense projections (QKV, output projection, lm_head) on the same tensor cores with the
-// operands swapped: 128 WEIGHT rows sit on the TMEM lanes and up to 64 token columns on N, so the
-// kernel streams each weight once from HBM (TMA, 3-stage ring, two CTAs per SM) while the hi and lo activation planes
-// of the K range are re-read from L2.  With 64 tokens carried as (hi, lo) pairs these projections
+// operands swapped: 128 WEIGHT rows sit on the TMEM lanes and up to 256 token columns on N, so the
+// kernel streams each weight once from HBM (TMA ring; two CTAs per SM at <= 64 tokens) while the hi and
+// lo activation planes of the K range are re-read from L2.  With 64 tokens carried as (hi, lo) pairs these projections
 // are tensor-bound on the mma.sync path (128 columns per weight row); here they are HBM streams again.
 // gridDim.y splits K; every split writes an fp32 partial [split][token][row] that the consumer adds
 // in a fixed order.
-constexpr int kSwStages = 3;
-constexpr int kSwTok = 64;
+// NB = 1 .. 4 boxes of 64 token rows per activation plane: 64 .. 256 token columns per pass.
 constexpr int kSwABytes = 128 * kUmStageK * 2;                       // 16 KB of weights per stage
-constexpr int kSwBBytes = kSwTok * kUmStageK * 2;                    // 8 KB per activation plane
-constexpr int kSwStageBytes = kSwABytes + 2 * kSwBBytes;
-constexpr uint32_t kSwIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSwTok >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+constexpr int kSwBoxBytes = 64 * kUmStageK * 2;                      // 8 KB: one box of 64 token rows
+template <int NB>
+struct SwCfg {
+    static constexpr int kTok = 64 * NB;
+    static constexpr int kPlaneBytes = NB * kSwBoxBytes;
+    static constexpr int kStageBytes = kSwABytes + 2 * kPlaneBytes;
+    static constexpr int kStages = NB == 4 ? 2 : 3;                  // 96 / 144 / 192 / 160 KB of ring
+    static constexpr int kTmemCols = NB == 3 ? 256 : kTok;           // allocations are powers of two
+    static constexpr int kCtasPerSm = NB == 1 ? 2 : 1;
+    static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    static constexpr size_t smem_bytes() { return (size_t)kStages * kStageBytes + 1024; }
+};
 
 struct SwapParams {
     int rows, n_tok, k_per_split;      // weight rows, token columns (<= 64), K range of one split (multiple of 64)
@@ -369,8 +379,12 @@ struct SwapParams {
     int32_t* err;
 };
 
-__global__ void __launch_bounds__(kUmThreads, 2)
+template <int NB>
+__global__ void __launch_bounds__(kUmThreads, SwCfg<NB>::kCtasPerSm)
 umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, SwapParams p) {
+    constexpr int kSwStages = SwCfg<NB>::kStages, kSwTok = SwCfg<NB>::kTok, kSwStageBytes = SwCfg<NB>::kStageBytes;
+    constexpr int kSwBBytes = SwCfg<NB>::kPlaneBytes;
+    constexpr uint32_t kSwIdesc = SwCfg<NB>::kIdesc;
     extern __shared__ unsigned char um_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)um_raw + 1023) & ~(uintptr_t)1023);
     __shared__ __align__(8) uint64_t full_bar[kSwStages], empty_bar[kSwStages], accum_bar;
@@ -389,7 +403,7 @@ umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
     }
     if (warp == 2) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
-                     "r"(kSwTok));
+                     "r"(SwCfg<NB>::kTmemCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
@@ -413,8 +427,11 @@ umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
             for (int ks = 0; ks < pre; ++ks) {
                 unsigned char* st = smem + (size_t)ks * kSwStageBytes;
                 const int k = k0 + ks * kUmStageK;
-                um_tma_3d(st + kSwABytes, &tm_x, k, 0, 0, &full_bar[ks]);
-                um_tma_3d(st + kSwABytes + kSwBBytes, &tm_x, k, 1, 0, &full_bar[ks]);
+#pragma unroll
+                for (int bx = 0; bx < NB; ++bx) {
+                    um_tma_3d(st + kSwABytes + bx * kSwBoxBytes, &tm_x, k, 0, 64 * bx, &full_bar[ks]);
+                    um_tma_3d(st + kSwABytes + kSwBBytes + bx * kSwBoxBytes, &tm_x, k, 1, 64 * bx, &full_bar[ks]);
+                }
             }
             for (int ks = pre; ks < nk && !dead; ++ks) {
                 const int s = ks % kSwStages;
@@ -426,8 +443,11 @@ umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
                 um_expect_tx(&full_bar[s], kSwStageBytes);
                 um_tma_2d(st, &tm_w, k, row0, &full_bar[s]);
                 um_tma_2d(st + 8192, &tm_w, k, row0 + 64, &full_bar[s]);
-                um_tma_3d(st + kSwABytes, &tm_x, k, 0, 0, &full_bar[s]);
-                um_tma_3d(st + kSwABytes + kSwBBytes, &tm_x, k, 1, 0, &full_bar[s]);
+#pragma unroll
+                for (int bx = 0; bx < NB; ++bx) {
+                    um_tma_3d(st + kSwABytes + bx * kSwBoxBytes, &tm_x, k, 0, 64 * bx, &full_bar[s]);
+                    um_tma_3d(st + kSwABytes + kSwBBytes + bx * kSwBoxBytes, &tm_x, k, 1, 64 * bx, &full_bar[s]);
+                }
             }
         }
     } else if (warp == 1) {
@@ -459,7 +479,7 @@ umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
             const uint32_t lane_base = tmem_d + ((uint32_t)(quarter * 32) << 16);
             float* out = p.out + (size_t)blockIdx.y * p.n_tok * p.rows;
 #pragma unroll 1
-            for (int c = 0; c < kSwTok; c += 32) {
+            for (int c = 0; c < kSwTok && c < p.n_tok; c += 32) {
                 uint32_t v[32];
                 um_ld32(lane_base + c, v);
                 if (row < p.rows) {
@@ -474,18 +494,37 @@ umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
     __syncthreads();
     if (warp == 2) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kSwTok));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(SwCfg<NB>::kTmemCols));
     }
 }
 
-static size_t swap_smem_bytes() { return (size_t)kSwStages * kSwStageBytes + 1024; }
-
-// out[split][t][row] for t < n_tok <= 64; K = splits * k_per_split.
+// out[split][t][row] for t < n_tok <= 256; K = splits * k_per_split.
 int launch_umma_swap(const CUtensorMap& tm_w, const CUtensorMap& tm_x, int rows, int n_tok, int K, int splits, float* out,
                      int32_t* err, cudaStream_t st) {
     SwapParams p{rows, n_tok, K / splits, out, err};
-    launch_chained(umma_swap_kernel, dim3((rows + 127) / 128, splits), dim3(kUmThreads), swap_smem_bytes(), st, tm_w, tm_x, p);
+    const dim3 grid((rows + 127) / 128, splits);
+    if (n_tok <= 64)
+        launch_chained(umma_swap_kernel<1>, grid, dim3(kUmThreads), SwCfg<1>::smem_bytes(), st, tm_w, tm_x, p);
+    else if (n_tok <= 128)
+        launch_chained(umma_swap_kernel<2>, grid, dim3(kUmThreads), SwCfg<2>::smem_bytes(), st, tm_w, tm_x, p);
+    else if (n_tok <= 192)
+        launch_chained(umma_swap_kernel<3>, grid, dim3(kUmThreads), SwCfg<3>::smem_bytes(), st, tm_w, tm_x, p);
+    else
+        launch_chained(umma_swap_kernel<4>, grid, dim3(kUmThreads), SwCfg<4>::smem_bytes(), st, tm_w, tm_x, p);
     return 1;
+}
+int umma_swap_max_tokens() { return 256; }
+
+// Number of K splits of a swap-AB projection: as many as divide the 64-wide K stages evenly (at least 8
+// stages each, at most K / 256 splits: the partial buffers are sized for that) while all CTAs still run
+// in one wave.
+int umma_swap_splits(int rows, int n_tok, int K) {
+    const int tiles = (rows + 127) / 128, stages = K / kUmStageK;
+    const int slots = g_umma_sms * (n_tok <= 64 ? 2 : 1);
+    int best = 1;
+    for (int s = 1; s <= K / 256; s *= 2)
+        if (stages % s == 0 && stages / s >= 8 && tiles * s <= slots) best = s;
+    return best;
 }
 
 // Rows of the normalised activations gathered into expert-slot order: xperm[slot] = h[slot_token[slot]]
@@ -502,7 +541,6 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(Buffers b, int H, int 
 static size_t umma_smem_bytes() { return (size_t)kUmStages * kUmStageBytes + 1024; }
 
 // Persistent grid: one CTA per SM, or fewer when there are fewer tiles.
-static int g_umma_sms = 0;
 static int umma_grid(int tiles) { return tiles < g_umma_sms ? (tiles < 1 ? 1 : tiles) : g_umma_sms; }
 
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
@@ -581,7 +619,13 @@ cudaError_t init_umma_kernels() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes());
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(umma_swap_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)swap_smem_bytes());
+    e = cudaFuncSetAttribute(umma_swap_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SwCfg<1>::smem_bytes());
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_swap_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SwCfg<2>::smem_bytes());
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_swap_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SwCfg<3>::smem_bytes());
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(umma_swap_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SwCfg<4>::smem_bytes());
 }
 
 }  // namespace mars

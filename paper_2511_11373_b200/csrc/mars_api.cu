@@ -98,8 +98,8 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
     t.x = (float*)take(n * H * 4);
     t.h = (__nv_bfloat16*)take(n * 2 * H * 2);
     // split-K partials: up to K/256 of them for decode-sized calls, one otherwise
-    const size_t n64 = n < 64 ? n : 64;
-    const size_t qkv_parts = std::max(n, n64 * (H / 256)), o_parts = std::max(n, n64 * (nq * D / 256));
+    const size_t n_sw = std::min<size_t>(n, (size_t)umma_swap_max_tokens());
+    const size_t qkv_parts = std::max(n, n_sw * (H / 256)), o_parts = std::max(n, n_sw * (nq * D / 256));
     t.qkv = (float*)take(qkv_parts * (nq + 2 * nkv) * D * 4);
     t.opart = (float*)take(o_parts * H * 4);
     t.q = (__nv_bfloat16*)take(n * 2 * nq * D * 2);
@@ -890,7 +890,12 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     run(MARS_K_OTHER, [&] {
         return launch_embed(s, b, lay, m->embed, plan.tokens_dev, m->layers[0].attn_norm, taps.hidden, n_tok, st);
     });
-    const bool umma = m->umma_ready && n_tok > kUmmaMinTokens;
+    // Three regimes by token rows: up to 64 and up to 256 rows are weight streams (swap-AB projections with
+    // 64 / 128 / 256 token columns, split-K partials, streaming expert kernels); beyond that the
+    // projections and the experts are dense contractions on 128 x 256 tensor-core tiles.
+    const bool umma = m->umma_ready && n_tok > umma_swap_max_tokens();
+    const int qkv_split = umma_swap_splits((s.nq + 2 * s.nkv) * s.D, n_tok, s.H);
+    const int o_split = umma_swap_splits(s.H, n_tok, s.nq * s.D);
     for (int l = 0; l < s.L; ++l) {
         const LayerW& w = m->layers[l];
         if (umma) {   // prefill-sized call: dense contractions on tcgen05 / TMEM
@@ -901,8 +906,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             });
         } else {      // decode-sized call: weights stream once through tcgen05 with the operands swapped
             run(MARS_K_QKV, [&] {
-                int ks, ksplit, phases;
-                gemm_plan(s.H, n_tok, false, &ks, &ksplit, &phases);
+                const int ksplit = qkv_split;
                 int n = launch_umma_swap(m->tm_wqkv[l], m->tm_h64, (s.nq + 2 * s.nkv) * s.D, n_tok, s.H, ksplit, b.qkv, b.err, st);
                 return n + launch_qkv_post(s, b, lay, w, kv->view, l, n_tok, ksplit, st);
             });
@@ -937,11 +941,9 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             });
         } else {
             run(MARS_K_OPROJ, [&] {
-                int ks, ksplit, phases;
-                gemm_plan(s.nq * s.D, n_tok, false, &ks, &ksplit, &phases);
-                return launch_umma_swap(m->tm_wo[l], m->tm_o64, s.H, n_tok, s.nq * s.D, ksplit, b.opart, b.err, st);
+                return launch_umma_swap(m->tm_wo[l], m->tm_o64, s.H, n_tok, s.nq * s.D, o_split, b.opart, b.err, st);
             });
-            run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, 0, st); });
+            run(MARS_K_ROUTER, [&] { return launch_router(s, b, w, taps, l, n_tok, 0, o_split, st); });
             run(MARS_K_GATE_UP, [&] { return launch_gate_up(s, b, w, n_tok, m->sm_count, st); });
             run(MARS_K_DOWN, [&] { return launch_down(s, b, w, n_tok, st); });
         }
@@ -952,9 +954,10 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     if (n_emit) {
         run(MARS_K_LM_HEAD, [&] {
             // decode: the emitting rows are the token rows in order, so the tensor maps over b.h apply
+            // (more token columns would make the swapped kernel re-read the activations once per 128 vocabulary rows)
             if (!plan.prefill && n_emit <= kUmmaMinTokens)
                 return launch_umma_swap(m->tm_lm, m->tm_h64, s.V, n_emit, s.H, 1, b.logits, b.err, st);
-            if (!plan.prefill && umma)
+            if (!plan.prefill && m->umma_ready)
                 return launch_umma_dense(m->tm_h, m->tm_lm, n_emit, s.V, s.H, b.logits, b.err, st);
             return launch_lm_head(s, b, lay, m->lm_head, n_emit, m->sm_count, st);
         });
@@ -1365,7 +1368,11 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
         launch_attention(s, buf, lay, view, tm_k, tm_v, l, sms, st);
         launch_attn_merge(s, buf, lay, n_seqs, st);
         launch_oproj(s, buf, lw, n_seqs, sms, st);
-        launch_router(s, buf, lw, taps, l, n_seqs, 0, st);
+        {
+            int ks, o_ksplit, phases;      // as launch_oproj plans it
+            gemm_plan(s.nq * s.D, n_seqs, false, &ks, &o_ksplit, &phases);
+            launch_router(s, buf, lw, taps, l, n_seqs, 0, o_ksplit, st);
+        }
         launch_gate_up(s, buf, lw, n_seqs, sms, st);
         launch_down(s, buf, lw, n_seqs, st);
         const __nv_bfloat16* next_gain =

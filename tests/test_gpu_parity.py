@@ -344,14 +344,16 @@ def test_prefill_in_two_calls_equals_one_call():
     assert (res[0][0] - res[1][0]).abs().max() < 1e-3 and res[0][1] == res[1][1]
 
 
-def test_decode_with_more_than_64_sequences():
-    """More than 64 decode rows switch the dense projections and the lm_head to the 128-row
-    tensor-core tiles (and the experts to grouped tiles); results must not change."""
+@pytest.mark.parametrize("n_seq", [70, 150, 256, 260])
+def test_decode_with_more_than_64_sequences(n_seq):
+    """65 to 256 decode rows keep the weight-streaming kernels (swap-AB projections with 128 or 256 token
+    columns, streaming experts with up to 16 tokens per group); beyond 256 rows the dense projections,
+    the lm_head and the experts move to the 128-row tensor-core tiles.  Results must not change."""
     model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=1)
-    ctx = [5 + 7 * i for i in range(70)]
+    ctx = [5 + (7 * i) % 300 for i in range(n_seq)]
     case = Case(model, 16, ctx, seed=31)
     tokens = wl.make_tokens(len(ctx), model["vocab"], seed=8)
     _, _, stats = run_and_compare(case, tokens, sampling=dict(greedy=0, temperature=0.85, top_p=0.95), step=3, seed=5,
-                                  label="decode-70")
-    print("decode-70", stats)
+                                  label=f"decode-{n_seq}")
+    print(f"decode-{n_seq}", stats)
     check_cache_append(case, ctx)
