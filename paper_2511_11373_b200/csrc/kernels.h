@@ -85,6 +85,23 @@ int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const Debug
 int launch_resid_norm(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int o_ksplit, cudaStream_t st);
 int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int group_cap,
                         cudaStream_t st);
+// The QKV projection with its post-processing in the epilogue of the contraction kernel.  A thread owns one
+// token row of a tile and, in it, whole heads (256 / head_dim of them): per-head RMS norm (optional),
+// rotary embedding at the token's position, then queries as (hi, lo) bf16 pairs into q_out
+// [token][2][nq * D] and keys / values rounded to bf16 into the token's page slot -- the fp32
+// projection never goes to memory.
+struct QkvEpilogue {
+    const int32_t* tok_pos;     // [m_rows]
+    const int32_t* tok_seq;     // [m_rows]
+    const int32_t* block_table; // [seqs][max_pages_per_seq]
+    const float2* rope;         // [m_rows][D / 2] (cos, sin)
+    const __nv_bfloat16 *q_gain, *k_gain;
+    __nv_bfloat16 *q_out, *k_pool, *v_pool;
+    int max_pages_per_seq, n_pages, page_size, layer, nq, nkv, head_dim, qk_norm;
+    float eps;
+};
+int launch_umma_qkv(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, const QkvEpilogue& ep,
+                    int32_t* err, cudaStream_t st);
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
                       int32_t* err, cudaStream_t st);
 // Decode-sized projection on tcgen05 with swapped operands: out[split][t][row], t < n_tok <= umma_swap_max_tokens().

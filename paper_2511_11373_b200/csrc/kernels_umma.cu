@@ -118,7 +118,8 @@ struct UmmaParams {
     int b_rows_per_expert;    // rows of B per expert (grouped calls)
     int n_cols;               // output columns (store mode) or expert_inter (SwiGLU mode)
     int swiglu;               // 0: out[m][n_cols] fp32; 1: act[m][2][n_cols] from (gate, up) column halves;
-                              // 2: per-row softmax statistics of the tile's columns (scoring pass, see below)
+                              // 2: per-row softmax statistics of the tile's columns (scoring pass, see below);
+                              // 3: QKV projection with norm, RoPE and the cache append in the epilogue
     float* out;               // mode 2: optional copy of the raw logits [m][n_cols], or null
     __nv_bfloat16* act;
     int32_t* err;
@@ -130,7 +131,74 @@ struct UmmaParams {
     float2* score_ml;
     float* score_tgt;
     int tiles_x;              // column tiles per row tile (mode 1: 128 output columns each, else 256)
+    QkvEpilogue qkv;          // mode 3: the tile's columns are whole heads of the QKV projection (kernels.h)
 };
+
+template <int D>
+__device__ __forceinline__ void qkv_head_epilogue(const QkvEpilogue& e, uint32_t taddr, int head, int t) {
+    constexpr int HALF = D / 2;
+    float v[D];
+#pragma unroll
+    for (int c = 0; c < D; c += 32) {
+        uint32_t raw[32];
+        um_ld32(taddr + c, raw);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[c + j] = __uint_as_float(raw[j]);
+    }
+    if (t < 0) return;                                    // row past the call's tokens: the loads above are warp-wide
+    const bool is_q = head < e.nq, is_k = !is_q && head < e.nq + e.nkv;
+    const int pos = e.tok_pos[t];
+    __nv_bfloat16* cache_row = nullptr;
+    if (!is_q) {
+        const int page = e.block_table[(size_t)e.tok_seq[t] * e.max_pages_per_seq + pos / e.page_size];
+        const int hk = is_k ? head - e.nq : head - e.nq - e.nkv;
+        cache_row = (is_k ? e.k_pool : e.v_pool) +
+                    ((((size_t)e.layer * e.n_pages + page) * e.nkv + hk) * e.page_size + pos % e.page_size) * D;
+    }
+    if (is_q || is_k) {
+        if (e.qk_norm) {
+            float ss = 0.f;
+#pragma unroll
+            for (int i = 0; i < D; ++i) ss += v[i] * v[i];
+            const float r = rsqrtf(ss / (float)D + e.eps);
+            const __nv_bfloat16* g = is_q ? e.q_gain : e.k_gain;
+#pragma unroll
+            for (int i = 0; i < D; i += 8) {
+                const uint4 gv = *reinterpret_cast<const uint4*>(g + i);
+                const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) { v[i + 2 * q] *= r * bf16_lo(gw[q]); v[i + 2 * q + 1] *= r * bf16_hi(gw[q]); }
+            }
+        }
+        const float2* cs = e.rope + (size_t)t * HALF;
+#pragma unroll
+        for (int i = 0; i < HALF; i += 2) {
+            const float4 c2 = *reinterpret_cast<const float4*>(cs + i);      // (cos, sin) of i and i + 1
+            const float a0 = v[i] * c2.x - v[i + HALF] * c2.y, b0 = v[i + HALF] * c2.x + v[i] * c2.y;
+            const float a1 = v[i + 1] * c2.z - v[i + 1 + HALF] * c2.w, b1 = v[i + 1 + HALF] * c2.z + v[i + 1] * c2.w;
+            v[i] = a0; v[i + HALF] = b0; v[i + 1] = a1; v[i + 1 + HALF] = b1;
+        }
+    }
+    if (is_q) {
+        __nv_bfloat16* dq = e.q_out + (size_t)t * 2 * e.nq * D + (size_t)head * D;
+#pragma unroll
+        for (int i = 0; i < D; i += 8) {
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                hi[q] = pack_bf16(v[i + 2 * q], v[i + 2 * q + 1]);
+                lo[q] = pack_bf16(v[i + 2 * q] - bf16_lo(hi[q]), v[i + 2 * q + 1] - bf16_hi(hi[q]));
+            }
+            *reinterpret_cast<uint4*>(dq + i) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(dq + (size_t)e.nq * D + i) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < D; i += 8)
+            *reinterpret_cast<uint4*>(cache_row + i) = make_uint4(pack_bf16(v[i], v[i + 1]), pack_bf16(v[i + 2], v[i + 3]),
+                                                                  pack_bf16(v[i + 4], v[i + 5]), pack_bf16(v[i + 6], v[i + 7]));
+    }
+}
 
 // The kernel is persistent: CTA c computes tiles c, c + gridDim.x, ... (column tile fastest, so that
 // CTAs running side by side share the row tile's activations and, for grouped calls, an expert's
@@ -268,6 +336,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                                     make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
                                                 __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
                     }
+                }
+            } else if (p.swiglu == 3) {
+                const QkvEpilogue& e = p.qkv;
+                const int t = r < m_valid ? m0 + r : -1;
+                const int n_heads = e.nq + 2 * e.nkv;
+                if (e.head_dim == 128) {
+#pragma unroll 1
+                    for (int hh = 0; hh < kUmTileN / 128; ++hh)
+                        if (col0 / 128 + hh < n_heads) qkv_head_epilogue<128>(e, lane_base + hh * 128, col0 / 128 + hh, t);
+                } else {
+#pragma unroll 1
+                    for (int hh = 0; hh < kUmTileN / 64; ++hh)
+                        if (col0 / 64 + hh < n_heads) qkv_head_epilogue<64>(e, lane_base + hh * 64, col0 / 64 + hh, t);
                 }
             } else if (p.swiglu == 2) {
                 const bool live = r < m_valid;
@@ -546,7 +627,16 @@ static int umma_grid(int tiles) { return tiles < g_umma_sms ? (tiles < 1 ? 1 : t
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
                       int32_t* err, cudaStream_t st) {
     const int tx = (n_cols + kUmTileN - 1) / kUmTileN, ty = (m_rows + kUmTileM - 1) / kUmTileM;
-    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err, nullptr, 0.f, nullptr, nullptr, tx};
+    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err, nullptr, 0.f, nullptr, nullptr, tx, QkvEpilogue{}};
+    launch_chained(umma_gemm_kernel, dim3(umma_grid(tx * ty)), dim3(kUmThreads), umma_smem_bytes(), st, tm_a, tm_b, p);
+    return 1;
+}
+
+// QKV projection of a prefill-sized call with the per-head norm, RoPE and cache append in its epilogue.
+int launch_umma_qkv(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, const QkvEpilogue& ep,
+                    int32_t* err, cudaStream_t st) {
+    const int tx = (n_cols + kUmTileN - 1) / kUmTileN, ty = (m_rows + kUmTileM - 1) / kUmTileM;
+    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 3, nullptr, nullptr, err, nullptr, 0.f, nullptr, nullptr, tx, ep};
     launch_chained(umma_gemm_kernel, dim3(umma_grid(tx * ty)), dim3(kUmThreads), umma_smem_bytes(), st, tm_a, tm_b, p);
     return 1;
 }
@@ -557,10 +647,10 @@ int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_
     const int max_groups = s.E + (n_slots + kUmTileM - 1) / kUmTileM;
     launch_chained(gather_rows_kernel, dim3(n_slots), dim3(256), 0, st, b, s.H, n_slots);
     const int gx = (s.I + 127) / 128, dx = (s.H + kUmTileN - 1) / kUmTileN;
-    UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err, nullptr, 0.f, nullptr, nullptr, gx};
+    UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err, nullptr, 0.f, nullptr, nullptr, gx, QkvEpilogue{}};
     launch_chained(umma_gemm_kernel, dim3(umma_grid(gx * max_groups)), dim3(kUmThreads), umma_smem_bytes(), st, tm_xperm,
                    tm_wgu, gu);
-    UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err, nullptr, 0.f, nullptr, nullptr, dx};
+    UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err, nullptr, 0.f, nullptr, nullptr, dx, QkvEpilogue{}};
     launch_chained(umma_gemm_kernel, dim3(umma_grid(dx * max_groups)), dim3(kUmThreads), umma_smem_bytes(), st, tm_act,
                    tm_wdown, dn);
     return 3;
@@ -601,7 +691,7 @@ int launch_umma_score(const CUtensorMap& tm_h, const CUtensorMap& tm_lm, int n_r
                       float* out_logprobs, int32_t* err, cudaStream_t st) {
     const int n_tiles = (vocab + kUmTileN - 1) / kUmTileN;
     UmmaParams p{K, n_rows, nullptr, nullptr, 0, vocab, 2, logits_tap, nullptr, err, targets, inv_temp, score_ml, score_tgt,
-                 n_tiles};
+                 n_tiles, QkvEpilogue{}};
     launch_chained(umma_gemm_kernel, dim3(umma_grid(n_tiles * ((n_rows + kUmTileM - 1) / kUmTileM))), dim3(kUmThreads),
                    umma_smem_bytes(), st, tm_h, tm_lm, p);
     launch_chained(score_combine_kernel, dim3((n_rows + 7) / 8), dim3(256), 0, st, score_ml, score_tgt, targets, n_rows, n_tiles, vocab,

@@ -900,9 +900,11 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         const LayerW& w = m->layers[l];
         if (umma) {   // prefill-sized call: dense contractions on tcgen05 / TMEM
             const int qkv_rows = (s.nq + 2 * s.nkv) * s.D;
-            run(MARS_K_QKV, [&] {
-                int n = launch_umma_dense(m->tm_h, m->tm_wqkv[l], n_tok, qkv_rows, s.H, b.qkv, b.err, st);
-                return n + launch_qkv_post(s, b, lay, w, kv->view, l, n_tok, 1, st);
+            run(MARS_K_QKV, [&] {   // per-head norm, RoPE and the cache append happen in the contraction's epilogue
+                const QkvEpilogue ep{b.step + lay.tok_pos, b.step + lay.tok_seq, kv->view.block_table, b.rope, w.q_norm, w.k_norm,
+                                     b.q, kv->view.k_pool, kv->view.v_pool, kv->view.max_pages_per_seq, kv->view.n_pages,
+                                     kv->view.page_size, l, s.nq, s.nkv, s.D, s.qk_norm, s.eps};
+                return launch_umma_qkv(m->tm_h, m->tm_wqkv[l], n_tok, qkv_rows, s.H, ep, b.err, st);
             });
         } else {      // decode-sized call: weights stream once through tcgen05 with the operands swapped
             run(MARS_K_QKV, [&] {
