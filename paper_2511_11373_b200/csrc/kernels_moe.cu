@@ -523,34 +523,51 @@ __global__ void __launch_bounds__(kRouterThreads) resid_norm_kernel(Shape s, Buf
                                                                    int o_ksplit) {
     __shared__ float scratch[32];
     pdl_wait();
+    // four consecutive columns per thread and visit (hidden is a multiple of 256): 16-byte loads and stores
+    constexpr int kVec = kRowMaxPer / 4;
     const int t = blockIdx.x, tid = threadIdx.x, H = s.H;
-    float v[kRowMaxPer];
+    float4 v[kVec];
     const float* __restrict__ xin = b.x + (size_t)t * H;
 #pragma unroll
-    for (int i = 0; i < kRowMaxPer; ++i) {
-        const int c = tid + i * kRouterThreads;
-        v[i] = c < H ? xin[c] : 0.f;
+    for (int i = 0; i < kVec; ++i) {
+        const int c = (tid + i * kRouterThreads) * 4;
+        v[i] = c < H ? *reinterpret_cast<const float4*>(xin + c) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     for (int sp = 0; sp < o_ksplit; ++sp) {
         const float* __restrict__ part = b.opart + ((size_t)sp * n_tok + t) * H;
 #pragma unroll
-        for (int i = 0; i < kRowMaxPer; ++i) {
-            const int c = tid + i * kRouterThreads;
-            if (c < H) v[i] += part[c];
+        for (int i = 0; i < kVec; ++i) {
+            const int c = (tid + i * kRouterThreads) * 4;
+            if (c < H) {
+                const float4 pv = *reinterpret_cast<const float4*>(part + c);
+                v[i].x += pv.x; v[i].y += pv.y; v[i].z += pv.z; v[i].w += pv.w;
+            }
         }
     }
     float ss = 0.f;
 #pragma unroll
-    for (int i = 0; i < kRowMaxPer; ++i) {
-        const int c = tid + i * kRouterThreads;
-        if (c < H) { b.x[(size_t)t * H + c] = v[i]; ss += v[i] * v[i]; }
+    for (int i = 0; i < kVec; ++i) {
+        const int c = (tid + i * kRouterThreads) * 4;
+        if (c < H) {
+            *reinterpret_cast<float4*>(b.x + (size_t)t * H + c) = v[i];
+            ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+        }
     }
     ss = block_sum(ss, scratch);
     const float r = rsqrtf(ss / (float)H + s.eps);
 #pragma unroll
-    for (int i = 0; i < kRowMaxPer; ++i) {
-        const int c = tid + i * kRouterThreads;
-        if (c < H) split_bf16(v[i] * r * __bfloat162float(gain[c]), b.h[(size_t)t * 2 * H + c], b.h[(size_t)t * 2 * H + H + c]);
+    for (int i = 0; i < kVec; ++i) {
+        const int c = (tid + i * kRouterThreads) * 4;
+        if (c < H) {
+            const uint2 gw = *reinterpret_cast<const uint2*>(gain + c);
+            const float e0 = v[i].x * r * bf16_lo(gw.x), e1 = v[i].y * r * bf16_hi(gw.x);
+            const float e2 = v[i].z * r * bf16_lo(gw.y), e3 = v[i].w * r * bf16_hi(gw.y);
+            const uint32_t h0 = pack_bf16(e0, e1), h1 = pack_bf16(e2, e3);
+            const uint32_t l0 = pack_bf16(e0 - bf16_lo(h0), e1 - bf16_hi(h0)), l1 = pack_bf16(e2 - bf16_lo(h1), e3 - bf16_hi(h1));
+            __nv_bfloat16* hrow = b.h + (size_t)t * 2 * H + c;
+            *reinterpret_cast<uint2*>(hrow) = make_uint2(h0, h1);
+            *reinterpret_cast<uint2*>(hrow + H) = make_uint2(l0, l1);
+        }
     }
 }
 
