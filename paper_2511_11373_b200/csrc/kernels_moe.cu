@@ -166,14 +166,21 @@ __global__ void __launch_bounds__(kRouterCta) router_kernel(Shape s, Buffers b, 
 // Token permutation: histogram of expert ids, exclusive offsets, and for every expert the list of
 // token rows it serves (slot order inside an expert is arbitrary: every (token, expert) product is
 // computed independently of its slot).  Single block; also counts the distinct experts used.
-__global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int layer, int n_pairs, int tok_cap) {
+// `counted`: the per-expert counts were accumulated in b.perm_cnt by permute_count_kernel (large calls);
+// then this block only scans them, writes the offsets, the group list and b.perm_cur, clears b.perm_cnt
+// for the next use and leaves the slot assignment to permute_scatter_kernel.
+__global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int layer, int n_pairs, int tok_cap, int counted) {
     __shared__ int cnt[kMaxExperts];
     __shared__ int off[kMaxExperts + 1];
     pdl_wait();
     const int tid = threadIdx.x, E = s.E;
-    for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
-    __syncthreads();
-    for (int i = tid; i < n_pairs; i += blockDim.x) atomicAdd(&cnt[b.route_idx[i]], 1);
+    if (counted) {
+        for (int e = tid; e < E; e += blockDim.x) { cnt[e] = b.perm_cnt[e]; b.perm_cnt[e] = 0; }
+    } else {
+        for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
+        __syncthreads();
+        for (int i = tid; i < n_pairs; i += blockDim.x) atomicAdd(&cnt[b.route_idx[i]], 1);
+    }
     __syncthreads();
     // one expert per thread (E <= 1024): exclusive scans of the token counts (slot offsets), of the
     // group counts (positions in the group list) and of "has tokens" (distinct experts)
@@ -216,6 +223,10 @@ __global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int l
     }
     __syncthreads();
     for (int e = tid; e <= E; e += blockDim.x) b.expert_off[e] = off[e];
+    if (counted) {
+        for (int e = tid; e < E; e += blockDim.x) b.perm_cur[e] = off[e];
+        return;
+    }
     for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
     __syncthreads();
     for (int i = tid; i < n_pairs; i += blockDim.x) {
@@ -224,6 +235,61 @@ __global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int l
         b.slot_token[slot] = i / s.k;
         b.slot_of[i] = slot;
     }
+}
+
+// Large calls (tens of thousands of (token, expert) pairs) count and hand out the slots with many
+// blocks: every block histograms its chunk of pairs in shared memory and adds it to the global
+// counts; after the scan above, every block reserves a run of slots per expert with one atomic
+// per (block, expert) and places its pairs inside the run.  Which slot a pair gets depends on
+// scheduling; the results do not (every pair's product is computed on its own and combined per
+// token in a fixed order).
+constexpr int kPermChunk = 1024;     // pairs per block
+__global__ void __launch_bounds__(1024) permute_count_kernel(Shape s, Buffers b, int n_pairs) {
+    __shared__ int cnt[kMaxExperts];
+    pdl_wait();
+    const int tid = threadIdx.x, E = s.E;
+    for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
+    __syncthreads();
+    const int i0 = blockIdx.x * kPermChunk, i1 = min(n_pairs, i0 + kPermChunk);
+    for (int i = i0 + tid; i < i1; i += blockDim.x) atomicAdd(&cnt[b.route_idx[i]], 1);
+    __syncthreads();
+    for (int e = tid; e < E; e += blockDim.x)
+        if (cnt[e]) atomicAdd(&b.perm_cnt[e], cnt[e]);
+}
+
+__global__ void __launch_bounds__(1024) permute_scatter_kernel(Shape s, Buffers b, int n_pairs) {
+    __shared__ int cnt[kMaxExperts];
+    __shared__ int base[kMaxExperts];
+    pdl_wait();
+    const int tid = threadIdx.x, E = s.E;
+    for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
+    __syncthreads();
+    const int i0 = blockIdx.x * kPermChunk, i1 = min(n_pairs, i0 + kPermChunk);
+    for (int i = i0 + tid; i < i1; i += blockDim.x) atomicAdd(&cnt[b.route_idx[i]], 1);
+    __syncthreads();
+    for (int e = tid; e < E; e += blockDim.x) {
+        base[e] = cnt[e] ? atomicAdd(&b.perm_cur[e], cnt[e]) : 0;
+        cnt[e] = 0;
+    }
+    __syncthreads();
+    for (int i = i0 + tid; i < i1; i += blockDim.x) {
+        const int e = b.route_idx[i];
+        const int slot = base[e] + atomicAdd(&cnt[e], 1);
+        b.slot_token[slot] = i / s.k;
+        b.slot_of[i] = slot;
+    }
+}
+
+static int launch_permute(const Shape& s, const Buffers& b, int layer, int n_pairs, int cap, cudaStream_t st) {
+    if (n_pairs < 4 * kPermChunk) {
+        launch_chained(permute_kernel, dim3(1), dim3(1024), 0, st, s, b, layer, n_pairs, cap, 0);
+        return 1;
+    }
+    const int blocks = (n_pairs + kPermChunk - 1) / kPermChunk;
+    launch_chained(permute_count_kernel, dim3(blocks), dim3(1024), 0, st, s, b, n_pairs);
+    launch_chained(permute_kernel, dim3(1), dim3(1024), 0, st, s, b, layer, n_pairs, cap, 1);
+    launch_chained(permute_scatter_kernel, dim3(blocks), dim3(1024), 0, st, s, b, n_pairs);
+    return 3;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -592,8 +658,7 @@ int launch_resid_norm(const Shape& s, const Buffers& b, const LayerW& w, int n_t
 int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int group_cap,
                         cudaStream_t st) {
     launch_chained(route_select_kernel, dim3((n_tok + 3) / 4), dim3(128), 4 * s.E * sizeof(float), st, s, b, dbg, layer, n_tok);
-    launch_chained(permute_kernel, dim3(1), dim3(1024), 0, st, s, b, layer, n_tok * s.k, group_cap);
-    return 2;
+    return 1 + launch_permute(s, b, layer, n_tok * s.k, group_cap, st);
 }
 
 // Tokens per group (4 per column tile); experts with more tokens are cut into several groups and
@@ -616,8 +681,7 @@ int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const Debug
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
     if (group_cap > 0) cap = group_cap;          // the tensor-core expert path wants one 128-row tile per group
-    launch_chained(permute_kernel, dim3(1), dim3(1024), 0, st, s, b, layer, n_tok * s.k, cap);
-    return 2;
+    return 1 + launch_permute(s, b, layer, n_tok * s.k, cap, st);
 }
 
 int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st) {

@@ -116,6 +116,8 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
     t.slot_of = (int32_t*)take(n * kk * 4);
     t.groups = (int32_t*)take(((size_t)c.n_experts + n * kk / 4 + 1) * 16);
     t.n_groups = (int32_t*)take(256);
+    t.perm_cnt = (int32_t*)take((size_t)c.n_experts * 4);
+    t.perm_cur = (int32_t*)take((size_t)c.n_experts * 4);
     t.active = (int32_t*)take((size_t)c.n_layers * 4);
     t.act = (__nv_bfloat16*)take(n * kk * 2 * c.expert_inter * 2);
     t.xperm = (__nv_bfloat16*)take(n > kUmmaMinTokens ? n * kk * 2 * H * 2 : 0);
@@ -329,6 +331,8 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
     e = cudaMemset(m->buf.err, 0, 256);
     if (e != cudaSuccess) return fail(e);
     e = cudaMemset(m->buf.active, 0, (size_t)cfg->n_layers * 4);
+    if (e != cudaSuccess) return fail(e);
+    e = cudaMemset(m->buf.perm_cnt, 0, (size_t)cfg->n_experts * 4);
     if (e != cudaSuccess) return fail(e);
     // tensor maps of the prefill path (calls with more than kUmmaMinTokens token rows)
     m->umma_ready = false;

@@ -68,6 +68,8 @@ struct Buffers {
     int32_t* slot_of;       // [n_tok k] slot of (token, j)
     int32_t* groups;        // [n_groups][4] (expert, first slot, tokens, 0): the expert kernels' work list
     int32_t* n_groups;
+    int32_t* perm_cnt;      // [E] tokens per expert, counted by many blocks (large calls); zero between uses
+    int32_t* perm_cur;      // [E] next free slot of every expert while the slots are handed out (large calls)
     int32_t* active;        // [L] distinct experts per layer
     __nv_bfloat16* act;     // [n_tok k, 2, I] SwiGLU activations, (hi, lo) rows
     __nv_bfloat16* xperm;   // [n_tok k, 2, H] activations gathered into expert-slot order (prefill path only)

@@ -308,6 +308,13 @@ def test_prefill_many_tokens_tensor_core_path():
     run_and_compare(case, toks, label="decode after large prefill")
 
 
+def test_prefill_with_thousands_of_tokens_uses_the_multi_block_permutation():
+    """From 4096 (token, expert) pairs on, the expert slots are counted and handed out by many blocks
+    (which slot a pair gets then depends on scheduling; the results must not)."""
+    model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=1)
+    prefill_and_compare(model, 32, [0, 10, 40], [1300, 640, 310], seed=27, label="prefill-2250")
+
+
 MODEL_GQA8 = dict(n_layers=2, hidden=512, n_q_heads=16, n_kv_heads=2, head_dim=128, n_experts=8, top_k=2, expert_inter=128,
                   vocab=1024, qk_norm=1, rope_theta=1e6, rms_eps=1e-6)
 
