@@ -272,7 +272,7 @@ def run_mixed(args):
     torch.cuda.set_device(device)
     cfg = wl.CONFIGS[args.workload]
     pf = cfg["prefill"]
-    w = DecodeWorkload(cfg, args.warmup + args.steps + 4, device, prefill_reqs=pf["requests"], prefill_chunk=pf["chunk"])
+    w = DecodeWorkload(cfg, 3 * (args.warmup + args.steps) + 16, device, prefill_reqs=pf["requests"], prefill_chunk=pf["chunk"])
     model = cfg["model"]
     n_pf = pf["requests"] * pf["chunk"]
     toks = wl.make_tokens(n_pf, model["vocab"], seed=1, name="prompts").to(device)
@@ -282,6 +282,18 @@ def run_mixed(args):
     smp = binding.make_sampling(seed=3, step=0, **w.sampling)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
     stream = torch.cuda.current_stream()
+    # decode steps back to back (steady state of a decode-only phase)
+    for _ in range(max(args.warmup, 3)):
+        w.step()
+    n_steady = max(args.steps, 6)
+    torch.cuda.synchronize()
+    ev[0].record(stream)
+    for _ in range(n_steady):
+        w.step()
+    ev[1].record(stream)
+    torch.cuda.synchronize()
+    steady_ms = ev[0].elapsed_time(ev[1]) / n_steady
+    steady_bytes = algorithmic_bytes(model, w.kv_tokens_now() - w.B * n_steady // 2, w.model.active_experts().tolist())
     t_pf, t_dec = [], []
     for it in range(args.warmup + args.steps):
         for s_ in ids:
@@ -343,7 +355,10 @@ def run_mixed(args):
                 data="synthetic",
                 config=dict(workload=cfg["name"], decode_seqs=w.B, prefill_requests=pf["requests"], prefill_chunk=pf["chunk"],
                             l2="inputs larger than L2"),
-                decode=dict(ms=dec_ms, bytes=dec_bytes["total"], frac_of_measured_hbm=dec_bytes["total"] / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]),
+                decode=dict(ms=dec_ms, bytes=dec_bytes["total"], frac_of_measured_hbm=dec_bytes["total"] / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                            note="one decode step right after each prefill call"),
+                decode_back_to_back=dict(ms=steady_ms, tokens_per_s=w.B / (steady_ms / 1e3), bytes=steady_bytes["total"],
+                                         frac_of_measured_hbm=steady_bytes["total"] / (steady_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]),
                 prefill=dict(ms=pf_ms, tokens_per_s=n_pf / (pf_ms / 1e3), algorithmic_tflop=flops / 1e12,
                              achieved_tflops=flops / (pf_ms * 1e-3) / 1e12, frac_of_measured_bf16=flops / (pf_ms * 1e-3) / 1e12 / tflops_peak,
                              note="activations are (hi, lo) bf16 pairs: the tensor cores execute twice the algorithmic flops in the projections"),
