@@ -186,10 +186,11 @@ MARS_API int32_t mars_kv_page_refs(const mars_kv_t *kv, int32_t page);
 /* Reading a shared prefix once (on by default).  When several DECODE rows of one call list the same
  * pages from position 0 on -- the members of a rollout group after mars_kv_seq_fork (Section 3.3:
  * the outputs of a group continue one common input) -- the decode step reads the common whole pages
- * once per block of 4 such rows instead of once per row: every K/V tile of the prefix is fetched
- * into shared memory once and scored against the queries of all rows of the block, each row keeps
- * its own online softmax, and the per-row partial results join the row's own spans in the usual
- * log-sum-exp merge.  Results equal those of the per-row reading up to fp32 summation order.
+ * once per block of such rows instead of once per row (blocks of 16 rows on the tensor-core kernel
+ * for head_dim 128 with 8 query heads per KV head, blocks of 4 rows otherwise): every K/V tile of the
+ * prefix is fetched into shared memory once and scored against the queries of all rows of the block,
+ * each row keeps its own online softmax, and the per-row partial results join the row's own spans in
+ * the usual log-sum-exp merge.  Results equal those of the per-row reading up to fp32 summation order.
  * Prefixes shorter than 128 tokens, prompt rows, and the allocation-free entry point read per row.
  * enable == 0 switches the grouping off (every row reads its whole context), e.g. to compare. */
 MARS_API mars_status_t mars_kv_share_reads(mars_kv_t *kv, int32_t enable);

@@ -74,6 +74,13 @@ int fattn_block_tokens();
 int launch_fattn_prefill(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_q,
                          const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
                          cudaStream_t st);
+// Shared spans of decode rows on the same kernel: items of fattn_shared_item_words() words, up to
+// fattn_shared_rows() rows each; tm_q1 is the query map with one-token boxes.
+int fattn_shared_rows();
+int fattn_shared_item_words();
+int launch_fattn_shared(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_q1,
+                        const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
+                        cudaStream_t st);
 int launch_attn_merge(const Shape& s, const Buffers& b, const StepLayout& lay, int n_tok, cudaStream_t st);
 
 // o_ksplit: number of split-K partials of the output projection that the router kernel adds to the residual.

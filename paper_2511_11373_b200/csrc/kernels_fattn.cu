@@ -22,6 +22,12 @@
 //                       when the running max moves).  Eight warps, two per scheduler, hide each
 //                       other's instruction latencies; with four the kernel ran at half the speed.
 // While the softmax warps work on tile j the tensor pipe already computes S of tile j + 1.
+//
+// SHARED mode (decode): the 16 "tokens" of a block are decode rows of DIFFERENT sequences that list the
+// same pages for a span of cached tokens (members of a rollout group forked from one prompt).  An
+// item is (first cached token, tokens, rows <= 16, 0, token row x 16, partial slot x 16); the query
+// tile is assembled from one-token TMA boxes, every row sees the whole span, and each row's (max,
+// sum, unnormalised O) goes to its partial slot for the span merge.
 // Every wait is bounded: a wait that gives up sets the device status word, all roles stop, the CTA
 // frees its TMEM columns and returns.
 #include "common.cuh"
@@ -48,11 +54,15 @@ constexpr int kFaSoftmaxThreads = 256;
 constexpr int kFaTmemCols = 512;           // S buffers at columns 0 and 64, O_tile buffers at 128 and 256
 constexpr uint32_t kFaSpin = 1u << 22;
 
+constexpr int kFaShItem = 4 + 2 * kFaQ;   // words of a shared item
+
 struct FaParams {
     const int32_t* step;
     StepLayout lay;
     const int32_t* block_table;
     __nv_bfloat16* o_out;      // [n_tok][2][nq * D]
+    float* part_o;             // [slots][nq][D] (shared mode)
+    float2* part_ml;           // [slots][nq]
     int32_t* err;
     int max_pages_per_seq, n_pages, page_size, box_rows, nkv, nq, layer;
     float scale_log2;
@@ -148,21 +158,29 @@ __device__ __forceinline__ float fa_exp2(float x) {
     return y;
 }
 
-struct FaUnit { int row0, len, nq_blk, hk, n_tiles; const int32_t* bt; };
+struct FaUnit { int row0, start, len, nq_blk, hk, n_tiles; const int32_t* bt; const int32_t* it; };
 
+template <bool SHARED>
 __device__ __forceinline__ FaUnit fa_unit(const FaParams& p, int u) {
     FaUnit c;
     const int item = u / p.nkv;
     c.hk = u - item * p.nkv;
-    const int4 it = reinterpret_cast<const int4*>(p.step + p.lay.items)[p.step[H_PF_FIRST] + item];
-    c.row0 = it.x; c.len = it.z; c.nq_blk = it.w;                  // len: keys visible to the LAST query of the block
+    if (SHARED) {
+        c.it = p.step + p.lay.sh_items + kFaShItem * item;
+        c.start = c.it[0]; c.len = c.it[1]; c.nq_blk = c.it[2]; c.row0 = c.it[4];
+    } else {
+        const int4 it = reinterpret_cast<const int4*>(p.step + p.lay.items)[p.step[H_PF_FIRST] + item];
+        c.it = nullptr;
+        c.row0 = it.x; c.start = 0; c.len = it.z; c.nq_blk = it.w;  // len: keys visible to the LAST query of the block
+    }
     c.n_tiles = (c.len + kFaKv - 1) / kFaKv;
     c.bt = p.block_table + (size_t)p.step[p.lay.tok_seq + c.row0] * p.max_pages_per_seq;
     return c;
 }
 
+template <bool SHARED>
 __global__ void __launch_bounds__(kFaThreads, 1)
-fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, FaParams p) {
     extern __shared__ unsigned char fa_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)fa_raw + 1023) & ~(uintptr_t)1023);
@@ -198,7 +216,7 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const uint32_t tmem = tmem_slot;
     pdl_wait();
 
-    const int n_units = p.step[H_PF_ITEMS] * p.nkv;
+    const int n_units = p.step[SHARED ? H_SH_ITEMS : H_PF_ITEMS] * p.nkv;
 
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
@@ -206,7 +224,7 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             uint32_t g = 0;                                          // tiles requested so far (ring positions)
             int local = 0;
             for (int u = blockIdx.x; u < n_units && !dead; u += gridDim.x, ++local) {
-                const FaUnit c = fa_unit(p, u);
+                const FaUnit c = fa_unit<SHARED>(p, u);
                 // tile j of this unit: K into its ring, V into its ring (separate lifetimes: K is free once
                 // S is computed, V only after P V)
                 auto load_tile = [&](int j) -> bool {
@@ -220,7 +238,7 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     fa_expect_tx(&k_full[ks], (uint32_t)(n_boxes * p.box_rows * 128 * 2));
                     fa_expect_tx(&v_full[vs], (uint32_t)(n_boxes * p.box_rows * 128 * 2));
                     for (int bi = 0; bi < n_boxes; ++bi) {
-                        const int tok = j * kFaKv + bi * p.box_rows;
+                        const int tok = c.start + j * kFaKv + bi * p.box_rows;
                         const int page = c.bt[tok / p.page_size];
                         const int y = (((p.layer * p.n_pages + page) * p.nkv + c.hk) * p.page_size) + tok % p.page_size;
                         const int off = bi * p.box_rows * 128;
@@ -237,7 +255,17 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 bool ok = true;
                 for (int j = 0; j < early && ok; ++j) ok = load_tile(j);
                 if (ok) ok = fa_wait(&q_free, (local & 1) ^ 1);
-                if (ok) {
+                if (ok && SHARED) {
+                    // one-token boxes (8 heads x 128 B = 1 KB each): row i of the block is token row it[4 + i]
+                    fa_expect_tx(&q_full, (uint32_t)c.nq_blk * 4096u);
+                    for (int i = 0; i < c.nq_blk; ++i)
+#pragma unroll
+                        for (int pl = 0; pl < 2; ++pl)
+#pragma unroll
+                            for (int hf = 0; hf < 2; ++hf)
+                                fa_tma_4d(q_smem + (pl * 2 + hf) * kFaQTile + i * 1024, &tm_q, hf * 64, c.hk * kFaHeads, pl,
+                                          c.it[4 + i], &q_full);
+                } else if (ok) {
                     fa_expect_tx(&q_full, kFaQBytes);
 #pragma unroll
                     for (int pl = 0; pl < 2; ++pl)
@@ -278,7 +306,7 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 return true;
             };
             for (int u = blockIdx.x; u < n_units && !dead; u += gridDim.x, ++local) {
-                const FaUnit c = fa_unit(p, u);
+                const FaUnit c = fa_unit<SHARED>(p, u);
                 bool ok = fa_wait(&q_full, local & 1);
                 if (ok) ok = issue_s(g);
                 if (ok && c.n_tiles > 1) ok = issue_s(g + 1);
@@ -313,9 +341,9 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         constexpr int SC = kFaKv / 2, OC = kFaD / 2;                 // score and output columns of this thread
         uint32_t g = 0;
         for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-            const FaUnit c = fa_unit(p, u);
+            const FaUnit c = fa_unit<SHARED>(p, u);
             // keys visible to this row's query; rows past the block's last token are computed but never stored
-            const int my_len = min(c.len, c.len - (c.nq_blk - 1 - q_tok));
+            const int my_len = SHARED ? c.len : min(c.len, c.len - (c.nq_blk - 1 - q_tok));
             float o[OC];
 #pragma unroll
             for (int i = 0; i < OC; ++i) o[i] = 0.f;
@@ -410,7 +438,15 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             xsum[half][r] = l_run;
             asm volatile("bar.sync 1, %0;" ::"n"(kFaSoftmaxThreads) : "memory");
             const float l_row = l_run + xsum[half ^ 1][r];
-            if (q_tok < c.nq_blk) {
+            if (SHARED) {
+                if (q_tok < c.nq_blk) {
+                    const size_t ph = (size_t)c.it[4 + kFaQ + q_tok] * p.nq + c.hk * kFaHeads + head;
+                    float* dst = p.part_o + ph * kFaD + half * OC;
+#pragma unroll
+                    for (int i = 0; i < OC; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+                    if (half == 0) p.part_ml[ph] = make_float2(m_run, l_row);
+                }
+            } else if (q_tok < c.nq_blk) {
                 const float inv = 1.f / l_row;
                 __nv_bfloat16* dst = p.o_out + (size_t)(c.row0 + q_tok) * 2 * p.nq * kFaD + (size_t)(c.hk * kFaHeads + head) * kFaD +
                                      half * OC;
@@ -440,24 +476,46 @@ fattn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 bool fattn_supported(const Shape& s) { return s.D == kFaD && s.nq / s.nkv == kFaHeads; }
 int fattn_block_tokens() { return kFaQ; }
 
-int launch_fattn_prefill(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_q,
-                         const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
-                         cudaStream_t st) {
+static FaParams fa_params(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, int layer) {
     FaParams p;
-    p.step = b.step; p.lay = lay; p.block_table = kv.block_table; p.o_out = b.o; p.err = b.err;
+    p.step = b.step; p.lay = lay; p.block_table = kv.block_table; p.o_out = b.o; p.part_o = b.part_o; p.part_ml = b.part_ml;
+    p.err = b.err;
     p.max_pages_per_seq = kv.max_pages_per_seq; p.n_pages = kv.n_pages; p.page_size = kv.page_size;
     p.box_rows = kv.page_size < kFaKv ? kv.page_size : kFaKv;
     p.nkv = s.nkv; p.nq = s.nq; p.layer = layer;
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
+    return p;
+}
+
+int launch_fattn_prefill(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_q,
+                         const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
+                         cudaStream_t st) {
+    const FaParams p = fa_params(s, b, lay, kv, layer);
     int grid = n_items * s.nkv;
     if (grid > sm_count) grid = sm_count;
     if (grid < 1) grid = 1;
-    launch_chained(fattn_prefill_kernel, dim3(grid), dim3(kFaThreads), (size_t)kFaSmem + 1024, st, tm_q, tm_k, tm_v, p);
+    launch_chained(fattn_kernel<false>, dim3(grid), dim3(kFaThreads), (size_t)kFaSmem + 1024, st, tm_q, tm_k, tm_v, p);
+    return 1;
+}
+
+// Shared spans of decode rows: tm_q1 is the query map with one-token boxes.
+int fattn_shared_rows() { return kFaQ; }
+int fattn_shared_item_words() { return kFaShItem; }
+int launch_fattn_shared(const Shape& s, const Buffers& b, const StepLayout& lay, const KvView& kv, const CUtensorMap& tm_q1,
+                        const CUtensorMap& tm_k, const CUtensorMap& tm_v, int layer, int n_items, int sm_count,
+                        cudaStream_t st) {
+    const FaParams p = fa_params(s, b, lay, kv, layer);
+    int grid = n_items * s.nkv;
+    if (grid > sm_count) grid = sm_count;
+    if (grid < 1) grid = 1;
+    launch_chained(fattn_kernel<true>, dim3(grid), dim3(kFaThreads), (size_t)kFaSmem + 1024, st, tm_q1, tm_k, tm_v, p);
     return 1;
 }
 
 cudaError_t init_fattn_kernels() {
-    return cudaFuncSetAttribute(fattn_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmem + 1024);
+    cudaError_t e = cudaFuncSetAttribute(fattn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmem + 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(fattn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmem + 1024);
 }
 
 }  // namespace mars

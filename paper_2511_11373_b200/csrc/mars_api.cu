@@ -38,7 +38,8 @@ namespace {
 constexpr int kSpanTokens = 1024;   // cached tokens per attention work item at decode
 constexpr int kStagingSlots = 4;
 constexpr int kUmmaMinTokens = 64;  // calls with more token rows take the tensor-core (tcgen05) contraction path
-constexpr int kSharedRows = 4;      // decode rows per work item of the shared-prefix attention kernel
+constexpr int kSharedRows = 4;      // decode rows per work item of the shared-prefix attention kernel on mma.sync
+constexpr int kSharedItemWords = 36; // capacity per shared item: the tcgen05 kernel's items hold 16 rows
 constexpr int kMinSharedTokens = 128;  // shorter common prefixes are read per row as usual
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -70,7 +71,7 @@ StepLayout make_layout(const Caps& k) {
     l.emit_slot = take(k.n_emit);
     l.updates = take(3 * k.n_updates);
     l.items = take(4 * k.n_items);
-    l.sh_items = take(12 * (k.n_items / 2 + 1));   // a shared item stands for the spans of at least two rows
+    l.sh_items = take(kSharedItemWords * (k.n_items / 2 + 1));   // a shared item stands for the spans of at least two rows
     l.total_words = at;
     return l;
 }
@@ -158,9 +159,10 @@ static mars_status_t make_tiled_map(CUtensorMap* tm, const void* base, int rank,
     return MARS_OK;
 }
 // queries [token][2][nq][D] as a 4-D tensor (d, head, plane, token): boxes of 64 elements x 8 heads x 16 tokens
-static mars_status_t make_query_map(CUtensorMap* tm, const void* q, uint64_t tokens, uint64_t nq, uint64_t D) {
+static mars_status_t make_query_map(CUtensorMap* tm, const void* q, uint64_t tokens, uint64_t nq, uint64_t D,
+                                    uint32_t box_tokens = 16) {
     const cuuint64_t dims[4] = {D, nq, 2, tokens}, strides[3] = {D * 2, nq * D * 2, 2 * nq * D * 2};
-    const cuuint32_t box[4] = {64u, 8u, 1u, 16u};
+    const cuuint32_t box[4] = {64u, 8u, 1u, box_tokens};
     return make_tiled_map(tm, q, 4, dims, strides, box);
 }
 // weights [rows][K]: boxes of 64 rows x 64 elements
@@ -188,7 +190,8 @@ struct mars_model {
     CUtensorMap tm_h, tm_o, tm_xperm, tm_act;
     CUtensorMap tm_h64, tm_o64, tm_lm;      // decode-sized (64 token rows per box) and the lm_head
     CUtensorMap tm_q;                       // queries for the tcgen05 prefill attention: (d, head, plane, token)
-    bool fattn_ready;
+    CUtensorMap tm_q1;                      // the same tensor with one-token boxes (shared spans of decode rows)
+    bool fattn_ready, fattn_shared_ready;
     bool umma_ready;
     const __nv_bfloat16 *embed, *final_norm, *lm_head;
     int32_t *io_in, *io_out;
@@ -361,6 +364,11 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
             if (rc == MARS_OK) rc = make_pair_map(&m->tm_act, m->buf.act, slots, I);
         }
         m->fattn_ready = false;
+        m->fattn_shared_ready = false;
+        if (rc == MARS_OK && fattn_supported(m->shape)) {
+            rc = make_query_map(&m->tm_q1, m->buf.q, n, (uint64_t)cfg->n_q_heads, (uint64_t)cfg->head_dim, 1);
+            m->fattn_shared_ready = rc == MARS_OK;
+        }
         if (rc == MARS_OK && big && fattn_supported(m->shape)) {
             rc = make_query_map(&m->tm_q, m->buf.q, n, (uint64_t)cfg->n_q_heads, (uint64_t)cfg->head_dim);
             m->fattn_ready = rc == MARS_OK;
@@ -755,6 +763,10 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         ++pf_items;
     }
     if (pf_items > m->caps.n_items) return MARS_ERR_INVALID_ARG;
+    // rows per shared item and words per item: 16 rows on the tcgen05 kernel, 4 on the mma.sync kernel
+    const bool fa_shared = m->fattn_shared_ready;
+    const int sh_rows = fa_shared ? fattn_shared_rows() : kSharedRows;
+    const int sh_words = fa_shared ? fattn_shared_item_words() : 12;
     int64_t dec_items = 0, dec_slots = 0, sh_items = 0;
     for (;;) {
         dec_items = dec_slots = sh_items = 0;
@@ -764,7 +776,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             dec_slots += own + (row_shared[t] + span - 1) / span;
         }
         for (const SharedGroup& g : shared)
-            sh_items += (int64_t)((g.tokens + span - 1) / span) * (((int64_t)g.rows.size() + kSharedRows - 1) / kSharedRows);
+            sh_items += (int64_t)((g.tokens + span - 1) / span) * (((int64_t)g.rows.size() + sh_rows - 1) / sh_rows);
         if (dec_slots + pf_items <= m->caps.n_items && sh_items <= m->caps.n_items / 2 + 1) break;
         if (span > (1 << 28)) return MARS_ERR_INVALID_ARG;
         span *= 2;
@@ -826,14 +838,14 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         int sh_at = 0;
         for (const SharedGroup& g : shared) {
             for (int s0 = 0; s0 < g.tokens; s0 += span) {
-                for (size_t r0 = 0; r0 < g.rows.size(); r0 += kSharedRows) {
-                    const int nr = (int)std::min<size_t>(kSharedRows, g.rows.size() - r0);
-                    int32_t* it = sh + 12 * sh_at++;
+                for (size_t r0 = 0; r0 < g.rows.size(); r0 += (size_t)sh_rows) {
+                    const int nr = (int)std::min<size_t>((size_t)sh_rows, g.rows.size() - r0);
+                    int32_t* it = sh + sh_words * sh_at++;
                     it[0] = s0; it[1] = std::min(span, g.tokens - s0); it[2] = nr; it[3] = 0;
-                    for (int i = 0; i < kSharedRows; ++i) {
+                    for (int i = 0; i < sh_rows; ++i) {
                         const int row = g.rows[r0 + (size_t)std::min(i, nr - 1)];
                         it[4 + i] = row;
-                        it[8 + i] = off[row] + s0 / span;
+                        it[4 + sh_rows + i] = off[row] + s0 / span;
                     }
                     kv_streamed += it[1];
                 }
@@ -858,7 +870,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
     const size_t used_words = (size_t)lay.items + 4 * (size_t)(dec_items + pf_items);
     CUDA_TRY(cudaMemcpyAsync(m->buf.step, blk, used_words * 4, cudaMemcpyHostToDevice, st));
     if (sh_items)
-        CUDA_TRY(cudaMemcpyAsync(m->buf.step + lay.sh_items, blk + lay.sh_items, (size_t)sh_items * 12 * 4,
+        CUDA_TRY(cudaMemcpyAsync(m->buf.step + lay.sh_items, blk + lay.sh_items, (size_t)sh_items * sh_words * 4,
                                  cudaMemcpyHostToDevice, st));
     CUDA_TRY(cudaEventRecord(m->staged[slot], st));
 
@@ -920,6 +932,9 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         if (n_dec > 0) {      // decode rows: spans of cached tokens, then the merge of each row's spans
             if (sh_items)
                 run(MARS_K_ATTN, [&] {
+                    if (fa_shared)
+                        return launch_fattn_shared(s, b, lay, kv->view, m->tm_q1, kv->tm_k, kv->tm_v, l, (int)sh_items,
+                                                   m->sm_count, st);
                     return launch_attention_shared(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, (int)sh_items, m->sm_count, st);
                 });
             run(MARS_K_ATTN, [&] { return launch_attention(s, b, lay, kv->view, kv->tm_k, kv->tm_v, l, m->sm_count, st); });

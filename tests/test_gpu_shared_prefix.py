@@ -115,6 +115,33 @@ def test_head_dim_128_pages_of_64_and_two_shared_spans():
         tokens = g["tokens"]
 
 
+MODEL_GQA8 = dict(n_layers=2, hidden=512, n_q_heads=16, n_kv_heads=2, head_dim=128, n_experts=8, top_k=2, expert_inter=128,
+                  vocab=1024, qk_norm=1, rope_theta=1e6, rms_eps=1e-6)
+
+
+@pytest.mark.parametrize("ps", [16, 64])
+def test_groups_on_the_tensor_core_kernel(ps):
+    """head_dim 128 with 8 query heads per KV head: the shared spans run on tcgen05, up to 16 member rows x
+    8 heads as the 128 accumulator rows of one pass over the keys.  A group of 18 members (blocks of
+    16 + 2 rows) whose prompt spans two spans (1024 + 256 tokens, plus a partly filled page that is
+    copied per member), a pair with a short prompt, and a loner."""
+    ctx = [1290, 200, 77]
+    forks = [(0, s) for s in range(3, 20)] + [(1, 20)]
+    shared = build(MODEL_GQA8, ps, ctx, forks, True, seed=65 + ps, headroom=4, spare=40)
+    plain = build(MODEL_GQA8, ps, ctx, forks, False, seed=65 + ps, headroom=4, spare=40)
+    ids = [7, 2, 0, 20] + [s for s in range(3, 20) if s != 7] + [1]
+    tokens = wl.make_tokens(len(ids), MODEL_GQA8["vocab"], seed=9)
+    big = (1290 // ps) * ps                                  # whole pages of the long prompt
+    small = (200 // ps) * ps
+    smp = dict(greedy=0, temperature=0.85, top_p=0.95)
+    for step in range(3):
+        g, stats = step_both(shared, plain, ids, tokens, smp, step, 11, f"tcgen05 groups ps={ps} step {step}")
+        info = shared.model.last_step_info()
+        assert info["kv_tokens_streamed"] == info["kv_tokens_read"] - (18 - 2) * big - (2 - 1) * small
+        print("shared-prefix tcgen05", ps, step, stats, info)
+        tokens = g["tokens"]
+
+
 def test_short_common_prefix_and_single_rows_take_the_per_row_path():
     model = dict(wl.MODEL_TINY, n_layers=1)
     shared = build(model, 16, [100, 200], [(0, 2)], True, seed=63, headroom=4, spare=8)   # 96 shared tokens < 128
