@@ -123,7 +123,9 @@ class DecodeWorkload:
         self.cfg, self.device = cfg, device
         model, ps = cfg["model"], cfg["page_size"]
         self.model_shape = model
-        self.ctx, self.stages = wl.make_context_lengths(cfg, seed=seed)
+        # the uniform context draw of configs 2 / 3 uses the seed whose total is closest to its expectation
+        ctx_seed = wl.CONFIG3_CONTEXT_SEED if "ctx_range" in cfg else seed
+        self.ctx, self.stages = wl.make_context_lengths(cfg, seed=ctx_seed)
         B = len(self.ctx)
         self.B = B
         cap = [c + total_steps + 1 for c in self.ctx]
@@ -184,7 +186,7 @@ class OracleSample:
         self.oracle, self.cfg = oracle, cfg
         self.model = dict(cfg["model"])
         one = dict(self.model, n_layers=1)
-        ctx_all, _ = wl.make_context_lengths(cfg, seed=seed)
+        ctx_all, _ = wl.make_context_lengths(cfg, seed=wl.CONFIG3_CONTEXT_SEED if "ctx_range" in cfg else seed)
         self.n_all = len(ctx_all)
         self.n_seq = min(n_seq, self.n_all)
         ctx = ctx_all[: self.n_seq]

@@ -106,6 +106,9 @@ typedef struct {
     int32_t *router_idx;       /* [n_layers, n, top_k], larger probability first                  */
     const int32_t *forced_idx; /* [n_layers, n, top_k] or NULL: route to these experts instead    */
     float *nucleus_mass;       /* [rows]: probability mass of the nucleus (1 when greedy)         */
+    int32_t *expert_off;       /* [n_layers, n_experts + 1]: exclusive offsets of the token permutation
+                                  (expert e serves slots expert_off[e] .. expert_off[e + 1] - 1)  */
+    int32_t *slot_token;       /* [n_layers, n * top_k]: token row served by every expert slot    */
 } mars_debug_t;
 
 typedef struct mars_model mars_model_t;
@@ -116,8 +119,8 @@ typedef struct mars_kv mars_kv_t;
 MARS_API size_t mars_workspace_bytes(const mars_config_t *cfg, int32_t max_decode_seqs, int32_t max_prefill_tokens);
 
 /* Validates the shape (MARS_ERR_UNSUPPORTED unless head_dim is 64 or 128, n_q_heads / n_kv_heads
- * is an integer <= 8, hidden and expert_inter are multiples of 64, top_k <= n_experts <= 1024,
- * top_k <= 32), records the borrowed weight pointers (no copy) and carves the workspace.  The
+ * is an integer <= 8, hidden is a multiple of 256 in [256, 8192], expert_inter a multiple of 64 in
+ * [64, 3136], top_k <= n_experts <= 1024, top_k <= 32), records the borrowed weight pointers (no copy) and carves the workspace.  The
  * workspace content is private to the library between calls. */
 MARS_API mars_status_t mars_model_load(const mars_config_t *cfg, const mars_weights_t *weights, void *workspace,
                               size_t workspace_bytes, int32_t max_decode_seqs, int32_t max_prefill_tokens,
@@ -137,7 +140,12 @@ MARS_API mars_status_t mars_kv_free(mars_kv_t *kv);
 MARS_API int32_t mars_kv_num_pages(const mars_kv_t *kv);
 MARS_API int32_t mars_kv_free_pages(const mars_kv_t *kv);
 
-/* Sequence slots 0 .. max_seqs-1.  reserve: make room for n_tokens_total tokens (allocates the
+/* Stream contract of the calls below that take no stream (reserve, adopt): the block-table entries
+ * they write are on the device when the call returns (copied on a private stream of the cache and
+ * waited for), so a step launched afterwards on any stream, blocking or not, sees them.  They only
+ * write entries that no step in flight reads (pages appended to a slot, or an empty slot's row).
+ *
+ * Sequence slots 0 .. max_seqs-1.  reserve: make room for n_tokens_total tokens (allocates the
  * missing pages from the free list; MARS_ERR_KV_FULL leaves the slot unchanged).  adopt: hand the
  * slot a list of specific free pages that the caller has filled, with ctx_len tokens valid
  * (MARS_ERR_BAD_HANDLE if a page is owned already or the slot is not empty).  set_len: declare how
@@ -286,6 +294,10 @@ MARS_API mars_status_t mars_decode_step_host(mars_model_t *model, mars_kv_t *kv,
  * out of range are read as token 0 (this call has no status word to poll).
  * First call on a device: the address of the built-in array is looked up and the kernels' launch
  * attributes are set, once per device; make that first call outside any stream capture.
+ * No call may be made on a capturing stream: the step reads ctx_lens on the host and uploads its
+ * work lists from host memory that is gone when the call returns, so a recorded copy would replay
+ * stale data.  A stream that is capturing is refused with MARS_ERR_UNSUPPORTED before anything is
+ * enqueued.
  * Sharing: all calls in the process use the same array, which keeps whatever the previous call
  * left; the call clears what must start from zero itself.  Two calls that overlap on the GPU (two
  * streams, two threads) overwrite each other's intermediates: serialise them. */
@@ -300,6 +312,15 @@ MARS_API mars_status_t mars_decode_step_static(const mars_config_t *cfg, const m
 /* Synchronises the stream of the last call and reads the device status word: MARS_OK,
  * MARS_ERR_BAD_TOKEN or MARS_ERR_TIMEOUT; the word is cleared. */
 MARS_API mars_status_t mars_poll_status(mars_model_t *model);
+
+/* Self-test of the bounded device-side waits (a test hook; the paper has no counterpart).  Every
+ * wait of the TMA / tensor-core kernels polls its barrier a limited number of times and, when the
+ * limit is reached, sets the timeout bit of the status word, releases its tensor memory and lets the
+ * kernel return.  This call launches one small block that takes exactly that path: a lane waits (at
+ * most 4096 polls) for an arrival that another lane delivers when arrive != 0 and withholds when
+ * arrive == 0.  With arrive == 0 the next mars_poll_status returns MARS_ERR_TIMEOUT once and the
+ * handle stays fully usable; nothing hangs, traps or faults.  Asynchronous on the stream. */
+MARS_API mars_status_t mars_debug_bounded_wait(mars_model_t *model, void *cuda_stream, int32_t arrive);
 
 /* Counters of the last step call: kernels launched by it, attention work items, cached tokens read. */
 typedef struct {

@@ -53,7 +53,7 @@ class mars_sampling_t(ctypes.Structure):
 
 class mars_debug_t(ctypes.Structure):
     _fields_ = [("logits", c_void_p), ("hidden", c_void_p), ("router_w", c_void_p), ("router_idx", c_void_p),
-                ("forced_idx", c_void_p), ("nucleus_mass", c_void_p)]
+                ("forced_idx", c_void_p), ("nucleus_mass", c_void_p), ("expert_off", c_void_p), ("slot_token", c_void_p)]
 
 
 class mars_step_info_t(ctypes.Structure):
@@ -101,6 +101,7 @@ SIGNATURES = {
                                           c_int32, c_void_p, c_int32, POINTER(c_int32), c_void_p, c_int32, c_void_p,
                                           POINTER(mars_sampling_t), c_void_p, c_void_p]),
     "mars_poll_status": (c_int32, [c_void_p]),
+    "mars_debug_bounded_wait": (c_int32, [c_void_p, c_void_p, c_int32]),
     "mars_profile_enable": (c_int32, [c_void_p, c_int32]),
     "mars_profile_read": (c_int32, [c_void_p, POINTER(ctypes.c_double), POINTER(c_int64)]),
     "mars_last_step_info": (c_int32, [c_void_p, POINTER(mars_step_info_t)]),
@@ -157,10 +158,11 @@ def make_sampling(greedy=True, temperature=1.0, top_p=1.0, seed=0, step=0) -> ma
     return mars_sampling_t(float(temperature), float(top_p), int(bool(greedy)), 0, int(seed), int(step))
 
 
-def make_debug(logits=None, hidden=None, router_w=None, router_idx=None, forced_idx=None, nucleus_mass=None):
-    d = mars_debug_t(*[t.data_ptr() if t is not None else None
-                       for t in (logits, hidden, router_w, router_idx, forced_idx, nucleus_mass)])
-    d._keep = (logits, hidden, router_w, router_idx, forced_idx, nucleus_mass)
+def make_debug(logits=None, hidden=None, router_w=None, router_idx=None, forced_idx=None, nucleus_mass=None,
+               expert_off=None, slot_token=None):
+    taps = (logits, hidden, router_w, router_idx, forced_idx, nucleus_mass, expert_off, slot_token)
+    d = mars_debug_t(*[t.data_ptr() if t is not None else None for t in taps])
+    d._keep = taps
     return d
 
 
@@ -197,6 +199,11 @@ class Model:
 
     def poll_status(self) -> int:
         return lib().mars_poll_status(self.handle)
+
+    def bounded_wait_selftest(self, arrive: bool, stream=None) -> int:
+        """Launches the library's bounded-wait self-test (see mars_debug_bounded_wait); returns the status code."""
+        with torch.cuda.device(self.device):
+            return lib().mars_debug_bounded_wait(self.handle, _stream_handle(stream), 1 if arrive else 0)
 
     def last_step_info(self) -> dict:
         info = mars_step_info_t()

@@ -124,6 +124,9 @@ int score_vocab_tiles(int vocab);
 int launch_umma_score(const CUtensorMap& tm_h, const CUtensorMap& tm_lm, int n_rows, int vocab, int K,
                       const int32_t* targets, float inv_temp, float2* score_ml, float* score_tgt, float* logits_tap,
                       float* out_logprobs, int32_t* err, cudaStream_t st);
+// One CTA that waits, with a limit of `limit` polls, for an mbarrier arrival that comes (arrive != 0) or
+// never comes (arrive == 0): the give-up path of the bounded waits, run without hanging anything.
+int launch_wait_probe(int32_t* err, int arrive, uint32_t limit, cudaStream_t st);
 int launch_qkv_post(const Shape& s, const Buffers& b, const StepLayout& lay, const LayerW& w, const KvView& kv, int layer,
                     int n_tok, int ksplit, cudaStream_t st);
 int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st);

@@ -39,8 +39,10 @@ __device__ __forceinline__ void um_mbar_init(uint64_t* bar, int count) {
 __device__ __forceinline__ void um_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool um_wait(uint64_t* bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kUmSpin; ++i) {
+// Bounded wait on an mbarrier phase: at most `limit` polls, then false (the caller sets the status
+// word, stops issuing, frees its tensor memory and returns).
+__device__ __forceinline__ bool um_wait_n(uint64_t* bar, uint32_t parity, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -51,6 +53,7 @@ __device__ __forceinline__ bool um_wait(uint64_t* bar, uint32_t parity) {
     }
     return false;
 }
+__device__ __forceinline__ bool um_wait(uint64_t* bar, uint32_t parity) { return um_wait_n(bar, parity, kUmSpin); }
 __device__ __forceinline__ void um_tma_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(smem_u32(dst)), "l"((uint64_t)tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
@@ -700,6 +703,42 @@ int launch_umma_score(const CUtensorMap& tm_h, const CUtensorMap& tm_lm, int n_r
 }
 
 int score_vocab_tiles(int vocab) { return (vocab + kUmTileN - 1) / kUmTileN; }
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the give-up path that every bounded wait above takes.  One CTA with the same roles as
+// the contraction kernels: a warp allocates tensor-memory columns, a consumer lane waits on an
+// mbarrier with um_wait_n, a producer lane arrives on it -- or, when `arrive` is 0, does not, so that
+// the wait runs out after `limit` polls.  The consumer then sets the timeout bit of the status word,
+// the CTA frees its tensor memory and the kernel returns normally; nothing traps, spins on or faults.
+__global__ void __launch_bounds__(96) wait_probe_kernel(int32_t* err, int arrive, uint32_t limit) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t tmem_slot;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        um_mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(32));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    pdl_wait();
+    if (warp == 1 && lane == 0 && arrive) um_arrive(&bar);
+    if (warp == 0 && lane == 0 && !um_wait_n(&bar, 0, limit)) atomicOr(err, kErrTimeout);
+    __syncthreads();
+    if (warp == 2) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_slot), "r"(32));
+    }
+}
+
+int launch_wait_probe(int32_t* err, int arrive, uint32_t limit, cudaStream_t st) {
+    launch_chained(wait_probe_kernel, dim3(1), dim3(96), 0, st, err, arrive, limit);
+    return 1;
+}
 
 cudaError_t init_umma_kernels() {
     int dev = 0;

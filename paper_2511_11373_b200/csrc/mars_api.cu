@@ -83,6 +83,9 @@ bool shape_supported(const mars_config_t& c) {
     if ((c.n_q_heads * c.head_dim) % 256) return false;
     if (c.n_experts < 1 || c.n_experts > 1024 || c.top_k < 1 || c.top_k > 32 || c.top_k > c.n_experts) return false;
     if (c.expert_inter < 64 || c.expert_inter % 64) return false;
+    // the streaming down kernel keeps up to 16 tokens x (hi, lo) activation rows of expert_inter elements in
+    // shared memory (200 KB are requested for it)
+    if ((size_t)32 * (2 * (size_t)c.expert_inter + 64) > 200u * 1024u) return false;
     if (c.vocab < 2 || c.max_pos < 1) return false;
     return true;
 }
@@ -225,6 +228,7 @@ struct mars_kv {
     std::vector<int32_t> free_list;   // stack of free page ids
     std::vector<int32_t> refs;        // number of sequence slots that list the page (0 = free)
     bool share_reads = true;          // decode rows with a common page prefix read it once (mars_kv_share_reads)
+    cudaStream_t copy_stream = nullptr;   // private stream of the block-table uploads (see upload_row)
 };
 
 extern "C" {
@@ -447,8 +451,11 @@ mars_status_t mars_kv_alloc(mars_model_t* m, void* k_pool, void* v_pool, size_t 
     mars_status_t st = make_pool_map(&kv->tm_k, k_pool, rows, c.head_dim, box_rows);
     if (st == MARS_OK) st = make_pool_map(&kv->tm_v, v_pool, rows, c.head_dim, box_rows);
     if (st != MARS_OK) { delete kv; return st; }
-    cudaError_t e = cudaMemset(meta, 0, mars_kv_meta_bytes(max_seqs, max_pages_per_seq));
+    cudaError_t e = cudaStreamCreateWithFlags(&kv->copy_stream, cudaStreamNonBlocking);
     if (e != cudaSuccess) { g_last_cuda_error = (int32_t)e; delete kv; return MARS_ERR_CUDA; }
+    e = cudaMemsetAsync(meta, 0, mars_kv_meta_bytes(max_seqs, max_pages_per_seq), kv->copy_stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(kv->copy_stream);
+    if (e != cudaSuccess) { g_last_cuda_error = (int32_t)e; cudaStreamDestroy(kv->copy_stream); delete kv; return MARS_ERR_CUDA; }
     kv->seqs.resize(max_seqs);
     kv->refs.assign(n_pages, 0);
     kv->free_list.resize(n_pages);
@@ -459,6 +466,7 @@ mars_status_t mars_kv_alloc(mars_model_t* m, void* k_pool, void* v_pool, size_t 
 
 mars_status_t mars_kv_free(mars_kv_t* kv) {
     if (!kv) return MARS_ERR_BAD_HANDLE;
+    if (kv->copy_stream) cudaStreamDestroy(kv->copy_stream);
     delete kv;
     return MARS_OK;
 }
@@ -466,10 +474,17 @@ mars_status_t mars_kv_free(mars_kv_t* kv) {
 int32_t mars_kv_num_pages(const mars_kv_t* kv) { return kv ? kv->view.n_pages : -1; }
 int32_t mars_kv_free_pages(const mars_kv_t* kv) { return kv ? (int32_t)kv->free_list.size() : -1; }
 
+// Writes entries [first, first + count) of a slot's block-table row.  The copy runs on the cache's own
+// stream and has finished when this returns, so kernels launched afterwards on ANY stream (blocking or
+// not) see the row; a synchronous copy on the default stream would only be ordered against blocking
+// streams.  The entries written are new to the device (pages appended to a slot, or a slot that was
+// empty), so steps still in flight on the caller's stream never read them.
 static mars_status_t upload_row(mars_kv* kv, int seq, int first, int count) {
     if (count <= 0) return MARS_OK;
-    CUDA_TRY(cudaMemcpy(kv->view.block_table + (size_t)seq * kv->view.max_pages_per_seq + first,
-                        kv->seqs[seq].pages.data() + first, (size_t)count * 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpyAsync(kv->view.block_table + (size_t)seq * kv->view.max_pages_per_seq + first,
+                             kv->seqs[seq].pages.data() + first, (size_t)count * 4, cudaMemcpyHostToDevice,
+                             kv->copy_stream));
+    CUDA_TRY(cudaStreamSynchronize(kv->copy_stream));
     return MARS_OK;
 }
 
@@ -968,6 +983,12 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             run(MARS_K_GATE_UP, [&] { return launch_gate_up(s, b, w, n_tok, m->sm_count, st); });
             run(MARS_K_DOWN, [&] { return launch_down(s, b, w, n_tok, st); });
         }
+        if (dbg && dbg->expert_off)      // the permutation's integer outputs, for tests
+            CUDA_TRY(cudaMemcpyAsync(dbg->expert_off + (size_t)l * (s.E + 1), b.expert_off, ((size_t)s.E + 1) * 4,
+                                     cudaMemcpyDeviceToDevice, st));
+        if (dbg && dbg->slot_token)
+            CUDA_TRY(cudaMemcpyAsync(dbg->slot_token + (size_t)l * n_tok * s.k, b.slot_token, (size_t)n_tok * s.k * 4,
+                                     cudaMemcpyDeviceToDevice, st));
         const __nv_bfloat16* next_gain = l + 1 < s.L ? m->layers[l + 1].attn_norm : m->final_norm;
         float* tap = taps.hidden ? taps.hidden + (size_t)(l + 1) * hid_stride : nullptr;
         run(MARS_K_COMBINE, [&] { return launch_combine(s, b, next_gain, tap, n_tok, st); });
@@ -1288,6 +1309,13 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
     if (!sampling->greedy && (!(sampling->temperature > 0.f) || !(sampling->top_p > 0.f) || sampling->top_p > 1.f))
         return MARS_ERR_INVALID_ARG;
     if (!shape_supported(*cfg)) return MARS_ERR_UNSUPPORTED;
+    {   // The call reads ctx_lens on the host and uploads its step block from host memory that dies when it
+        // returns: a captured copy of it would replay stale lengths from freed memory.  Refuse a capturing stream
+        // before anything is enqueued.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        CUDA_TRY(cudaStreamIsCapturing((cudaStream_t)cuda_stream, &cap));
+        if (cap != cudaStreamCaptureStatusNone) return MARS_ERR_UNSUPPORTED;
+    }
     for (int l = 0; l < cfg->n_layers; ++l) {
         const mars_layer_t& s = w->layers[l];
         if (!s.attn_norm || !s.wqkv || !s.wo || !s.mlp_norm || !s.router || !s.w_gate_up || !s.w_down)
@@ -1366,6 +1394,7 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
     // the array keeps the previous call's contents: clear what the kernels only OR into or count in
     CUDA_TRY(cudaMemsetAsync(buf.err, 0, 256, st));
     CUDA_TRY(cudaMemsetAsync(buf.active, 0, (size_t)cfg->n_layers * 4, st));
+    CUDA_TRY(cudaMemsetAsync(buf.perm_cnt, 0, (size_t)cfg->n_experts * 4, st));   // its offset moves with the shape
     CUDA_TRY(cudaMemcpyAsync(buf.step, blk.data(), blk.size() * 4, cudaMemcpyHostToDevice, st));
     CUDA_TRY(cudaMemcpyAsync(buf.inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice, st));
 
@@ -1414,6 +1443,15 @@ mars_status_t mars_poll_status(mars_model_t* m) {
     if (word) CUDA_TRY(cudaMemset(m->buf.err, 0, 4));
     if (word & kErrTimeout) return MARS_ERR_TIMEOUT;
     if (word & kErrBadToken) return MARS_ERR_BAD_TOKEN;
+    return MARS_OK;
+}
+
+mars_status_t mars_debug_bounded_wait(mars_model_t* m, void* cuda_stream, int32_t arrive) {
+    if (!m) return MARS_ERR_BAD_HANDLE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    launch_wait_probe(m->buf.err, arrive ? 1 : 0, 4096u, st);
+    CUDA_TRY(cudaGetLastError());
+    m->last_stream = st;
     return MARS_OK;
 }
 

@@ -18,6 +18,7 @@ TOL_LOGIT_GAP = 1e-2
 TOL_LOGIT_ABS = 2e-2
 TOL_HIDDEN_REL = 1e-2
 TOL_ROUTER_W = 2e-3
+CACHE_ABS_FLOOR = 1e-4   # of the row RMS, on top of one bf16 step (see check_cache_rows)
 
 
 class Case:
@@ -80,14 +81,19 @@ class Case:
                    hidden=torch.empty(L + 1, n, H, dtype=torch.float32, device=dev),
                    router_w=torch.empty(L, n, k, dtype=torch.float32, device=dev),
                    router_idx=torch.empty(L, n, k, dtype=torch.int32, device=dev),
-                   nucleus_mass=torch.empty(n, dtype=torch.float32, device=dev))
+                   nucleus_mass=torch.empty(n, dtype=torch.float32, device=dev),
+                   expert_off=torch.empty(L, m["n_experts"] + 1, dtype=torch.int32, device=dev),
+                   slot_token=torch.empty(L, n * k, dtype=torch.int32, device=dev))
         f = None if forced_idx is None else forced_idx.to(dev).contiguous()
-        dbg = binding.make_debug(out["logits"], out["hidden"], out["router_w"], out["router_idx"], f, out["nucleus_mass"])
+        dbg = binding.make_debug(out["logits"], out["hidden"], out["router_w"], out["router_idx"], f, out["nucleus_mass"],
+                                 out["expert_off"], out["slot_token"])
         smp = binding.make_sampling(seed=seed, step=step, **sampling)
         st = binding.mars_decode_step(self.model, self.kv, ids, tokens.to(dev), smp, out["tokens"], out["logp"], dbg)
         assert st == 0, binding.STATUS_NAMES.get(st, st)
         assert self.model.poll_status() == 0
-        return {k_: v.cpu() for k_, v in out.items()}
+        res = {k_: v.cpu() for k_, v in out.items()}
+        res["active_experts"] = self.model.active_experts()
+        return res
 
     # ------------------------------------------------------------------ oracle side
     def oracle_decode(self, tokens: torch.Tensor, forced_idx=None, seq_ids=None):
@@ -101,12 +107,67 @@ class Case:
         return res
 
 
+def check_cache_rows(got_k, got_v, want_k, want_v, rows, label=""):
+    """The key/value rows written by the step land within one bf16 step of the oracle's.
+
+    got_* / want_*: pools [L, pages, n_kv_heads, page_size, head_dim] (the CUDA path's, the oracle's);
+    rows: (page, slot) of every row to compare.  Both sides round an fp32 value to bf16; the two fp32
+    values differ by the projection's own error (activations travel as (hi, lo) bf16 pairs, sums are
+    fp32: a few 1e-6 of the row's RMS), so the stored values are equal or neighbours:
+    |g - w| <= ulp(w) <= 2^-7 |w|, plus that small absolute error for elements near zero, where an
+    ulp is smaller than it.  Returns the largest excess over one bf16 step, in units of the row RMS."""
+    worst = 0.0
+    for page, slot in rows:
+        for got, want in ((got_k, want_k), (got_v, want_v)):
+            g, w = got[:, page, :, slot].float().cpu(), want[:, page, :, slot].float().cpu()
+            assert torch.isfinite(g).all(), (label, page, slot)
+            rms = w.pow(2).mean(-1, keepdim=True).sqrt()
+            assert ((g - w).norm(dim=-1) <= 4e-3 * w.norm(dim=-1)).all(), (label, page, slot, "row L2")
+            excess = ((g - w).abs() - 0.0079 * w.abs()) / rms
+            worst = max(worst, float(excess.max()))
+            assert (excess <= CACHE_ABS_FLOOR).all(), (label, page, slot, float(excess.max()))
+    return worst
+
+
+def check_cache_append(case: "Case", ctx_before, label=""):
+    """Rows appended by one decode step at positions ctx_before[b] of every sequence b."""
+    rows = [(case.pages[b][c // case.ps], c % case.ps) for b, c in enumerate(ctx_before)]
+    return check_cache_rows(case.k_pool, case.v_pool, case.k_cpu, case.v_cpu, rows, label)
+
+
 def topk_margin(probs: torch.Tensor, k: int) -> torch.Tensor:
     """pi_k - pi_{k+1} of the sorted probabilities (inf when k == E)."""
     s = torch.sort(probs.double(), dim=-1, descending=True).values
     if s.shape[-1] == k:
         return torch.full(s.shape[:-1], float("inf"), dtype=torch.float64)
     return s[..., k - 1] - s[..., k]
+
+
+def check_permutation(gpu: dict, orc: dict, label: str = "") -> dict:
+    """Integer outputs of the token permutation, bit for bit: the exclusive offsets equal the running
+    sum of the histogram of the ORACLE's expert ids (which are the GPU's forced ones, checked against
+    the oracle's own choice by compare_step), every expert's slots list exactly the token rows routed
+    to it (slot order inside an expert is free), and the distinct-expert counter equals the number of
+    experts with at least one token."""
+    oi = orc["router_idx"].long()                        # [L, n, k]
+    L, n, k = oi.shape
+    off, slots = gpu["expert_off"].long(), gpu["slot_token"].long()
+    E = off.shape[1] - 1
+    for l in range(L):
+        cnt = torch.bincount(oi[l].flatten(), minlength=E)
+        want = torch.cat([torch.zeros(1, dtype=torch.long), torch.cumsum(cnt, 0)])
+        assert torch.equal(off[l], want), (label, l, "permutation offsets")
+        rows = torch.arange(n)[:, None].expand(n, k).flatten()
+        order = torch.argsort(oi[l].flatten() * n + rows)            # pairs sorted by (expert, token row)
+        want_rows = rows[order]
+        got = slots[l].clone()
+        for e in range(E):
+            a, b = int(want[e]), int(want[e + 1])
+            got[a:b] = torch.sort(got[a:b]).values
+        assert torch.equal(got, want_rows), (label, l, "tokens listed per expert")
+        if "active_experts" in gpu:
+            assert int(gpu["active_experts"][l]) == int((cnt > 0).sum()), (label, l, "distinct experts")
+    return dict(permute_checked=L)
 
 
 def compare_step(gpu: dict, orc: dict, k: int, greedy: bool, label: str = "") -> dict:
@@ -128,6 +189,8 @@ def compare_step(gpu: dict, orc: dict, k: int, greedy: bool, label: str = "") ->
     stats["routing_checked"] = int((margin >= TOL_ROUTE_MARGIN).sum())
     stats["routing_total"] = L * n
     assert bad == 0, f"{label}: {bad} routing decisions differ where the oracle margin >= {TOL_ROUTE_MARGIN}"
+    if "expert_off" in gpu:
+        stats.update(check_permutation(gpu, orc, label))
     # weights: compare per expert index (order of near-equal entries may differ)
     gi, gw = gpu["router_idx"].long(), gpu["router_w"].double()
     oi, ow = orc["router_idx"].long(), orc["router_w"].double()
@@ -160,13 +223,15 @@ def compare_step(gpu: dict, orc: dict, k: int, greedy: bool, label: str = "") ->
     return stats
 
 
-def compare_sampled(gpu: dict, orc: dict, temperature: float, top_p: float, seed: int, step: int, slots, label=""):
+def compare_sampled(gpu: dict, orc: dict, temperature: float, top_p: float, seed: int, step: int, slots, label="",
+                    logit_err: float | None = None):
     """Nucleus sampling: the GPU's token must lie in the oracle's nucleus (or within the mass the
     logit error can move the edge by) and the oracle's cumulative interval of that token (ascending
     token id over the nucleus) must contain the uniform, within the shift that the measured logit
-    error allows (each probability moves by a factor of at most exp(2 max|dlogit| / T))."""
-    lg, lo = gpu["logits"].double(), orc["logits"].double()
-    err = float((lg - lo).abs().max())
+    error allows (each probability moves by a factor of at most exp(2 max|dlogit| / T)).  An entry
+    point without a logits tap passes the logit error it is allowed (`logit_err`) instead."""
+    lo = orc["logits"].double()
+    err = float((gpu["logits"].double() - lo).abs().max()) if logit_err is None else logit_err
     tol = 2.0 * err / temperature * 2.0 + 1e-6
     stats = dict(cdf_tol=tol, worst=0.0)
     for i, slot in enumerate(slots):
@@ -187,5 +252,50 @@ def compare_sampled(gpu: dict, orc: dict, temperature: float, top_p: float, seed
         assert miss <= tol, (label, i, t, r["token"], lo_t, u, hi_t, tol)
         lp_want = float(torch.log(pi[t]))
         assert abs(float(gpu["logp"][i]) - lp_want) <= TOL_LOGIT_ABS, (label, i)
-        assert abs(float(gpu["nucleus_mass"][i]) - r["nucleus_mass"]) <= max(tol, 1e-4), (label, i)
+        if "nucleus_mass" in gpu:
+            assert abs(float(gpu["nucleus_mass"][i]) - r["nucleus_mass"]) <= max(tol, 1e-4), (label, i)
     return stats
+
+
+def prefill_and_compare(model, ps, ctx, lens, seed, label, check_rows="all"):
+    """One mars_prefill_chunk call over several requests (request r continues ctx[r] cached tokens
+    with lens[r] new ones) against the oracle with the GPU's routing forced: every tap, the
+    permutation's integer outputs and the appended cache rows (all of them, or the first and last
+    of every request).  Returns the case (positions advanced) and the sampled tokens."""
+    n = sum(lens)
+    case = Case(model, ps, ctx, seed=seed, headroom=max(lens) + 4, max_prefill_tokens=n, poison=True)
+    dev = case.device
+    L, H, k, V, E = model["n_layers"], model["hidden"], model["top_k"], model["vocab"], model["n_experts"]
+    toks = wl.make_tokens(n, V, seed=seed + 100)
+    R = len(lens)
+    out_t = torch.empty(R, dtype=torch.int32, device=dev)
+    out_l = torch.empty(R, dtype=torch.float32, device=dev)
+    logits = torch.empty(R, V, dtype=torch.float32, device=dev)
+    hidden = torch.empty(L + 1, n, H, dtype=torch.float32, device=dev)
+    ridx = torch.empty(L, n, k, dtype=torch.int32, device=dev)
+    rw = torch.empty(L, n, k, dtype=torch.float32, device=dev)
+    eoff = torch.empty(L, E + 1, dtype=torch.int32, device=dev)
+    stok = torch.empty(L, n * k, dtype=torch.int32, device=dev)
+    dbg = binding.make_debug(logits, hidden, rw, ridx, expert_off=eoff, slot_token=stok)
+    st = binding.mars_prefill_chunk(case.model, case.kv, list(range(R)), lens, toks.to(dev), [1] * R,
+                                    binding.make_sampling(greedy=1), out_t, out_l, dbg)
+    assert st == 0 and case.model.poll_status() == 0
+    seq = torch.tensor([r for r in range(R) for _ in range(lens[r])], dtype=torch.int32)
+    pos = torch.tensor([ctx[r] + i for r in range(R) for i in range(lens[r])], dtype=torch.int32)
+    orc = oracle.forward(case.ocfg, case.w_cpu, toks, seq, pos, case.k_cpu, case.v_cpu, case.bt, ps,
+                         forced_idx=ridx.cpu().contiguous())
+    last = torch.tensor([sum(lens[: r + 1]) - 1 for r in range(R)])
+    gpu = dict(router_idx=ridx.cpu(), router_w=rw.cpu(), hidden=hidden.cpu(), logits=logits.cpu(), tokens=out_t.cpu(),
+               logp=out_l.cpu(), expert_off=eoff.cpu(), slot_token=stok.cpu(), active_experts=case.model.active_experts())
+    stats = compare_step(gpu, dict(orc, logits=orc["logits"][last]), k, greedy=True, label=label)
+    for r in range(R):
+        assert case.kv.seq_len(r) == ctx[r] + lens[r]
+    rows = []
+    for r in range(R):
+        ts = range(ctx[r], ctx[r] + lens[r]) if check_rows == "all" else sorted({ctx[r], ctx[r] + lens[r] - 1})
+        rows += [(case.pages[r][t // ps], t % ps) for t in ts]
+    stats["cache_excess"] = check_cache_rows(case.k_pool.cpu(), case.v_pool.cpu(), case.k_cpu, case.v_cpu, rows, label)
+    print(label, stats)
+    case.cur = [c + l for c, l in zip(ctx, lens)]
+    case.last_gpu = gpu
+    return case, out_t.cpu()

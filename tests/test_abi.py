@@ -53,11 +53,27 @@ def test_workspace_and_meta_sizes_are_host_only(lib):
     assert 64 * 151936 * 4 < ws < 2 << 30
 
 
+def test_expert_inter_beyond_the_down_kernels_shared_memory_is_unsupported(lib):
+    """The streaming down kernel stages (hi, lo) activation rows of expert_inter elements in shared
+    memory; a size that cannot fit is refused up front, not in mid-step after cache rows were written."""
+    ok = binding.make_config(dict(wl.MODEL_TINY, expert_inter=3136), max_pos=512)
+    assert lib.mars_workspace_bytes(ctypes.byref(ok), 4, 0) > 0
+    big = binding.make_config(dict(wl.MODEL_TINY, expert_inter=3200), max_pos=512)
+    assert lib.mars_workspace_bytes(ctypes.byref(big), 4, 0) == 0
+    fake = ctypes.c_void_p(256)                               # never dereferenced: the shape is checked first
+    layer = binding.mars_layer_t(*[256] * len(binding.LAYER_FIELDS))
+    w = binding.mars_weights_t(fake, fake, fake, ctypes.pointer(layer))
+    out = ctypes.c_void_p()
+    assert lib.mars_model_load(ctypes.byref(big), ctypes.byref(w), fake, 1 << 30, 4, 0, ctypes.byref(out)) == 2
+    assert not out.value
+
+
 def test_null_and_bad_arguments_are_rejected_without_a_device(lib):
     assert lib.mars_model_free(None) == 6
     assert lib.mars_kv_free(None) == 6
     assert lib.mars_kv_seq_len(None, 0) == -1
     assert lib.mars_poll_status(None) == 6
+    assert lib.mars_debug_bounded_wait(None, None, 0) == 6
     out = ctypes.c_void_p()
     cfg = binding.make_config(wl.MODEL_TINY, max_pos=512)
     assert lib.mars_model_load(ctypes.byref(cfg), None, None, 0, 4, 0, ctypes.byref(out)) == 1

@@ -8,7 +8,7 @@ import pytest
 import torch
 
 import oracle
-from harness import compare_sampled, compare_step
+from harness import check_cache_rows, check_permutation, compare_sampled, compare_step
 from paper_2511_11373_b200 import binding, workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -28,11 +28,14 @@ def full_weights():
 
 
 class FullCase:
-    def __init__(self, cfg, weights, steps, seed=0):
+    def __init__(self, cfg, weights, steps, seed=0, page_edge=None):
         self.cfg, self.model, self.ps = cfg, cfg["model"], cfg["page_size"]
         self.weights = weights
         self.ctx, _ = wl.make_context_lengths(cfg, seed=seed)
         self.B = len(self.ctx)
+        if page_edge is not None:       # this sequence's context ends one token short of a page boundary:
+            b = page_edge               # the first step fills the page, the second must take a new one
+            self.ctx[b] = self.ctx[b] - self.ctx[b] % self.ps + self.ps - 1
         cap = [c + steps + 1 for c in self.ctx]
         self.n_pages = sum(wl.pages_needed(c, self.ps) for c in cap) + 4
         self.max_pages = max(wl.pages_needed(c, self.ps) for c in cap) + 1
@@ -41,8 +44,11 @@ class FullCase:
         self.m = binding.Model(self.model, weights, max_decode_seqs=self.B, max_pos=max(cap) + 8)
         self.kv = binding.KvCache(self.m, self.k_pool, self.v_pool, self.ps, self.B, self.max_pages)
         for b in range(self.B):
+            if b == page_edge:          # only the pages its context touches: the library must find the next one itself
+                self.pages[b] = self.pages[b][: wl.pages_needed(self.ctx[b] + 1, self.ps)]
             self.kv.seq_adopt(b, self.pages[b], self.ctx[b])
         self.cur = list(self.ctx)
+        self.page_edge = page_edge
 
     def gpu_step(self, tokens, sampling, step, seed):
         L, H, k, V, n = self.model["n_layers"], self.model["hidden"], self.model["top_k"], self.model["vocab"], self.B
@@ -50,12 +56,21 @@ class FullCase:
                    logits=torch.empty(n, V, device=DEV), hidden=torch.empty(L + 1, n, H, device=DEV),
                    router_w=torch.empty(L, n, k, device=DEV),
                    router_idx=torch.empty(L, n, k, dtype=torch.int32, device=DEV),
-                   nucleus_mass=torch.empty(n, device=DEV))
+                   nucleus_mass=torch.empty(n, device=DEV),
+                   expert_off=torch.empty(L, self.model["n_experts"] + 1, dtype=torch.int32, device=DEV),
+                   slot_token=torch.empty(L, n * k, dtype=torch.int32, device=DEV))
         dbg = binding.make_debug(out["logits"], out["hidden"], out["router_w"], out["router_idx"], None,
-                                 out["nucleus_mass"])
+                                 out["nucleus_mass"], out["expert_off"], out["slot_token"])
         smp = binding.make_sampling(seed=seed, step=step, **sampling)
         st = binding.mars_decode_step(self.m, self.kv, list(range(n)), tokens.to(DEV), smp, out["tokens"], out["logp"], dbg)
         assert st == 0 and self.m.poll_status() == 0
+        # the permutation of the WHOLE batch is consistent with the routing taps, whose subset rows the
+        # oracle checks (offsets, tokens per expert, distinct experts: integer work, bit for bit)
+        whole = dict(expert_off=out["expert_off"].cpu(), slot_token=out["slot_token"].cpu(),
+                     active_experts=self.m.active_experts())
+        check_permutation(whole, dict(router_idx=out["router_idx"].cpu()), label="whole batch")
+        if self.page_edge is not None:  # a page taken from the free list inside the step shows up in the block table
+            self.pages[self.page_edge] = self.kv.block_table(self.page_edge)
         return out
 
     def oracle_subset(self, subset, tokens, gpu_router_idx):
@@ -81,6 +96,12 @@ class FullCase:
             forced = gpu_router_idx[l, subset].contiguous()
             o = oracle.layer_forward(ocfg, layer, x, seq, pos, kp, vp, bt, ps, forced_idx=forced)
             hidden.append(x.clone()); ridx.append(o["router_idx"]); rw.append(o["router_w"]); rp.append(o["router_probs"])
+            # the key / value rows appended at this step: kp / vp were copied from the device after the CUDA step and
+            # the oracle has just overwritten its own rows in them; a fresh copy still holds what the CUDA path stored
+            if l in (0, model["n_layers"] // 2, model["n_layers"] - 1):
+                rows = [(int(bt[i, self.cur[b] // ps]), self.cur[b] % ps) for i, b in enumerate(subset)]
+                okp, ovp = self.k_pool[l, flat].cpu(), self.v_pool[l, flat].cpu()
+                check_cache_rows(okp[None], ovp[None], kp[None], vp[None], rows, label=f"layer {l} appended rows")
         logits = oracle.lm_head(ocfg.__class__(**model), self.weights["final_norm"].cpu(), self.weights["lm_head"].cpu(), x)
         return dict(hidden=torch.stack(hidden), router_idx=torch.stack(ridx), router_w=torch.stack(rw),
                     router_probs=torch.stack(rp), logits=logits)
@@ -94,14 +115,24 @@ def take(gpu, subset):
 
 
 def test_config3_full_model_decode_top_p(full_weights):
+    """Step 0 is checked on 8 of the 64 sequences (spread over the sorted context lengths), step 1 on 3.
+    One checked sequence ends one token short of a 64-token page and owns no page beyond it: step 0
+    fills the page, step 1 makes the library take a new page from the free list inside the step."""
     cfg = wl.CONFIGS[3]
-    case = FullCase(cfg, full_weights, steps=2)
+    ctx0, _ = wl.make_context_lengths(cfg, seed=wl.CONFIG3_CONTEXT_SEED)
+    order = sorted(range(len(ctx0)), key=lambda b: ctx0[b])
+    edge = order[len(order) // 2]
+    case = FullCase(cfg, full_weights, steps=2, seed=wl.CONFIG3_CONTEXT_SEED, page_edge=edge)
+    assert case.ctx[edge] % 64 == 63
     tokens = wl.make_tokens(case.B, cfg["model"]["vocab"], seed=0)
     smp = dict(greedy=0, temperature=1.0, top_p=0.95)
-    order = sorted(range(case.B), key=lambda b: case.ctx[b])
-    subset = [order[0], order[len(order) // 2], order[-1]]          # shortest, median, longest context
-    for step in range(2):
+    eight = [order[i] for i in (0, 9, 18, 27, 32, 45, 54, 63)]      # includes the shortest, the edge one and the longest
+    assert edge in eight
+    for step, subset in enumerate((eight, [order[0], edge, order[-1]])):
+        free_before = case.kv.free_pages
         gpu = case.gpu_step(tokens, smp, step=step, seed=7)
+        if step == 1:
+            assert case.kv.free_pages == free_before - 1 and case.cur[edge] % 64 == 0    # the in-step page grab
         orc = case.oracle_subset(subset, tokens, gpu["router_idx"].cpu())
         g = take(gpu, subset)
         stats = compare_step(g, orc, cfg["model"]["top_k"], greedy=False, label=f"config3 step {step}")
@@ -127,8 +158,8 @@ def test_config5_long_context_decode_greedy(full_weights):
         pytest.skip(f"not enough free device memory for the 16 x 64k cache ({free >> 30} GiB free)")
     case = FullCase(cfg, full_weights, steps=2)
     tokens = wl.make_tokens(case.B, model["vocab"], seed=5)
-    subset = [3]
     for step in range(2):
+        subset = [3, 12] if step == 0 else [3]
         gpu = case.gpu_step(tokens, dict(greedy=1, temperature=1.0, top_p=1.0), step=step, seed=0)
         orc = case.oracle_subset(subset, tokens, gpu["router_idx"].cpu())
         stats = compare_step(take(gpu, subset), orc, model["top_k"], greedy=True, label=f"config5 step {step}")
@@ -143,9 +174,11 @@ def test_config5_long_context_decode_greedy(full_weights):
 
 def test_config4_mixed_batch_decode_and_prefill(full_weights):
     """192 decode sequences (lognormal contexts by stage) plus chunked prefill on the 48-layer model.
-    The decode step is checked against the oracle on three sequences.  Prefill: a 96-token chunk
-    that continues a cached context is checked against the oracle token by token (a 2048-token
-    chunk would cost the CPU oracle tens of minutes); the full 8 x 2048 call of the benchmark is
+    The decode step is checked against the oracle on three sequences.  Prefill: a 264-token chunk
+    that continues a cached context -- more than 256 rows, so it runs on the dense tensor-core
+    contractions and the tensor-core causal attention like the benchmark's call -- is checked against
+    the oracle token by token through all 48 layers (a 2048-token chunk would cost the CPU oracle
+    tens of minutes); the full 8 x 2048 call of the benchmark is
     checked by a property that holds at any size: one call of 2048 tokens and two calls of 1024
     give the same last-position logits and the same sampled token."""
     cfg = wl.CONFIGS[4]
@@ -184,9 +217,9 @@ def test_config4_mixed_batch_decode_and_prefill(full_weights):
     assert torch.isfinite(gpu["hidden"]).all()
     del gpu
 
-    # --- prefill, oracle-checked: 96 tokens continuing 40 cached tokens of a fresh slot
+    # --- prefill, oracle-checked: 264 tokens (> 256: the dense tcgen05 path) continuing 40 cached tokens of a fresh slot
     L, H, k, V = model["n_layers"], model["hidden"], model["top_k"], model["vocab"]
-    slot, prior, n = B, 40, 96
+    slot, prior, n = B, 40, 264
     kv.seq_adopt(slot, pages[slot], prior)
     ptoks = wl.make_tokens(n, V, seed=9, name="prompt")
     out_t = torch.empty(1, dtype=torch.int32, device=DEV)
@@ -228,7 +261,7 @@ def test_config4_mixed_batch_decode_and_prefill(full_weights):
     slp = torch.empty(n, device=DEV)
     st = binding.mars_score_chunk(m, kv, [slot], [n], ptoks.to(DEV), tgt.to(DEV), 0.85, slp)
     assert st == 0 and m.poll_status() == 0
-    rows = [0, 17, 50, n - 1]
+    rows = [0, 17, 150, n - 1]
     olog = oracle.lm_head(oracle.Config(**model), full_weights["final_norm"].cpu(), full_weights["lm_head"].cpu(),
                           x[torch.tensor(rows)].contiguous())
     werr = max(abs(float(slp[r]) - oracle.logprob_of(olog[i].contiguous(), 0.85, int(tgt[r]))) for i, r in enumerate(rows))

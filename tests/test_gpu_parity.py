@@ -3,7 +3,7 @@ import pytest
 import torch
 
 import oracle
-from harness import Case, compare_sampled, compare_step
+from harness import Case, check_cache_append, compare_sampled, compare_step, prefill_and_compare
 from paper_2511_11373_b200 import binding, workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -21,22 +21,6 @@ def run_and_compare(case: Case, tokens, sampling=GREEDY, label="", step=0, seed=
         stats.update(compare_sampled(gpu, orc, sampling["temperature"], sampling["top_p"], seed, step,
                                      list(range(case.B)), label))
     return gpu, orc, stats
-
-
-def check_cache_append(case: Case, ctx_before):
-    """The new key/value rows written by the step equal the oracle's within one bf16 step."""
-    kg, vg = case.k_pool.cpu(), case.v_pool.cpu()
-    for b, c in enumerate(ctx_before):
-        page, slot = case.pages[b][c // case.ps], c % case.ps
-        for got, want in ((kg, case.k_cpu), (vg, case.v_cpu)):
-            g, w = got[:, page, :, slot].float(), want[:, page, :, slot].float()
-            assert torch.isfinite(g).all()
-            # both sides round to bf16 values that differ by the projection's own error (activations
-            # are bf16 on the GPU): relative L2 per head row as for hidden states, plus an elementwise
-            # bound of one bf16 step and 2% of the row's RMS
-            rms = w.pow(2).mean(-1, keepdim=True).sqrt()
-            assert ((g - w).norm(dim=-1) <= 1e-2 * w.norm(dim=-1)).all(), (b, "row L2")
-            assert ((g - w).abs() <= 0.0079 * w.abs() + 0.02 * rms).all(), (b, float((g - w).abs().max()))
 
 
 # ------------------------------------------------------------------ config 1: tiny single layer
@@ -228,6 +212,23 @@ def test_error_paths_leave_state_unchanged():
     assert case.model.poll_status() == 0 and case.kv.seq_len(0) == 17
 
 
+def test_bounded_wait_gives_up_and_the_handle_stays_usable():
+    """Every TMA / tensor-core wait is bounded; when its limit is reached the kernel sets the timeout
+    bit, frees its tensor memory and returns.  The library's self-test block takes that path with an
+    arrival that never comes: the status is MARS_ERR_TIMEOUT once, then clear, and a decode step on the
+    same handle still matches the oracle.  Nothing hangs, traps or faults."""
+    model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=1)
+    case = Case(model, 16, [20, 77], seed=12)
+    assert case.model.bounded_wait_selftest(arrive=True) == 0
+    assert case.model.poll_status() == 0                     # the arrival came: nothing to report
+    assert case.model.bounded_wait_selftest(arrive=False) == 0
+    assert case.model.poll_status() == 5                     # the wait ran out
+    assert case.model.poll_status() == 0                     # reading clears the word
+    tokens = wl.make_tokens(2, model["vocab"], seed=6)
+    run_and_compare(case, tokens, label="decode after a timed-out wait")
+    check_cache_append(case, [20, 77])
+
+
 def test_library_allocator_path_matches_adopted_pages():
     """Pages handed out by the library's own free list give the same results as caller-chosen ones."""
     model = dict(wl.MODEL_TINY, n_layers=1)
@@ -250,47 +251,6 @@ def test_library_allocator_path_matches_adopted_pages():
     gb = b.gpu_decode(tokens, GREEDY)
     assert torch.equal(ga["logits"], gb["logits"])
     assert len(b.kv.block_table(1)) == 2
-
-
-def prefill_and_compare(model, ps, ctx, lens, seed, label):
-    """One mars_prefill_chunk call over several requests (each continuing its cached context)
-    against the oracle with the GPU's routing forced; returns the case for follow-up steps."""
-    n = sum(lens)
-    case = Case(model, ps, ctx, seed=seed, headroom=max(lens) + 4, max_prefill_tokens=n, poison=True)
-    dev = case.device
-    L, H, k, V = model["n_layers"], model["hidden"], model["top_k"], model["vocab"]
-    toks = wl.make_tokens(n, V, seed=seed + 100)
-    R = len(lens)
-    out_t = torch.empty(R, dtype=torch.int32, device=dev)
-    out_l = torch.empty(R, dtype=torch.float32, device=dev)
-    logits = torch.empty(R, V, dtype=torch.float32, device=dev)
-    hidden = torch.empty(L + 1, n, H, dtype=torch.float32, device=dev)
-    ridx = torch.empty(L, n, k, dtype=torch.int32, device=dev)
-    rw = torch.empty(L, n, k, dtype=torch.float32, device=dev)
-    dbg = binding.make_debug(logits, hidden, rw, ridx)
-    st = binding.mars_prefill_chunk(case.model, case.kv, list(range(R)), lens, toks.to(dev), [1] * R,
-                                    binding.make_sampling(greedy=1), out_t, out_l, dbg)
-    assert st == 0 and case.model.poll_status() == 0
-    seq = torch.tensor([r for r in range(R) for _ in range(lens[r])], dtype=torch.int32)
-    pos = torch.tensor([ctx[r] + i for r in range(R) for i in range(lens[r])], dtype=torch.int32)
-    orc = oracle.forward(case.ocfg, case.w_cpu, toks, seq, pos, case.k_cpu, case.v_cpu, case.bt, ps,
-                         forced_idx=ridx.cpu().contiguous())
-    last = torch.tensor([sum(lens[: r + 1]) - 1 for r in range(R)])
-    gpu = dict(router_idx=ridx.cpu(), router_w=rw.cpu(), hidden=hidden.cpu(), logits=logits.cpu(), tokens=out_t.cpu(),
-               logp=out_l.cpu())
-    stats = compare_step(gpu, dict(orc, logits=orc["logits"][last]), k, greedy=True, label=label)
-    print(label, stats)
-    for r in range(R):
-        assert case.kv.seq_len(r) == ctx[r] + lens[r]
-    # the appended cache rows of every request agree with the oracle's
-    kg = case.k_pool.cpu()
-    for r in range(R):
-        for t in (ctx[r], ctx[r] + lens[r] - 1):
-            page, slot = case.pages[r][t // ps], t % ps
-            g, w = kg[:, page, :, slot].float(), case.k_cpu[:, page, :, slot].float()
-            assert ((g - w).norm(dim=-1) <= 1e-2 * w.norm(dim=-1)).all()
-    case.cur = [c + l for c, l in zip(ctx, lens)]
-    return case, out_t.cpu()
 
 
 def test_prefill_small_chunks_use_the_causal_kernel():
@@ -328,6 +288,23 @@ def test_prefill_attention_on_tensor_cores(ps):
     case, toks = prefill_and_compare(MODEL_GQA8, ps, [0, 21, 128, 300, 64], [70, 33, 150, 1, 64], seed=24 + ps,
                                      label=f"prefill-tcgen05-attention ps={ps}")
     run_and_compare(case, toks, label="decode after tcgen05 prefill attention")
+
+
+def test_prefill_tensor_core_path_at_the_full_layer_shape():
+    """The dense tcgen05 path at the shape it runs in the mixed benchmark (hidden 2048, 32 / 4 heads of
+    128, 128 experts top-8, expert_inter 768, per-head norm on, perturbed gains) with more than 256
+    token rows in one call: the QKV contraction with norm, RoPE and cache append in its epilogue over
+    20 column tiles, the output projection (8 tiles), the router logits as a contraction, the grouped
+    gate/up (6 tiles) and down (8 tiles) contractions with groups of every expert id, the causal
+    attention on tcgen05 and, from 4096 (token, expert) pairs on, the multi-block permutation.
+    Chunks continue contexts that start at 0, inside a page, on a page boundary and at a single
+    token; every tap and every appended cache row is compared with the oracle."""
+    case, toks = prefill_and_compare(wl.MODEL_LAYER, 64, [0, 37, 512, 129], [300, 150, 70, 1], seed=61,
+                                     label="prefill-full-shape-521")
+    assert len(set(case.last_gpu["router_idx"].flatten().tolist())) == wl.MODEL_LAYER["n_experts"]
+    run_and_compare(case, toks, label="decode after the full-shape prefill")
+    # 4096 pairs and more: the expert slots are counted and handed out by many blocks
+    prefill_and_compare(wl.MODEL_LAYER, 64, [0, 64], [400, 240], seed=62, label="prefill-full-shape-640")
 
 
 def test_prefill_in_two_calls_equals_one_call():

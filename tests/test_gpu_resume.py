@@ -186,3 +186,95 @@ def test_fork_at_a_page_boundary_and_without_free_pages():
     kv.seq_release(1)                                         # one page comes back: enough for one of the two
     assert binding.mars_decode_step(case.model, kv, [0], tok, binding.make_sampling(greedy=1), out_t, out_l) == 0
     assert case.model.poll_status() == 0 and kv.seq_len(0) == 33 and kv.seq_len(2) == 32
+
+
+def _slice_rows(d, rows, per_row=("tokens", "logp", "logits", "nucleus_mass")):
+    """Rows `rows` of a result dict (taps are [L, n, ...], outputs [n, ...])."""
+    idx = torch.tensor(rows)
+    out = {}
+    for key, v in d.items():
+        if key in ("expert_off", "slot_token", "active_experts"):
+            continue
+        out[key] = v[idx] if key in per_row else v[:, idx]
+    return out
+
+
+def test_resumed_sequences_match_the_oracle():
+    """Section 2.3 (segment rollouts): the first decode step of the next segment is compared with the
+    CPU oracle run over the whole prefix, for a slot that kept its pages, a slot restored from a host
+    image into other pages, and a slot whose prefix was prefilled again.  The oracle is teacher-forced
+    with the tokens of the first segment and, by the cascade rule, with the routing the CUDA path took
+    at every position of the prefix (the prefill call's and the decode steps' taps for the kept slots;
+    the re-prefill's own taps for the third)."""
+    import oracle
+    from harness import compare_step
+    model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=1)
+    ps, P, N1 = 16, 45, 7
+    L, H, k, V, E = model["n_layers"], model["hidden"], model["top_k"], model["vocab"], model["n_experts"]
+    case = Case(model, ps, [0, 0, 0], seed=43, headroom=P + N1 + 4, spare_pages=12, poison=False,
+                max_prefill_tokens=3 * (P + N1), extra_seqs=1)
+    kv, dev = case.kv, case.device
+
+    def prefill_taps(slots, tokens):
+        n, R = len(tokens) * len(slots), len(slots)
+        out = dict(tokens=torch.empty(R, dtype=torch.int32, device=dev), logp=torch.empty(R, device=dev),
+                   logits=torch.empty(R, V, device=dev), hidden=torch.empty(L + 1, n, H, device=dev),
+                   router_w=torch.empty(L, n, k, device=dev), router_idx=torch.empty(L, n, k, dtype=torch.int32, device=dev))
+        dbg = binding.make_debug(out["logits"], out["hidden"], out["router_w"], out["router_idx"])
+        st = binding.mars_prefill_chunk(case.model, kv, slots, [len(tokens)] * R, tokens.repeat(R).to(dev), [1] * R,
+                                        binding.make_sampling(greedy=1), out["tokens"], out["logp"], dbg)
+        assert st == 0 and case.model.poll_status() == 0
+        return {key: v.cpu() for key, v in out.items()}
+
+    # ---- first segment on slots 0 and 1: prompt, then N1 greedy steps; the taps of slot 0 are kept
+    prompt = wl.make_tokens(P, V, seed=91)
+    pf = prefill_taps([0, 1], prompt)
+    generated = [int(pf["tokens"][0])]
+    ridx_a, hid_a = [pf["router_idx"][:, :P]], [pf["hidden"][:, :P]]
+    for step in range(N1):
+        g = case.gpu_decode(torch.tensor([generated[-1]] * 2, dtype=torch.int32), GREEDY, seq_ids=[0, 1], step=step)
+        ridx_a.append(g["router_idx"][:, :1]); hid_a.append(g["hidden"][:, :1])
+        generated.append(int(g["tokens"][0]))
+    n_cached = P + N1
+    prefix = torch.cat([prompt, torch.tensor(generated[:N1], dtype=torch.int32)])
+
+    # ---- slot 1 goes through a host image into other pages; slot 2 prefills the prefix again
+    image = torch.empty(kv.seq_image_bytes(n_cached), dtype=torch.uint8).pin_memory()
+    assert kv.seq_export(1, image) == 0
+    old_pages = kv.block_table(1)
+    kv.seq_release(1)
+    torch.cuda.synchronize()
+    kv.seq_reserve(3, len(old_pages) * ps)
+    idx = torch.tensor(old_pages, device=dev)
+    case.k_pool[:, idx] = float("nan"); case.v_pool[:, idx] = float("nan")
+    assert kv.seq_import(1, image, n_cached) == 0
+    pf2 = prefill_taps([2], prefix)
+
+    # ---- oracle over the prefix, once per routing history
+    seq0, pos = torch.zeros(n_cached, dtype=torch.int32), torch.arange(n_cached, dtype=torch.int32)
+    bt = case.bt[:1].contiguous()
+    def oracle_prefix(forced):
+        kc, vc = case.k_cpu.clone(), case.v_cpu.clone()
+        res = oracle.forward(case.ocfg, case.w_cpu, prefix, seq0, pos, kc, vc, bt, ps, forced_idx=forced.contiguous())
+        return res, kc, vc
+    forced_a = torch.cat(ridx_a, dim=1)
+    orc_a, k_a, v_a = oracle_prefix(forced_a)
+    orc_b, k_b, v_b = oracle_prefix(pf2["router_idx"])
+    # the prefix itself: hidden states of every position on both histories, and the re-prefill's output
+    for name, got, orc in (("kept", torch.cat(hid_a, dim=1), orc_a), ("re-prefilled", pf2["hidden"], orc_b)):
+        rel = (got.double() - orc["hidden"].double()).norm(dim=-1) / orc["hidden"].double().norm(dim=-1).clamp_min(1e-30)
+        assert float(rel.max()) <= 1e-2, (name, float(rel.max()))
+    stats = compare_step(pf2, dict(orc_b, logits=orc_b["logits"][-1:]), k, greedy=True, label="re-prefill of the prefix")
+    print("resume: re-prefill vs oracle", stats)
+
+    # ---- the first step of the next segment, row by row against the oracle
+    tok = torch.tensor([generated[N1]] * 3, dtype=torch.int32)
+    g = case.gpu_decode(tok, GREEDY, seq_ids=[0, 1, 2], step=N1)
+    assert torch.equal(g["logits"][0], g["logits"][1]), "restored pages changed the result"
+    one = torch.tensor([n_cached], dtype=torch.int32)
+    for row, (kc, vc) in ((0, (k_a, v_a)), (1, (k_a, v_a)), (2, (k_b, v_b))):
+        gr = _slice_rows(g, [row])
+        o = oracle.forward(case.ocfg, case.w_cpu, tok[:1].contiguous(), seq0[:1].contiguous(), one, kc.clone(), vc.clone(), bt, ps,
+                           forced_idx=gr["router_idx"].contiguous())
+        stats = compare_step(gr, o, k, greedy=True, label=f"resumed row {row}")
+        print("resume: row", row, stats)

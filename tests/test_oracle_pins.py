@@ -51,6 +51,14 @@ def test_logprobs_exponentiate_to_one_and_greedy_closed_form():
     for T in (1.0, 0.6, 0.85):
         tot = sum(math.exp(oracle.logprob_of(logits, T, v)) for v in range(V))
         assert abs(tot - 1) < 1e-5
+    # the temperature divides the logits (R-10): library log-softmax of logits / T, entry by entry.
+    # A function that ignored T, or multiplied by it, still sums to one above but fails here.
+    for T in (0.6, 0.85, 1.0, 1.7):
+        want = torch.log_softmax(logits.double() / T, 0)
+        for v in (0, 1, 17, 50, V - 1, int(torch.argmax(logits)), int(torch.argmin(logits))):
+            assert abs(oracle.logprob_of(logits, T, v) - want[v].item()) < 2e-6, (T, v)
+    sharp, flat = oracle.logprob_of(logits, 0.6, int(torch.argmax(logits))), oracle.logprob_of(logits, 1.7, int(torch.argmax(logits)))
+    assert sharp > flat                                                  # a lower temperature sharpens the mode
     g = oracle.sample(logits, 0.7, 0.9, True, 0.3)
     assert g["token"] == int(torch.argmax(logits))
     lse = torch.logsumexp(logits.double(), 0).item()
