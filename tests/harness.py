@@ -18,7 +18,7 @@ TOL_LOGIT_GAP = 1e-2
 TOL_LOGIT_ABS = 2e-2
 TOL_HIDDEN_REL = 1e-2
 TOL_ROUTER_W = 2e-3
-CACHE_ABS_FLOOR = 1e-4   # of the row RMS, on top of one bf16 step (see check_cache_rows)
+CACHE_FLOOR_FIRST, CACHE_FLOOR_DEEP = 2e-5, 1e-3   # of the row RMS, on top of one bf16 step (see check_cache_rows)
 
 
 class Case:
@@ -107,16 +107,26 @@ class Case:
         return res
 
 
-def check_cache_rows(got_k, got_v, want_k, want_v, rows, label=""):
-    """The key/value rows written by the step land within one bf16 step of the oracle's.
+def check_cache_rows(got_k, got_v, want_k, want_v, rows, label="", first_layer=0):
+    """The key/value rows written by the step against the oracle's, element by element.
 
     got_* / want_*: pools [L, pages, n_kv_heads, page_size, head_dim] (the CUDA path's, the oracle's);
-    rows: (page, slot) of every row to compare.  Both sides round an fp32 value to bf16; the two fp32
-    values differ by the projection's own error (activations travel as (hi, lo) bf16 pairs, sums are
-    fp32: a few 1e-6 of the row's RMS), so the stored values are equal or neighbours:
-    |g - w| <= ulp(w) <= 2^-7 |w|, plus that small absolute error for elements near zero, where an
-    ulp is smaller than it.  Returns the largest excess over one bf16 step, in units of the row RMS."""
+    rows: (page, slot) of every row to compare; first_layer: model layer of pool index 0.
+    Both sides round an fp32 / fp64 value to bf16, so stored values are equal or neighbours wherever
+    the two pre-rounding values agree to well below an ulp: |g - w| <= ulp(w) <= 2^-7 |w|.  On top of
+    that one bf16 step an absolute part, in units of the row's RMS, covers elements near zero, where an
+    ulp is smaller than the pre-rounding difference:
+      layer 0     CACHE_FLOOR_FIRST: the layer's input is the embedding (exact), so only the projection's
+                  own error remains -- (hi, lo) activation pairs, fp32 sums; 7e-6 measured;
+      deeper      CACHE_FLOOR_DEEP: the layer's input already differs, because a key or value that one side
+                  rounded up and the other down (a fraction ~ error / ulp of all elements) is off by a whole
+                  bf16 step, which attention over few or all-new keys (short contexts, prefill chunks)
+                  passes on: 1e-4 .. 4e-4 of the RMS measured after one layer and in the middle of the
+                  48-layer model.  Still 10 times inside the 1e-2 hidden-state tolerance.
+    Returns the largest excess over one bf16 step, in units of the row RMS."""
     worst = 0.0
+    L = got_k.shape[0]
+    floor = torch.tensor([CACHE_FLOOR_FIRST if first_layer + l == 0 else CACHE_FLOOR_DEEP for l in range(L)])[:, None, None]
     for page, slot in rows:
         for got, want in ((got_k, want_k), (got_v, want_v)):
             g, w = got[:, page, :, slot].float().cpu(), want[:, page, :, slot].float().cpu()
@@ -125,7 +135,7 @@ def check_cache_rows(got_k, got_v, want_k, want_v, rows, label=""):
             assert ((g - w).norm(dim=-1) <= 4e-3 * w.norm(dim=-1)).all(), (label, page, slot, "row L2")
             excess = ((g - w).abs() - 0.0079 * w.abs()) / rms
             worst = max(worst, float(excess.max()))
-            assert (excess <= CACHE_ABS_FLOOR).all(), (label, page, slot, float(excess.max()))
+            assert (excess <= floor).all(), (label, page, slot, float(excess.max()), float(excess[0].max()))
     return worst
 
 

@@ -101,7 +101,7 @@ class FullCase:
             if l in (0, model["n_layers"] // 2, model["n_layers"] - 1):
                 rows = [(int(bt[i, self.cur[b] // ps]), self.cur[b] % ps) for i, b in enumerate(subset)]
                 okp, ovp = self.k_pool[l, flat].cpu(), self.v_pool[l, flat].cpu()
-                check_cache_rows(okp[None], ovp[None], kp[None], vp[None], rows, label=f"layer {l} appended rows")
+                check_cache_rows(okp[None], ovp[None], kp[None], vp[None], rows, label=f"layer {l} appended rows", first_layer=l)
         logits = oracle.lm_head(ocfg.__class__(**model), self.weights["final_norm"].cpu(), self.weights["lm_head"].cpu(), x)
         return dict(hidden=torch.stack(hidden), router_idx=torch.stack(ridx), router_w=torch.stack(rw),
                     router_probs=torch.stack(rp), logits=logits)
@@ -202,6 +202,7 @@ def test_config4_mixed_batch_decode_and_prefill(full_weights):
     case.cfg, case.model, case.ps, case.weights = cfg, model, ps, full_weights
     case.ctx, case.B, case.pages, case.k_pool, case.v_pool, case.m, case.kv = ctx, B, pages, k_pool, v_pool, m, kv
     case.cur = list(ctx)
+    case.page_edge = None
 
     # --- decode part
     tokens = wl.make_tokens(B, model["vocab"], seed=4)

@@ -35,8 +35,10 @@ def static_step(case, model, ps, bt, ctx_now, tokens, sampling):
 def test_static_scratch_step_matches_regular_step_and_oracle_twice():
     model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=1)
     ctx, ps, steps = [15, 40, 130, 600], 16, 2         # 15 -> 16 crosses a page boundary; 600 spans two work items
-    ref = Case(model, ps, ctx, seed=13, headroom=steps)
-    sta = Case(model, ps, ctx, seed=13, headroom=steps)  # same bytes, its own pools for the static call to append to
+    # seed 24: every gate of both steps has a top-k margin >= 5e-3 in the oracle (seeds with a near-tie would make
+    # the unforced oracle a coin toss against any implementation)
+    ref = Case(model, ps, ctx, seed=24, headroom=steps)
+    sta = Case(model, ps, ctx, seed=24, headroom=steps)  # same bytes, its own pools for the static call to append to
     dev = ref.device
     bt = sta.bt.to(dev)
     T, top_p, seed = 0.85, 0.95, 99
