@@ -117,7 +117,7 @@ class DecodeWorkload:
     """Builds a config (weights, cache, page tables) on one GPU and steps it through the C ABI."""
 
     def __init__(self, cfg: dict, total_steps: int, device: torch.device, seed: int = 0, prefill_reqs: int = 0,
-                 prefill_chunk: int = 0):
+                 prefill_chunk: int = 0, weights: dict | None = None):
         from paper_2511_11373_b200 import binding
         self.binding = binding
         self.cfg, self.device = cfg, device
@@ -133,7 +133,7 @@ class DecodeWorkload:
         max_pages = max(wl.pages_needed(c, ps) for c in cap + [prefill_chunk]) + 1
         free, _ = torch.cuda.mem_get_info(device)
         t0 = time.time()
-        self.weights = wl.make_weights(model, seed=seed, device=device, gains="ones")
+        self.weights = weights if weights is not None else wl.make_weights(model, seed=seed, device=device, gains="ones")
         self.k_pool, self.v_pool = wl.make_kv_pools(model, n_pages, ps, seed=seed, device=device)
         torch.cuda.synchronize(device)
         self.setup_s = time.time() - t0
@@ -173,6 +173,14 @@ class DecodeWorkload:
 
     def kv_tokens_now(self) -> int:
         return sum(self.kv.seq_len(b) for b in range(self.B))
+
+    def release_cache(self):
+        """Frees the cache pools and the library handles (the weights stay, for the next configuration)."""
+        torch.cuda.synchronize(self.device)
+        self.kv.close()
+        self.model.close()
+        del self.k_pool, self.v_pool, self.kv, self.model
+        torch.cuda.empty_cache()
 
 
 # ----------------------------------------------------------------------------------- CPU baseline
@@ -265,16 +273,14 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def run_mixed(args):
+def measure_mixed(cfg: dict, args, device, weights=None) -> dict:
     """Config 4: one chunked-prefill call (8 fresh prompts of 2048 tokens) followed by one decode step
-    over 192 sequences = one mixed step.  Prints decode-only against the HBM roofline, prefill-only
+    over 192 sequences = one mixed step.  Returns decode-only against the HBM roofline, prefill-only
     against the bf16 tensor peak, the pair, and the same work as one fused call (mars_mixed_step)."""
     from paper_2511_11373_b200 import binding
-    device = torch.device("cuda", 0)
-    torch.cuda.set_device(device)
-    cfg = wl.CONFIGS[args.workload]
     pf = cfg["prefill"]
-    w = DecodeWorkload(cfg, 3 * (args.warmup + args.steps) + 16, device, prefill_reqs=pf["requests"], prefill_chunk=pf["chunk"])
+    w = DecodeWorkload(cfg, 3 * (args.warmup + args.steps) + 16, device, prefill_reqs=pf["requests"], prefill_chunk=pf["chunk"],
+                       weights=weights)
     model = cfg["model"]
     n_pf = pf["requests"] * pf["chunk"]
     toks = wl.make_tokens(n_pf, model["vocab"], seed=1, name="prompts").to(device)
@@ -352,7 +358,8 @@ def run_mixed(args):
     flops = per_tok * n_pf + attn
     pf_ms, dec_ms = statistics.median(t_pf), statistics.median(t_dec)
     dec_bytes = algorithmic_bytes(model, w.kv_tokens_now(), active)
-    line = dict(metric=METRIC, value=w.B / (dec_ms / 1e3), unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
+    w.release_cache()
+    return dict(metric=METRIC, value=w.B / (dec_ms / 1e3), unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
                 ms_per_step=pf_ms + dec_ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic",
                 config=dict(workload=cfg["name"], decode_seqs=w.B, prefill_requests=pf["requests"], prefill_chunk=pf["chunk"],
@@ -365,7 +372,42 @@ def run_mixed(args):
                              achieved_tflops=flops / (pf_ms * 1e-3) / 1e12, frac_of_measured_bf16=flops / (pf_ms * 1e-3) / 1e12 / tflops_peak,
                              note="activations are (hi, lo) bf16 pairs: the tensor cores execute twice the algorithmic flops in the projections"),
                 mixed_ms=pf_ms + dec_ms, fused_mixed_step_ms=fused_ms, prefill_ms_by_class=pf_classes)
-    print(json.dumps(line))
+
+
+def run_mixed(args):
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    print(json.dumps(measure_mixed(wl.CONFIGS[args.workload], args, device)))
+
+
+def measure_decode(cfg: dict, steps: int, warmup: int, device, weights) -> dict:
+    """Decode-only timing of another configuration on the same weights (device-resident inputs, CUDA events on
+    the launching stream, clocks sampled during the timed steps)."""
+    w = DecodeWorkload(cfg, warmup + steps + 2, device, weights=weights)
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        w.step()
+    torch.cuda.synchronize()
+    kv0 = w.kv_tokens_now()
+    sampler = ClockSampler(device.index or 0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        w.step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    assert w.model.poll_status() == 0
+    ms = e0.elapsed_time(e1) / steps
+    active = w.model.active_experts().tolist()
+    by = algorithmic_bytes(cfg["model"], kv0 + w.B * (steps + 1) // 2, active)
+    peaks = load_peaks()
+    out = dict(workload=cfg["name"], batch=w.B, steps=steps, warmup=warmup, ms_per_step=ms, tokens_per_s=w.B / (ms / 1e3),
+               context_tokens=kv0, bytes_per_step=by["total"], achieved_gbs=by["total"] / (ms * 1e-3) / 1e9,
+               frac_of_measured_hbm=by["total"] / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+               active_experts_mean=sum(active) / len(active), clocks=clocks, setup_s=round(w.setup_s, 1))
+    w.release_cache()
+    return out
 
 
 def run_grouped(args):
@@ -522,8 +564,9 @@ def run_cuda(args):
             if name in per_launch:
                 kernels[name]["achieved_gbs"] = per_launch[name] / (kms / n * 1e-3) / 1e9
     top = max(per_launch, key=lambda k: kernels.get(k, {}).get("ms_per_step", 0.0))
-    # DRAM traffic per launch: ncu counters of a one-layer capture (profiles/decode_one_layer_b64_top_kernels.md),
-    # scaled to this launch by the units processed (traffic grows in proportion to the bytes streamed)
+    # DRAM traffic per launch: dram read + write bytes of this kernel in an ncu capture of the one-layer workload
+    # (64 sequences, contexts U[1k, 16k]), as a ratio to that launch's algorithmic bytes, scaled to this launch by
+    # the units processed (traffic grows in proportion to the bytes streamed)
     traffic = per_launch[top] * NCU_TRAFFIC_RATIO[top] if top in NCU_TRAFFIC_RATIO else None
     roofline = dict(bound="hbm", kernel=top, achieved=kernels[top]["achieved_gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
                     frac=kernels[top]["achieved_gbs"] / peaks["hbm_gbs"], traffic=traffic, peak_source=peaks["source"],
@@ -531,12 +574,30 @@ def run_cuda(args):
 
     if rank != 0:
         return
+    # the other full-model configurations on the same weights (one GPU, default workload only): config 5 (16 x 64k,
+    # greedy) decode-only, config 4 (192 sequences + 8 x 2048 prompt tokens) decode / prefill / both / fused
+    extra = {}
+    if world == 1 and args.workload == 3 and not args.no_extra_configs:
+        weights = w.weights
+        w.release_cache()
+        free, _ = torch.cuda.mem_get_info(device)
+        m5 = wl.CONFIGS[5]["model"]
+        need5 = 2 * m5["n_layers"] * 16 * (65536 + 128) * m5["n_kv_heads"] * m5["head_dim"] * 2 + (4 << 30)
+        if free >= need5:
+            extra["5"] = measure_decode(wl.CONFIGS[5], 8, 3, device, weights)
+        else:
+            extra["5"] = dict(skipped=f"{free >> 30} GiB free, {need5 >> 30} GiB needed")
+        sub = argparse.Namespace(steps=3, warmup=2, workload=4)
+        extra["4"] = measure_mixed(wl.CONFIGS[4], sub, device, weights=weights)
+        for k in ("metric", "unit", "n_gpus", "higher_is_better", "scaling", "vs_baseline", "dtype", "data", "value", "steps", "warmup"):
+            extra["4"].pop(k, None)
     cpu = OracleSample(cfg, 8).run()
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic",
                 config=dict(workload=cfg["name"], batch=w.B, n_layers=model["n_layers"], page_size=cfg["page_size"],
-                            context_tokens=kv_tokens_start, sampling=cfg["sampling"], l2="inputs larger than L2",
+                            context_tokens=kv_tokens_start, context_tokens_expected=len(w.ctx) * sum(cfg.get("ctx_range", (0, 0))) // 2,
+                            sampling=cfg["sampling"], l2="inputs larger than L2",
                             replicas=world, setup_s=round(w.setup_s, 1)),
                 clocks=clocks, e2e=e2e, gpu_launches=int(info["kernel_launches"]) * args.steps,
                 roofline=roofline,
@@ -546,6 +607,8 @@ def run_cuda(args):
                                    frac_of_nominal_8tbs=step_gbs / 8000.0,
                                    active_experts_mean=sum(active) / len(active)),
                 kernels=kernels, cpu_baseline={k: v for k, v in cpu.items() if k != "seconds"})
+    if extra:
+        line["configs"] = extra
     print(json.dumps(line))
 
 
@@ -556,6 +619,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", type=int, default=3, choices=[2, 3, 4, 5, 6, 7, 8])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-extra-configs", action="store_true",
+                    help="time configuration 3 only (by default one GPU also times configurations 5 and 4 on the same weights)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -90,7 +90,9 @@ int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const Debug
 // Prefill-sized contractions on tcgen05: out[m][n_cols] = A[m][2][K] (hi + lo planes) . B[n_cols][K]^T, and
 // the grouped expert pair (gather rows to slot order, gate/up + SwiGLU, down) over the group list.
 int launch_resid_norm(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int o_ksplit, cudaStream_t st);
-int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int group_cap,
+// n_parts: split-K partials of the gate logits in b.rlogits ([part][n_tok][E]); group_cap <= 0: the streaming
+// expert kernels' group size.  Small calls run the token permutation in the selection kernel's last block.
+int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int group_cap, int n_parts,
                         cudaStream_t st);
 // The QKV projection with its post-processing in the epilogue of the contraction kernel.  A thread owns one
 // token row of a tile and, in it, whole heads (256 / head_dim of them): per-head RMS norm (optional),

@@ -543,7 +543,7 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 
 // Merge of the spans of one (token row, query head): log-sum-exp rule on (max, sum, O).  The span
 // statistics are fetched in one round trip (one span per thread), then the partial outputs are
-// read four spans at a time.
+// read eight spans at a time.
 template <int D>
 __global__ void __launch_bounds__(D) attn_combine_kernel(Buffers b, StepLayout lay, int nq) {
     __shared__ float2 sml[D];
@@ -562,13 +562,13 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(Buffers b, StepLayout l
         const float rescale = exp2f(M - Mc);            // 0 for the first chunk (M = -inf)
         den *= rescale; o *= rescale;
         M = Mc;
-        for (int i = 0; i < n; i += 4) {
-            float pv[4];
+        for (int i = 0; i < n; i += 8) {
+            float pv[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
+            for (int q = 0; q < 8; ++q)
                 pv[q] = i + q < n ? b.part_o[((size_t)(c0 + i + q) * nq + j) * D + d] : 0.f;
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
+            for (int q = 0; q < 8; ++q)
                 if (i + q < n) {
                     const float sc = exp2f(sml[i + q].x - M);
                     den += sml[i + q].y * sc;

@@ -241,15 +241,27 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(Shape s, Buffers b, StepL
         float lo[PER], hi[PER];
         float ss = 0.f;
 #pragma unroll
-        for (int i = 0; i < PER; ++i) {
-            lo[i] = hi[i] = 0.f;
-            for (int sp = 0; sp < ksplit; ++sp) {      // split-K partials, fixed order
-                const float* part = raw + (size_t)sp * n_tok * n_heads * D;
-                lo[i] += part[head * D + lane + 32 * i];
-                hi[i] += part[head * D + lane + 32 * i + HALF];
+        for (int i = 0; i < PER; ++i) lo[i] = hi[i] = 0.f;
+        // split-K partials, added in a fixed order; the loads of up to eight partials are issued before the
+        // first add (one memory round trip, not one per partial)
+        for (int sp0 = 0; sp0 < ksplit; sp0 += 8) {
+            float pl[8][PER], ph[8][PER];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float* part = raw + (size_t)(sp0 + j) * n_tok * n_heads * D + head * D + lane;
+#pragma unroll
+                for (int i = 0; i < PER; ++i) {
+                    pl[j][i] = sp0 + j < ksplit ? part[32 * i] : 0.f;
+                    ph[j][i] = sp0 + j < ksplit ? part[32 * i + HALF] : 0.f;
+                }
             }
-            ss += lo[i] * lo[i] + hi[i] * hi[i];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int i = 0; i < PER; ++i) { lo[i] += pl[j][i]; hi[i] += ph[j][i]; }
         }
+#pragma unroll
+        for (int i = 0; i < PER; ++i) ss += lo[i] * lo[i] + hi[i] * hi[i];
         if (!is_q && !is_k) {  // value head: stored as is
             const int hk = head - s.nq - s.nkv;
             __nv_bfloat16* dst = kv.v_pool +

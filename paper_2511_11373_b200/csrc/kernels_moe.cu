@@ -66,14 +66,104 @@ __device__ void route_select(float* z, const Shape& s, const Buffers& b, const D
 }
 
 // ---------------------------------------------------------------------------------------------
+// Token permutation: histogram of expert ids, exclusive offsets, and for every expert the list of
+// token rows it serves (slot order inside an expert is arbitrary: every (token, expert) product is
+// computed independently of its slot).  Run by ONE block of at least E threads; also counts the
+// distinct experts used.
+// `counted`: the per-expert counts were accumulated in b.perm_cnt by permute_count_kernel (large calls);
+// then this block only scans them, writes the offsets, the group list and b.perm_cur, clears b.perm_cnt
+// for the next use and leaves the slot assignment to permute_scatter_kernel.
+// The routing indices are read with ld.global.cg: when the block runs at the end of the router kernel
+// they were written by other blocks of the same grid.
+struct PermuteSmem {
+    int cnt[kMaxExperts];
+    int off[kMaxExperts + 1];
+    int wtot[3][32];
+};
+
+__device__ void permute_block(const Shape& s, const Buffers& b, int layer, int n_pairs, int tok_cap, int counted, PermuteSmem& sm) {
+    int* cnt = sm.cnt;
+    int* off = sm.off;
+    const int tid = threadIdx.x, E = s.E;
+    if (counted) {
+        for (int e = tid; e < E; e += blockDim.x) { cnt[e] = b.perm_cnt[e]; b.perm_cnt[e] = 0; }
+    } else {
+        for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
+        __syncthreads();
+        for (int i = tid; i < n_pairs; i += blockDim.x) atomicAdd(&cnt[__ldcg(b.route_idx + i)], 1);
+    }
+    __syncthreads();
+    // one expert per thread (E <= 1024): exclusive scans of the token counts (slot offsets), of the
+    // group counts (positions in the group list) and of "has tokens" (distinct experts)
+    {
+        const int lane = tid & 31, warp = tid >> 5;
+        const int c = tid < E ? cnt[tid] : 0;
+        int inc[3] = {c, (c + tok_cap - 1) / tok_cap, c > 0 ? 1 : 0};
+        const int own[3] = {inc[0], inc[1], inc[2]};
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int nb = __shfl_up_sync(0xffffffffu, inc[q], o);
+                if (lane >= o) inc[q] += nb;
+            }
+            if (lane == 31) sm.wtot[q][warp] = inc[q];
+        }
+        __syncthreads();
+        int base[3] = {0, 0, 0}, tot[3] = {0, 0, 0};
+        for (int w = 0; w < 32; ++w)
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+                if (w < warp) base[q] += sm.wtot[q][w];
+                tot[q] += sm.wtot[q][w];
+            }
+        if (tid < E) {
+            const int o0 = base[0] + inc[0] - own[0];
+            off[tid] = o0;
+            // token groups for the expert kernels: (expert, first slot, tokens <= tok_cap, 0)
+            int ng = base[1] + inc[1] - own[1];
+            for (int t0 = 0; t0 < c; t0 += tok_cap, ++ng)
+                reinterpret_cast<int4*>(b.groups)[ng] = make_int4(tid, o0 + t0, min(tok_cap, c - t0), 0);
+        }
+        if (tid == 0) {
+            off[E] = tot[0];
+            *b.n_groups = tot[1];
+            b.active[layer] = tot[2];
+        }
+    }
+    __syncthreads();
+    for (int e = tid; e <= E; e += blockDim.x) b.expert_off[e] = off[e];
+    if (counted) {
+        for (int e = tid; e < E; e += blockDim.x) b.perm_cur[e] = off[e];
+        return;
+    }
+    for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
+    __syncthreads();
+    for (int i = tid; i < n_pairs; i += blockDim.x) {
+        const int e = __ldcg(b.route_idx + i);
+        const int slot = off[e] + atomicAdd(&cnt[e], 1);
+        b.slot_token[slot] = i / s.k;
+        b.slot_of[i] = slot;
+    }
+}
+
+__global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int layer, int n_pairs, int tok_cap, int counted) {
+    __shared__ PermuteSmem sm;
+    pdl_wait();
+    permute_block(s, b, layer, n_pairs, tok_cap, counted, sm);
+}
+
+// ---------------------------------------------------------------------------------------------
 // One block per token row.  h2 = rms(x) * g (kept in fp32 for the gate, stored as a (hi, lo) bf16
 // pair for the experts); z_e = <W_r[e], h2> accumulated in fp32 in a fixed order; pi = softmax(z); the k largest
 // pi (ties: lower index) and their renormalised weights.
 constexpr int kRouterCta = 1024;
 constexpr int kRouterPer = 8;    // hidden <= 8192
+// perm_cap > 0: the block that finishes last (counted in b.n_groups[1], which is zero between kernels) also
+// runs the token permutation with groups of perm_cap tokens, which saves a kernel boundary per layer.
 __global__ void __launch_bounds__(kRouterCta) router_kernel(Shape s, Buffers b, const __nv_bfloat16* gain,
                                                             const __nv_bfloat16* Wr, DebugTaps dbg, int layer, int n_tok,
-                                                            int o_ksplit) {
+                                                            int o_ksplit, int perm_cap) {
     // one column tile of activations: row 0 = hi, row 1 = lo of this token, rows 2..7 zero
     extern __shared__ __align__(16) unsigned char xt[];
     __shared__ float scratch[32];
@@ -94,16 +184,20 @@ __global__ void __launch_bounds__(kRouterCta) router_kernel(Shape s, Buffers b, 
         const int c = tid + i * kRouterCta;
         v[i] = c < H ? xin[c] : 0.f;
     }
-    for (int sp = 0; sp < o_ksplit; ++sp) {
-        const float* __restrict__ part = b.opart + ((size_t)sp * n_tok + t) * H;
-        float pv[kRouterPer];
+    // (per column the loads of up to eight partials are issued before the first add: one memory round trip, not eight)
+    for (int sp0 = 0; sp0 < o_ksplit; sp0 += 8) {
 #pragma unroll
         for (int i = 0; i < kRouterPer; ++i) {
             const int c = tid + i * kRouterCta;
-            pv[i] = c < H ? part[c] : 0.f;
-        }
+            if (c < H) {
+                float pv[8];
 #pragma unroll
-        for (int i = 0; i < kRouterPer; ++i) v[i] += pv[i];
+                for (int j = 0; j < 8; ++j)
+                    pv[j] = sp0 + j < o_ksplit ? b.opart[((size_t)(sp0 + j) * n_tok + t) * H + c] : 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[i] += pv[j];
+            }
+        }
     }
 #pragma unroll
     for (int i = 0; i < kRouterPer; ++i) {
@@ -159,82 +253,24 @@ __global__ void __launch_bounds__(kRouterCta) router_kernel(Shape s, Buffers b, 
     }
     __syncthreads();
 
-    if (warp == 0) route_select(z, s, b, dbg, layer, n_tok, t, lane);
-}
-
-// ---------------------------------------------------------------------------------------------
-// Token permutation: histogram of expert ids, exclusive offsets, and for every expert the list of
-// token rows it serves (slot order inside an expert is arbitrary: every (token, expert) product is
-// computed independently of its slot).  Single block; also counts the distinct experts used.
-// `counted`: the per-expert counts were accumulated in b.perm_cnt by permute_count_kernel (large calls);
-// then this block only scans them, writes the offsets, the group list and b.perm_cur, clears b.perm_cnt
-// for the next use and leaves the slot assignment to permute_scatter_kernel.
-__global__ void __launch_bounds__(1024) permute_kernel(Shape s, Buffers b, int layer, int n_pairs, int tok_cap, int counted) {
-    __shared__ int cnt[kMaxExperts];
-    __shared__ int off[kMaxExperts + 1];
-    pdl_wait();
-    const int tid = threadIdx.x, E = s.E;
-    if (counted) {
-        for (int e = tid; e < E; e += blockDim.x) { cnt[e] = b.perm_cnt[e]; b.perm_cnt[e] = 0; }
-    } else {
-        for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
-        __syncthreads();
-        for (int i = tid; i < n_pairs; i += blockDim.x) atomicAdd(&cnt[b.route_idx[i]], 1);
+    if (warp == 0) {
+        route_select(z, s, b, dbg, layer, n_tok, t, lane);
+        __threadfence();                 // this token's routing is visible to the whole device before the count below
+    }
+    if (perm_cap <= 0) return;
+    __shared__ int is_last;
+    __shared__ PermuteSmem perm_sm;
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const int prev = atomicAdd(b.n_groups + 1, 1);
+        is_last = prev == n_tok - 1;
+        if (is_last) b.n_groups[1] = 0;  // every block has counted: ready for the next launch
     }
     __syncthreads();
-    // one expert per thread (E <= 1024): exclusive scans of the token counts (slot offsets), of the
-    // group counts (positions in the group list) and of "has tokens" (distinct experts)
-    {
-        __shared__ int wtot[3][32];
-        const int lane = tid & 31, warp = tid >> 5;
-        const int c = tid < E ? cnt[tid] : 0;
-        int inc[3] = {c, (c + tok_cap - 1) / tok_cap, c > 0 ? 1 : 0};
-        const int own[3] = {inc[0], inc[1], inc[2]};
-#pragma unroll
-        for (int q = 0; q < 3; ++q) {
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int nb = __shfl_up_sync(0xffffffffu, inc[q], o);
-                if (lane >= o) inc[q] += nb;
-            }
-            if (lane == 31) wtot[q][warp] = inc[q];
-        }
-        __syncthreads();
-        int base[3] = {0, 0, 0}, tot[3] = {0, 0, 0};
-        for (int w = 0; w < 32; ++w)
-#pragma unroll
-            for (int q = 0; q < 3; ++q) {
-                if (w < warp) base[q] += wtot[q][w];
-                tot[q] += wtot[q][w];
-            }
-        if (tid < E) {
-            const int o0 = base[0] + inc[0] - own[0];
-            off[tid] = o0;
-            // token groups for the expert kernels: (expert, first slot, tokens <= tok_cap, 0)
-            int ng = base[1] + inc[1] - own[1];
-            for (int t0 = 0; t0 < c; t0 += tok_cap, ++ng)
-                reinterpret_cast<int4*>(b.groups)[ng] = make_int4(tid, o0 + t0, min(tok_cap, c - t0), 0);
-        }
-        if (tid == 0) {
-            off[E] = tot[0];
-            *b.n_groups = tot[1];
-            b.active[layer] = tot[2];
-        }
-    }
-    __syncthreads();
-    for (int e = tid; e <= E; e += blockDim.x) b.expert_off[e] = off[e];
-    if (counted) {
-        for (int e = tid; e < E; e += blockDim.x) b.perm_cur[e] = off[e];
-        return;
-    }
-    for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
-    __syncthreads();
-    for (int i = tid; i < n_pairs; i += blockDim.x) {
-        const int e = b.route_idx[i];
-        const int slot = off[e] + atomicAdd(&cnt[e], 1);
-        b.slot_token[slot] = i / s.k;
-        b.slot_of[i] = slot;
-    }
+    if (!is_last) return;
+    __threadfence();
+    permute_block(s, b, layer, n_tok * k, perm_cap, 0, perm_sm);
 }
 
 // Large calls (tens of thousands of (token, expert) pairs) count and hand out the slots with many
@@ -599,14 +635,19 @@ __global__ void __launch_bounds__(kRouterThreads) resid_norm_kernel(Shape s, Buf
         const int c = (tid + i * kRouterThreads) * 4;
         v[i] = c < H ? *reinterpret_cast<const float4*>(xin + c) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    for (int sp = 0; sp < o_ksplit; ++sp) {
-        const float* __restrict__ part = b.opart + ((size_t)sp * n_tok + t) * H;
+    // per column group the loads of up to eight partials are issued before the first add
+    for (int sp0 = 0; sp0 < o_ksplit; sp0 += 8) {
 #pragma unroll
         for (int i = 0; i < kVec; ++i) {
             const int c = (tid + i * kRouterThreads) * 4;
             if (c < H) {
-                const float4 pv = *reinterpret_cast<const float4*>(part + c);
-                v[i].x += pv.x; v[i].y += pv.y; v[i].z += pv.z; v[i].w += pv.w;
+                float4 pv[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    pv[j] = sp0 + j < o_ksplit ? *reinterpret_cast<const float4*>(b.opart + ((size_t)(sp0 + j) * n_tok + t) * H + c)
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { v[i].x += pv[j].x; v[i].y += pv[j].y; v[i].z += pv[j].z; v[i].w += pv[j].w; }
             }
         }
     }
@@ -637,17 +678,56 @@ __global__ void __launch_bounds__(kRouterThreads) resid_norm_kernel(Shape s, Buf
     }
 }
 
-// One warp per token row: logits [n_tok][E] (fp32, from the contraction) -> routing.
-__global__ void __launch_bounds__(128) route_select_kernel(Shape s, Buffers b, DebugTaps dbg, int layer, int n_tok) {
-    extern __shared__ float zs[];     // [4][E]
+// One warp per token row: gate logits (fp32, from the contraction: n_parts split-K partials
+// [part][n_tok][E], added in a fixed order) -> routing.  perm_cap > 0: the block that finishes last also
+// runs the token permutation (as in router_kernel).
+constexpr int kSelectWarps = 32;
+__global__ void __launch_bounds__(kSelectWarps * 32) route_select_kernel(Shape s, Buffers b, DebugTaps dbg, int layer, int n_tok,
+                                                                         int n_parts, int perm_cap) {
+    extern __shared__ float zs[];     // [warps][E]
     pdl_wait();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int t = blockIdx.x * 4 + warp;
-    if (t >= n_tok) return;
-    float* z = zs + (size_t)warp * s.E;
-    for (int e = lane; e < s.E; e += 32) z[e] = b.rlogits[(size_t)t * s.E + e];
-    __syncwarp();
-    route_select(z, s, b, dbg, layer, n_tok, t, lane);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int t = blockIdx.x * kSelectWarps + warp;
+    if (t < n_tok) {
+        float* z = zs + (size_t)warp * s.E;
+        const size_t part_stride = (size_t)n_tok * s.E;
+        for (int e0 = lane; e0 < s.E; e0 += 4 * 32) {       // four experts per lane and pass: their partials load together
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int sp0 = 0; sp0 < n_parts; sp0 += 8) {
+                float pv[8][4];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int e = e0 + 32 * q;
+                        pv[j][q] = (sp0 + j < n_parts && e < s.E) ? b.rlogits[(size_t)(sp0 + j) * part_stride + (size_t)t * s.E + e] : 0.f;
+                    }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) acc[q] += pv[j][q];
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (e0 + 32 * q < s.E) z[e0 + 32 * q] = acc[q];
+        }
+        __syncwarp();
+        route_select(z, s, b, dbg, layer, n_tok, t, lane);
+    }
+    if (perm_cap <= 0) return;
+    __shared__ int is_last;
+    __shared__ PermuteSmem perm_sm;
+    __syncthreads();                     // the block's routing has been written ...
+    if (tid == 0) {
+        __threadfence();                 // ... and is visible to the whole device before the count below
+        const int prev = atomicAdd(b.n_groups + 1, 1);
+        is_last = prev == (int)gridDim.x - 1;
+        if (is_last) b.n_groups[1] = 0;  // every block has counted: ready for the next launch
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    permute_block(s, b, layer, n_tok * s.k, perm_cap, 0, perm_sm);
 }
 
 int launch_resid_norm(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int o_ksplit, cudaStream_t st) {
@@ -655,10 +735,18 @@ int launch_resid_norm(const Shape& s, const Buffers& b, const LayerW& w, int n_t
     return 1;
 }
 
-int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int group_cap,
+static void expert_plan(const Shape& s, int n_tok, int* cap, int* warps);
+int launch_route_select(const Shape& s, const Buffers& b, const DebugTaps& dbg, int layer, int n_tok, int group_cap, int n_parts,
                         cudaStream_t st) {
-    launch_chained(route_select_kernel, dim3((n_tok + 3) / 4), dim3(128), 4 * s.E * sizeof(float), st, s, b, dbg, layer, n_tok);
-    return 1 + launch_permute(s, b, layer, n_tok * s.k, group_cap, st);
+    int cap = group_cap;                                 // > 0: the tensor-core expert path wants one 128-row tile per group
+    if (cap <= 0) {
+        int warps;
+        expert_plan(s, n_tok, &cap, &warps);
+    }
+    const bool fused = n_tok * s.k < 4 * kPermChunk;     // small permutations run in the selection's last block
+    launch_chained(route_select_kernel, dim3((n_tok + kSelectWarps - 1) / kSelectWarps), dim3(kSelectWarps * 32),
+                   (size_t)kSelectWarps * s.E * sizeof(float), st, s, b, dbg, layer, n_tok, n_parts, fused ? cap : 0);
+    return fused ? 1 : 1 + launch_permute(s, b, layer, n_tok * s.k, cap, st);
 }
 
 // Tokens per group (4 per column tile); experts with more tokens are cut into several groups and
@@ -676,12 +764,13 @@ static void expert_plan(const Shape& s, int n_tok, int* cap, int* warps) {
 // ---------------------------------------------------------------------------------------------
 int launch_router(const Shape& s, const Buffers& b, const LayerW& w, const DebugTaps& dbg, int layer, int n_tok,
                   int group_cap, int o_ksplit, cudaStream_t st) {
-    launch_chained(router_kernel, dim3(n_tok), dim3(kRouterCta), 8 * x_row_bytes(s.H), st, s, b, w.mlp_norm, w.router, dbg, layer, n_tok,
-                                                                       o_ksplit);
     int cap, warps;
     expert_plan(s, n_tok, &cap, &warps);
     if (group_cap > 0) cap = group_cap;          // the tensor-core expert path wants one 128-row tile per group
-    return 1 + launch_permute(s, b, layer, n_tok * s.k, cap, st);
+    const bool fused = n_tok * s.k < 4 * kPermChunk;   // small permutations run in the router's last block
+    launch_chained(router_kernel, dim3(n_tok), dim3(kRouterCta), 8 * x_row_bytes(s.H), st, s, b, w.mlp_norm, w.router, dbg, layer, n_tok,
+                   o_ksplit, fused ? cap : 0);
+    return fused ? 1 : 1 + launch_permute(s, b, layer, n_tok * s.k, cap, st);
 }
 
 int launch_gate_up(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, int sm_count, cudaStream_t st) {
@@ -711,6 +800,8 @@ cudaError_t init_moe_kernels() {
     cudaError_t e = cudaFuncSetAttribute(expert_gate_up_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(expert_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(route_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelectWarps * kMaxExperts * (int)sizeof(float));
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(router_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * x_row_bytes(8192));
 }

@@ -341,6 +341,8 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
     if (e != cudaSuccess) return fail(e);
     e = cudaMemset(m->buf.perm_cnt, 0, (size_t)cfg->n_experts * 4);
     if (e != cudaSuccess) return fail(e);
+    e = cudaMemset(m->buf.n_groups, 0, 256);      // [1]: arrival counter of the router blocks, zero between kernels
+    if (e != cudaSuccess) return fail(e);
     // tensor maps of the prefill path (calls with more than kUmmaMinTokens token rows)
     m->umma_ready = false;
     {
@@ -358,9 +360,9 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
             rc = make_weight_map(&m->tm_wqkv[l], q.wqkv, (uint64_t)(cfg->n_q_heads + 2 * cfg->n_kv_heads) * cfg->head_dim, H);
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_wo[l], q.wo, H, QD);
             if (!big) continue;
+            if (rc == MARS_OK) rc = make_weight_map(&m->tm_router[l], q.router, E, H);
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_wgu[l], q.w_gate_up, E * 2 * I, H);
             if (rc == MARS_OK) rc = make_weight_map(&m->tm_wdown[l], q.w_down, E * H, I);
-            if (rc == MARS_OK) rc = make_weight_map(&m->tm_router[l], q.router, E, H);
         }
         if (big) {
             if (rc == MARS_OK) rc = make_pair_map(&m->tm_o, m->buf.o, n, QD);
@@ -970,7 +972,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             run(MARS_K_ROUTER, [&] {
                 int n = launch_resid_norm(s, b, w, n_tok, 1, st);
                 n += launch_umma_dense(m->tm_h, m->tm_router[l], n_tok, s.E, s.H, b.rlogits, b.err, st);
-                return n + launch_route_select(s, b, taps, l, n_tok, 128, st);
+                return n + launch_route_select(s, b, taps, l, n_tok, 128, 1, st);
             });
             run(MARS_K_GATE_UP, [&] {
                 return launch_umma_experts(s, b, m->tm_xperm, m->tm_wgu[l], m->tm_act, m->tm_wdown[l], n_tok, st);
@@ -1395,6 +1397,7 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
     CUDA_TRY(cudaMemsetAsync(buf.err, 0, 256, st));
     CUDA_TRY(cudaMemsetAsync(buf.active, 0, (size_t)cfg->n_layers * 4, st));
     CUDA_TRY(cudaMemsetAsync(buf.perm_cnt, 0, (size_t)cfg->n_experts * 4, st));   // its offset moves with the shape
+    CUDA_TRY(cudaMemsetAsync(buf.n_groups, 0, 256, st));                         // the router blocks' arrival counter
     CUDA_TRY(cudaMemcpyAsync(buf.step, blk.data(), blk.size() * 4, cudaMemcpyHostToDevice, st));
     CUDA_TRY(cudaMemcpyAsync(buf.inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice, st));
 
