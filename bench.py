@@ -295,14 +295,17 @@ def measure_mixed(cfg: dict, args, device, weights=None) -> dict:
         w.step()
     n_steady = max(args.steps, 6)
     torch.cuda.synchronize()
+    clk = ClockSampler(device.index or 0)
     ev[0].record(stream)
     for _ in range(n_steady):
         w.step()
     ev[1].record(stream)
     torch.cuda.synchronize()
+    clocks_decode = clk.stop()
     steady_ms = ev[0].elapsed_time(ev[1]) / n_steady
     steady_bytes = algorithmic_bytes(model, w.kv_tokens_now() - w.B * n_steady // 2, w.model.active_experts().tolist())
     t_pf, t_dec = [], []
+    clk = ClockSampler(device.index or 0)
     for it in range(args.warmup + args.steps):
         for s_ in ids:
             w.kv.seq_reserve(s_, 0)
@@ -319,6 +322,7 @@ def measure_mixed(cfg: dict, args, device, weights=None) -> dict:
             w.kv.seq_release(s_)
         if it >= args.warmup:
             t_pf.append(ev[0].elapsed_time(ev[1])); t_dec.append(ev[1].elapsed_time(ev[2]))
+    clocks_alternating = clk.stop()
     # the same work as ONE call: decode rows and prompt chunks share every projection and every expert pass
     mix_t = torch.empty(w.B + pf["requests"], dtype=torch.int32, device=device)
     mix_l = torch.empty(w.B + pf["requests"], dtype=torch.float32, device=device)
@@ -365,8 +369,8 @@ def measure_mixed(cfg: dict, args, device, weights=None) -> dict:
                 config=dict(workload=cfg["name"], decode_seqs=w.B, prefill_requests=pf["requests"], prefill_chunk=pf["chunk"],
                             l2="inputs larger than L2"),
                 decode=dict(ms=dec_ms, bytes=dec_bytes["total"], frac_of_measured_hbm=dec_bytes["total"] / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                            note="one decode step right after each prefill call"),
-                decode_back_to_back=dict(ms=steady_ms, tokens_per_s=w.B / (steady_ms / 1e3), bytes=steady_bytes["total"],
+                            note="one decode step right after each prefill call", clocks=clocks_alternating),
+                decode_back_to_back=dict(ms=steady_ms, tokens_per_s=w.B / (steady_ms / 1e3), bytes=steady_bytes["total"], clocks=clocks_decode,
                                          frac_of_measured_hbm=steady_bytes["total"] / (steady_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]),
                 prefill=dict(ms=pf_ms, tokens_per_s=n_pf / (pf_ms / 1e3), algorithmic_tflop=flops / 1e12,
                              achieved_tflops=flops / (pf_ms * 1e-3) / 1e12, frac_of_measured_bf16=flops / (pf_ms * 1e-3) / 1e12 / tflops_peak,

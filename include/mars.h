@@ -309,6 +309,26 @@ MARS_API mars_status_t mars_decode_step_static(const mars_config_t *cfg, const m
                                       const int32_t *in_tokens, const mars_sampling_t *sampling,
                                       int32_t *out_tokens, float *out_logprobs);
 
+/* Precision of the dense contractions of LARGE calls (more than 256 token rows: chunked prefill, mixed
+ * steps, scoring).  Activations travel as (hi, lo) bf16 pairs (~16 mantissa bits); a contraction
+ * class whose bit is clear contracts the hi plane only, i.e. plain bf16 activations: half the
+ * tensor-core work for ~1e-3 relative error in that contraction's output.  Decode-sized calls and the
+ * lm_head always use both planes.  MARS_LO_DEFAULT is what mars_model_load sets: both planes for the QKV
+ * and output projections and the router, the hi plane only for the expert contractions.  Measured on a
+ * 264-token chunk through the 48-layer model against the CPU oracle (max relative L2 error of a hidden
+ * state / max absolute logit error / time of an 8 x 2048-token prefill): all planes 6.4e-4 / 1.3e-3 /
+ * 230 ms; QKV hi only 5.7e-3 / 8.1e-3 / 223 ms; output projection hi only 4.4e-3 / 9.0e-3 / 226 ms;
+ * router hi only 1.9e-3 / 3.2e-3 / 231 ms; gate/up hi only 2.2e-3 / 3.9e-3 / 213 ms; down hi only
+ * 1.8e-3 / 3.0e-3 / 221 ms; both expert contractions hi only 2.5e-3 / 3.9e-3 / 203 ms; everything hi only
+ * 7.2e-3 / 1.2e-2 / 191 ms.  The default is the fastest setting that stays inside HALF of the tolerances
+ * (1e-2 relative for hidden states, 2e-2 absolute for logits). */
+enum {
+    MARS_LO_QKV = 1, MARS_LO_OPROJ = 2, MARS_LO_ROUTER = 4, MARS_LO_GATE_UP = 8, MARS_LO_DOWN = 16,
+    MARS_LO_ALL = 31,
+    MARS_LO_DEFAULT = 7
+};
+MARS_API mars_status_t mars_set_prefill_lo_planes(mars_model_t *model, int32_t mask);
+
 /* Synchronises the stream of the last call and reads the device status word: MARS_OK,
  * MARS_ERR_BAD_TOKEN or MARS_ERR_TIMEOUT; the word is cleared. */
 MARS_API mars_status_t mars_poll_status(mars_model_t *model);

@@ -101,6 +101,7 @@ SIGNATURES = {
                                           c_int32, c_void_p, c_int32, POINTER(c_int32), c_void_p, c_int32, c_void_p,
                                           POINTER(mars_sampling_t), c_void_p, c_void_p]),
     "mars_poll_status": (c_int32, [c_void_p]),
+    "mars_set_prefill_lo_planes": (c_int32, [c_void_p, c_int32]),
     "mars_debug_bounded_wait": (c_int32, [c_void_p, c_void_p, c_int32]),
     "mars_profile_enable": (c_int32, [c_void_p, c_int32]),
     "mars_profile_read": (c_int32, [c_void_p, POINTER(ctypes.c_double), POINTER(c_int64)]),
@@ -204,6 +205,11 @@ class Model:
         """Launches the library's bounded-wait self-test (see mars_debug_bounded_wait); returns the status code."""
         with torch.cuda.device(self.device):
             return lib().mars_debug_bounded_wait(self.handle, _stream_handle(stream), 1 if arrive else 0)
+
+    def set_prefill_lo_planes(self, mask: int):
+        """Bit per contraction class of large calls (QKV 1, output projection 2, router 4, gate/up 8, down 16):
+        set = (hi, lo) activations, clear = hi plane only."""
+        _check(lib().mars_set_prefill_lo_planes(self.handle, int(mask)), "mars_set_prefill_lo_planes")
 
     def last_step_info(self) -> dict:
         info = mars_step_info_t()

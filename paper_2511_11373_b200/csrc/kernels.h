@@ -109,17 +109,19 @@ struct QkvEpilogue {
     int max_pages_per_seq, n_pages, page_size, layer, nq, nkv, head_dim, qk_norm;
     float eps;
 };
+// use_lo: 1 accumulates the lo plane of the (hi, lo) activations too; 0 contracts the hi plane only (bf16
+// activations: half the tensor work, ~1e-3 relative error per contraction).
 int launch_umma_qkv(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, const QkvEpilogue& ep,
-                    int32_t* err, cudaStream_t st);
+                    int32_t* err, int use_lo, cudaStream_t st);
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
-                      int32_t* err, cudaStream_t st);
+                      int32_t* err, int use_lo, cudaStream_t st);
 // Decode-sized projection on tcgen05 with swapped operands: out[split][t][row], t < n_tok <= umma_swap_max_tokens().
 int umma_swap_max_tokens();
 int umma_swap_splits(int rows, int n_tok, int K);
 int launch_umma_swap(const CUtensorMap& tm_w, const CUtensorMap& tm_x, int rows, int n_tok, int K, int splits, float* out,
                      int32_t* err, cudaStream_t st);
 int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_xperm, const CUtensorMap& tm_wgu,
-                        const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, cudaStream_t st);
+                        const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, int gate_up_lo, int down_lo, cudaStream_t st);
 // Scoring pass: out_logprobs[row] = log softmax(lm_head(h[row]) * inv_temp)[targets[row]] (0 where the
 // target is negative).  score_ml: [score_vocab_tiles(vocab)][n_rows] scratch, score_tgt: [n_rows] scratch.
 int score_vocab_tiles(int vocab);

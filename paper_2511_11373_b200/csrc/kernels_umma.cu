@@ -134,6 +134,7 @@ struct UmmaParams {
     float2* score_ml;
     float* score_tgt;
     int tiles_x;              // column tiles per row tile (mode 1: 128 output columns each, else 256)
+    int use_lo;               // 1: accumulate the lo plane of the activations as well (hi + lo = ~16 mantissa bits)
     QkvEpilogue qkv;          // mode 3: the tile's columns are whole heads of the QKV projection (kernels.h)
 };
 
@@ -273,9 +274,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                         dead = 1; atomicOr(p.err, kErrTimeout); break;
                     }
                     unsigned char* st = smem + (size_t)s * kUmStageBytes;
-                    um_expect_tx(&full_bar[s], kUmStageBytes);
+                    um_expect_tx(&full_bar[s], p.use_lo ? kUmStageBytes : kUmStageBytes - kUmTileBytes);
                     um_tma_3d(st, &tm_a, ks * kUmStageK, 0, t.m0, &full_bar[s]);
-                    um_tma_3d(st + kUmTileBytes, &tm_a, ks * kUmStageK, 1, t.m0, &full_bar[s]);
+                    if (p.use_lo) um_tma_3d(st + kUmTileBytes, &tm_a, ks * kUmStageK, 1, t.m0, &full_bar[s]);
                     unsigned char* sb = st + 2 * kUmTileBytes;        // four boxes of 64 weight rows (8 KB each)
                     um_tma_2d(sb, &tm_b, ks * kUmStageK, t.b_row0, &full_bar[s]);
                     um_tma_2d(sb + 8192, &tm_b, ks * kUmStageK, t.b_row0 + 64, &full_bar[s]);
@@ -304,7 +305,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 #pragma unroll
                     for (int kk = 0; kk < kUmStageK / 16; ++kk) {   // 32 bytes along K per step: +2 in the address field
                         um_mma(acc, d_hi + 2 * kk, d_b + 2 * kk, (ks | kk) != 0);
-                        um_mma(acc, d_lo + 2 * kk, d_b + 2 * kk, 1u);
+                        if (p.use_lo) um_mma(acc, d_lo + 2 * kk, d_b + 2 * kk, 1u);
                     }
                     um_commit(&empty_bar[s]);                        // the stage is free once these MMAs retire
                 }
@@ -628,32 +629,32 @@ static size_t umma_smem_bytes() { return (size_t)kUmStages * kUmStageBytes + 102
 static int umma_grid(int tiles) { return tiles < g_umma_sms ? (tiles < 1 ? 1 : tiles) : g_umma_sms; }
 
 int launch_umma_dense(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, float* out,
-                      int32_t* err, cudaStream_t st) {
+                      int32_t* err, int use_lo, cudaStream_t st) {
     const int tx = (n_cols + kUmTileN - 1) / kUmTileN, ty = (m_rows + kUmTileM - 1) / kUmTileM;
-    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err, nullptr, 0.f, nullptr, nullptr, tx, QkvEpilogue{}};
+    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 0, out, nullptr, err, nullptr, 0.f, nullptr, nullptr, tx, use_lo, QkvEpilogue{}};
     launch_chained(umma_gemm_kernel, dim3(umma_grid(tx * ty)), dim3(kUmThreads), umma_smem_bytes(), st, tm_a, tm_b, p);
     return 1;
 }
 
 // QKV projection of a prefill-sized call with the per-head norm, RoPE and cache append in its epilogue.
 int launch_umma_qkv(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int m_rows, int n_cols, int K, const QkvEpilogue& ep,
-                    int32_t* err, cudaStream_t st) {
+                    int32_t* err, int use_lo, cudaStream_t st) {
     const int tx = (n_cols + kUmTileN - 1) / kUmTileN, ty = (m_rows + kUmTileM - 1) / kUmTileM;
-    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 3, nullptr, nullptr, err, nullptr, 0.f, nullptr, nullptr, tx, ep};
+    UmmaParams p{K, m_rows, nullptr, nullptr, 0, n_cols, 3, nullptr, nullptr, err, nullptr, 0.f, nullptr, nullptr, tx, use_lo, ep};
     launch_chained(umma_gemm_kernel, dim3(umma_grid(tx * ty)), dim3(kUmThreads), umma_smem_bytes(), st, tm_a, tm_b, p);
     return 1;
 }
 
 int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_xperm, const CUtensorMap& tm_wgu,
-                        const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, cudaStream_t st) {
+                        const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, int gate_up_lo, int down_lo, cudaStream_t st) {
     const int n_slots = n_tok * s.k;
     const int max_groups = s.E + (n_slots + kUmTileM - 1) / kUmTileM;
     launch_chained(gather_rows_kernel, dim3(n_slots), dim3(256), 0, st, b, s.H, n_slots);
     const int gx = (s.I + 127) / 128, dx = (s.H + kUmTileN - 1) / kUmTileN;
-    UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err, nullptr, 0.f, nullptr, nullptr, gx, QkvEpilogue{}};
+    UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err, nullptr, 0.f, nullptr, nullptr, gx, gate_up_lo, QkvEpilogue{}};
     launch_chained(umma_gemm_kernel, dim3(umma_grid(gx * max_groups)), dim3(kUmThreads), umma_smem_bytes(), st, tm_xperm,
                    tm_wgu, gu);
-    UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err, nullptr, 0.f, nullptr, nullptr, dx, QkvEpilogue{}};
+    UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err, nullptr, 0.f, nullptr, nullptr, dx, down_lo, QkvEpilogue{}};
     launch_chained(umma_gemm_kernel, dim3(umma_grid(dx * max_groups)), dim3(kUmThreads), umma_smem_bytes(), st, tm_act,
                    tm_wdown, dn);
     return 3;
@@ -694,7 +695,7 @@ int launch_umma_score(const CUtensorMap& tm_h, const CUtensorMap& tm_lm, int n_r
                       float* out_logprobs, int32_t* err, cudaStream_t st) {
     const int n_tiles = (vocab + kUmTileN - 1) / kUmTileN;
     UmmaParams p{K, n_rows, nullptr, nullptr, 0, vocab, 2, logits_tap, nullptr, err, targets, inv_temp, score_ml, score_tgt,
-                 n_tiles, QkvEpilogue{}};
+                 n_tiles, 1, QkvEpilogue{}};
     launch_chained(umma_gemm_kernel, dim3(umma_grid(n_tiles * ((n_rows + kUmTileM - 1) / kUmTileM))), dim3(kUmThreads),
                    umma_smem_bytes(), st, tm_h, tm_lm, p);
     launch_chained(score_combine_kernel, dim3((n_rows + 7) / 8), dim3(256), 0, st, score_ml, score_tgt, targets, n_rows, n_tiles, vocab,

@@ -194,6 +194,7 @@ struct mars_model {
     CUtensorMap tm_h64, tm_o64, tm_lm;      // decode-sized (64 token rows per box) and the lm_head
     CUtensorMap tm_q;                       // queries for the tcgen05 prefill attention: (d, head, plane, token)
     CUtensorMap tm_q1;                      // the same tensor with one-token boxes (shared spans of decode rows)
+    int lo_planes;                          // bit per contraction class of large calls: 1 = (hi, lo) activations, 0 = hi only
     bool fattn_ready, fattn_shared_ready;
     bool umma_ready;
     const __nv_bfloat16 *embed, *final_norm, *lm_head;
@@ -315,6 +316,7 @@ mars_status_t mars_model_load(const mars_config_t* cfg, const mars_weights_t* w,
     m->next_slot = 0;
     m->last_stream = nullptr;
     m->profiling = false;
+    m->lo_planes = MARS_LO_DEFAULT;
     m->ev_used = 0;
     std::memset(&m->info, 0, sizeof(m->info));
     for (int i = 0; i < kStagingSlots; ++i) { m->staging[i] = nullptr; m->staged[i] = nullptr; }
@@ -937,7 +939,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
                 const QkvEpilogue ep{b.step + lay.tok_pos, b.step + lay.tok_seq, kv->view.block_table, b.rope, w.q_norm, w.k_norm,
                                      b.q, kv->view.k_pool, kv->view.v_pool, kv->view.max_pages_per_seq, kv->view.n_pages,
                                      kv->view.page_size, l, s.nq, s.nkv, s.D, s.qk_norm, s.eps};
-                return launch_umma_qkv(m->tm_h, m->tm_wqkv[l], n_tok, qkv_rows, s.H, ep, b.err, st);
+                return launch_umma_qkv(m->tm_h, m->tm_wqkv[l], n_tok, qkv_rows, s.H, ep, b.err, (m->lo_planes >> 0) & 1, st);
             });
         } else {      // decode-sized call: weights stream once through tcgen05 with the operands swapped
             run(MARS_K_QKV, [&] {
@@ -967,15 +969,16 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         }
         if (umma) {
             run(MARS_K_OPROJ, [&] {
-                return launch_umma_dense(m->tm_o, m->tm_wo[l], n_tok, s.H, s.nq * s.D, b.opart, b.err, st);
+                return launch_umma_dense(m->tm_o, m->tm_wo[l], n_tok, s.H, s.nq * s.D, b.opart, b.err, (m->lo_planes >> 1) & 1, st);
             });
             run(MARS_K_ROUTER, [&] {
                 int n = launch_resid_norm(s, b, w, n_tok, 1, st);
-                n += launch_umma_dense(m->tm_h, m->tm_router[l], n_tok, s.E, s.H, b.rlogits, b.err, st);
+                n += launch_umma_dense(m->tm_h, m->tm_router[l], n_tok, s.E, s.H, b.rlogits, b.err, (m->lo_planes >> 2) & 1, st);
                 return n + launch_route_select(s, b, taps, l, n_tok, 128, 1, st);
             });
             run(MARS_K_GATE_UP, [&] {
-                return launch_umma_experts(s, b, m->tm_xperm, m->tm_wgu[l], m->tm_act, m->tm_wdown[l], n_tok, st);
+                return launch_umma_experts(s, b, m->tm_xperm, m->tm_wgu[l], m->tm_act, m->tm_wdown[l], n_tok, (m->lo_planes >> 3) & 1,
+                                           (m->lo_planes >> 4) & 1, st);
             });
         } else {
             run(MARS_K_OPROJ, [&] {
@@ -1002,7 +1005,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
             if (!plan.prefill && n_emit <= kUmmaMinTokens)
                 return launch_umma_swap(m->tm_lm, m->tm_h64, s.V, n_emit, s.H, 1, b.logits, b.err, st);
             if (!plan.prefill && m->umma_ready)
-                return launch_umma_dense(m->tm_h, m->tm_lm, n_emit, s.V, s.H, b.logits, b.err, st);
+                return launch_umma_dense(m->tm_h, m->tm_lm, n_emit, s.V, s.H, b.logits, b.err, 1, st);
             return launch_lm_head(s, b, lay, m->lm_head, n_emit, m->sm_count, st);
         });
         if (dbg && dbg->logits)
@@ -1455,6 +1458,13 @@ mars_status_t mars_debug_bounded_wait(mars_model_t* m, void* cuda_stream, int32_
     launch_wait_probe(m->buf.err, arrive ? 1 : 0, 4096u, st);
     CUDA_TRY(cudaGetLastError());
     m->last_stream = st;
+    return MARS_OK;
+}
+
+mars_status_t mars_set_prefill_lo_planes(mars_model_t* m, int32_t mask) {
+    if (!m) return MARS_ERR_BAD_HANDLE;
+    if (mask < 0 || mask > MARS_LO_ALL) return MARS_ERR_INVALID_ARG;
+    m->lo_planes = mask;
     return MARS_OK;
 }
 

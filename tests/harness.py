@@ -18,7 +18,7 @@ TOL_LOGIT_GAP = 1e-2
 TOL_LOGIT_ABS = 2e-2
 TOL_HIDDEN_REL = 1e-2
 TOL_ROUTER_W = 2e-3
-CACHE_FLOOR_FIRST, CACHE_FLOOR_DEEP = 2e-5, 1e-3   # of the row RMS, on top of one bf16 step (see check_cache_rows)
+CACHE_FLOOR_FIRST, CACHE_FLOOR_DEEP, CACHE_FLOOR_LARGE = 2e-5, 1e-3, 5e-3   # of the row RMS, on top of one bf16 step (see check_cache_rows)
 
 
 class Case:
@@ -107,7 +107,7 @@ class Case:
         return res
 
 
-def check_cache_rows(got_k, got_v, want_k, want_v, rows, label="", first_layer=0):
+def check_cache_rows(got_k, got_v, want_k, want_v, rows, label="", first_layer=0, floor_deep=None):
     """The key/value rows written by the step against the oracle's, element by element.
 
     got_* / want_*: pools [L, pages, n_kv_heads, page_size, head_dim] (the CUDA path's, the oracle's);
@@ -122,11 +122,15 @@ def check_cache_rows(got_k, got_v, want_k, want_v, rows, label="", first_layer=0
                   rounded up and the other down (a fraction ~ error / ulp of all elements) is off by a whole
                   bf16 step, which attention over few or all-new keys (short contexts, prefill chunks)
                   passes on: 1e-4 .. 4e-4 of the RMS measured after one layer and in the middle of the
-                  48-layer model.  Still 10 times inside the 1e-2 hidden-state tolerance.
+                  48-layer model.  Still 10 times inside the 1e-2 hidden-state tolerance.  Calls of more
+                  than 256 rows contract the experts with plain bf16 activations (hidden-state error
+                  2.5e-3 over 48 layers instead of 6e-4, measured): they pass floor_deep = CACHE_FLOOR_LARGE,
+                  half the hidden-state tolerance.
     Returns the largest excess over one bf16 step, in units of the row RMS."""
     worst = 0.0
     L = got_k.shape[0]
-    floor = torch.tensor([CACHE_FLOOR_FIRST if first_layer + l == 0 else CACHE_FLOOR_DEEP for l in range(L)])[:, None, None]
+    deep = CACHE_FLOOR_DEEP if floor_deep is None else floor_deep
+    floor = torch.tensor([CACHE_FLOOR_FIRST if first_layer + l == 0 else deep for l in range(L)])[:, None, None]
     for page, slot in rows:
         for got, want in ((got_k, want_k), (got_v, want_v)):
             g, w = got[:, page, :, slot].float().cpu(), want[:, page, :, slot].float().cpu()
@@ -304,7 +308,8 @@ def prefill_and_compare(model, ps, ctx, lens, seed, label, check_rows="all"):
     for r in range(R):
         ts = range(ctx[r], ctx[r] + lens[r]) if check_rows == "all" else sorted({ctx[r], ctx[r] + lens[r] - 1})
         rows += [(case.pages[r][t // ps], t % ps) for t in ts]
-    stats["cache_excess"] = check_cache_rows(case.k_pool.cpu(), case.v_pool.cpu(), case.k_cpu, case.v_cpu, rows, label)
+    stats["cache_excess"] = check_cache_rows(case.k_pool.cpu(), case.v_pool.cpu(), case.k_cpu, case.v_cpu, rows, label,
+                                             floor_deep=CACHE_FLOOR_LARGE if n > 256 else None)
     print(label, stats)
     case.cur = [c + l for c, l in zip(ctx, lens)]
     case.last_gpu = gpu
