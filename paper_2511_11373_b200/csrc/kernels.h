@@ -138,7 +138,7 @@ int launch_down(const Shape& s, const Buffers& b, const LayerW& w, int n_tok, cu
 int launch_combine(const Shape& s, const Buffers& b, const __nv_bfloat16* next_gain, float* hidden_tap, int n_tok,
                    cudaStream_t st);
 
-int launch_sample(const Shape& s, const Buffers& b, const StepLayout& lay, int n_emit, int32_t* out_tokens,
+int launch_sample(const Shape& s, const Buffers& b, const StepLayout& lay, int n_emit, int sm_count, int32_t* out_tokens,
                   float* out_logprobs, float* nucleus_mass, cudaStream_t st);
 
 // Copies n_pages pages in each of n_layers layers: unit (layer, i) goes from

@@ -49,6 +49,7 @@ struct Caps {
     int n_emit;    // sampled rows per call
     int n_updates; // block-table writes per call
     int n_items;   // attention work items per call
+    bool keep_weights = true;   // room for the sampler's softmax weights (not in the fixed-scratch entry)
 };
 
 Caps make_caps(const mars_config_t& c, int max_decode, int max_prefill) {
@@ -127,6 +128,8 @@ size_t carve(const mars_config_t& c, const Caps& k, const StepLayout& lay, unsig
     t.xperm = (__nv_bfloat16*)take(n > kUmmaMinTokens ? n * kk * 2 * H * 2 : 0);
     t.y = (float*)take(n * kk * H * 4);
     t.logits = (float*)take((size_t)k.n_emit * c.vocab * 4);
+    t.expw = (float*)take(k.keep_weights ? (size_t)k.n_emit * c.vocab * 4 : 0);
+    if (!k.keep_weights) t.expw = nullptr;
     int32_t* a = (int32_t*)take((size_t)k.n_emit * 4);
     int32_t* o = (int32_t*)take((size_t)k.n_emit * 4);
     float* lp = (float*)take((size_t)k.n_emit * 4);
@@ -1011,7 +1014,7 @@ mars_status_t run_step(mars_model* m, mars_kv* kv, cudaStream_t st, const StepPl
         if (dbg && dbg->logits)
             CUDA_TRY(cudaMemcpyAsync(dbg->logits, b.logits, (size_t)n_emit * s.V * 4, cudaMemcpyDeviceToDevice, st));
         run(MARS_K_SAMPLE, [&] {
-            return launch_sample(s, b, lay, n_emit, out_tokens, out_logprobs, taps.nucleus_mass, st);
+            return launch_sample(s, b, lay, n_emit, m->sm_count, out_tokens, out_logprobs, taps.nucleus_mass, st);
         });
     }
     if (plan.score_targets) {
@@ -1338,7 +1341,8 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
     if (rows > 0x7fffffffull) return MARS_ERR_UNSUPPORTED;
 
     // everything the step needs must fit the built-in array
-    const Caps caps = make_caps(*cfg, n_seqs, 0);
+    Caps caps = make_caps(*cfg, n_seqs, 0);
+    caps.keep_weights = false;             // the sampler recomputes its weights: the fixed scratch has no room to keep them
     const StepLayout lay = make_layout(caps);
     const size_t need = carve(*cfg, caps, lay, nullptr, nullptr, nullptr, nullptr, nullptr);
     if (need > (size_t)MARS_STATIC_SCRATCH_BYTES) return MARS_ERR_TOO_LARGE;
@@ -1436,7 +1440,7 @@ mars_status_t mars_decode_step_static(const mars_config_t* cfg, const mars_weigh
         launch_combine(s, buf, next_gain, nullptr, n_seqs, st);
     }
     launch_lm_head(s, buf, lay, (const __nv_bfloat16*)w->lm_head, n_seqs, sms, st);
-    launch_sample(s, buf, lay, n_seqs, out_tokens, out_logprobs, nullptr, st);
+    launch_sample(s, buf, lay, n_seqs, 0, out_tokens, out_logprobs, nullptr, st);      // one block per row
     CUDA_TRY(cudaGetLastError());
     return MARS_OK;
 }

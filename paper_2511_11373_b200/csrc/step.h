@@ -75,6 +75,7 @@ struct Buffers {
     __nv_bfloat16* xperm;   // [n_tok k, 2, H] activations gathered into expert-slot order (prefill path only)
     float* y;               // [n_tok k, H]
     float* logits;          // [n_emit, V]
+    float* expw;            // [n_emit, V] softmax weights exp((l - max) / T) kept between the sampler's passes, or null
 };
 
 }  // namespace mars
