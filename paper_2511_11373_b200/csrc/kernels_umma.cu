@@ -136,6 +136,7 @@ struct UmmaParams {
     int tiles_x;              // column tiles per row tile (mode 1: 128 output columns each, else 256)
     int use_lo;               // 1: accumulate the lo plane of the activations as well (hi + lo = ~16 mantissa bits)
     QkvEpilogue qkv;          // mode 3: the tile's columns are whole heads of the QKV projection (kernels.h)
+    int out_lo;               // mode 1: 1 = write the lo plane of the activations too (the consumer reads it)
 };
 
 template <int D>
@@ -416,7 +417,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                                     lo[q] = pack_bf16(a[0] - bf16_lo(hi[q]), a[1] - bf16_hi(hi[q]));
                                 }
                                 *reinterpret_cast<uint4*>(dst + j) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                                *reinterpret_cast<uint4*>(dst + p.n_cols + j) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                                if (p.out_lo) *reinterpret_cast<uint4*>(dst + p.n_cols + j) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                             }
                     }
                 }
@@ -613,14 +614,14 @@ int umma_swap_splits(int rows, int n_tok, int K) {
 }
 
 // Rows of the normalised activations gathered into expert-slot order: xperm[slot] = h[slot_token[slot]]
-// (both planes), so that a group's rows are one contiguous TMA box.
-__global__ void __launch_bounds__(256) gather_rows_kernel(Buffers b, int H, int n_slots) {
+// (the hi plane, and the lo plane when the contraction uses it), so that a group's rows are one contiguous TMA box.
+__global__ void __launch_bounds__(256) gather_rows_kernel(Buffers b, int H, int n_slots, int planes) {
     pdl_wait();
     const int slot = blockIdx.x;
     if (slot >= n_slots) return;
     const uint4* src = reinterpret_cast<const uint4*>(b.h + (size_t)b.slot_token[slot] * 2 * H);
     uint4* dst = reinterpret_cast<uint4*>(b.xperm + (size_t)slot * 2 * H);
-    for (int i = threadIdx.x; i < 2 * H / 8; i += blockDim.x) dst[i] = src[i];
+    for (int i = threadIdx.x; i < planes * H / 8; i += blockDim.x) dst[i] = src[i];
 }
 
 static size_t umma_smem_bytes() { return (size_t)kUmStages * kUmStageBytes + 1024; }
@@ -649,9 +650,10 @@ int launch_umma_experts(const Shape& s, const Buffers& b, const CUtensorMap& tm_
                         const CUtensorMap& tm_act, const CUtensorMap& tm_wdown, int n_tok, int gate_up_lo, int down_lo, cudaStream_t st) {
     const int n_slots = n_tok * s.k;
     const int max_groups = s.E + (n_slots + kUmTileM - 1) / kUmTileM;
-    launch_chained(gather_rows_kernel, dim3(n_slots), dim3(256), 0, st, b, s.H, n_slots);
+    launch_chained(gather_rows_kernel, dim3(n_slots), dim3(256), 0, st, b, s.H, n_slots, gate_up_lo ? 2 : 1);
     const int gx = (s.I + 127) / 128, dx = (s.H + kUmTileN - 1) / kUmTileN;
     UmmaParams gu{s.H, n_slots, b.groups, b.n_groups, 2 * s.I, s.I, 1, nullptr, b.act, b.err, nullptr, 0.f, nullptr, nullptr, gx, gate_up_lo, QkvEpilogue{}};
+    gu.out_lo = down_lo;
     launch_chained(umma_gemm_kernel, dim3(umma_grid(gx * max_groups)), dim3(kUmThreads), umma_smem_bytes(), st, tm_xperm,
                    tm_wgu, gu);
     UmmaParams dn{s.I, n_slots, b.groups, b.n_groups, s.H, s.H, 0, b.y, nullptr, b.err, nullptr, 0.f, nullptr, nullptr, dx, down_lo, QkvEpilogue{}};
