@@ -184,6 +184,9 @@ class DecodeWorkload:
 
 
 # ----------------------------------------------------------------------------------- CPU baseline
+ORACLE_SAMPLE_SEQS = 8     # sequences of the workload that both arms' CPU-oracle figures are taken on
+
+
 class OracleSample:
     """The CPU oracle, as it stands, on a bounded sample of the workload: ONE decoder layer plus the
     lm_head and sampling over the first n_seq sequences (own CPU-generated weights and cache of the
@@ -256,7 +259,7 @@ def run_reference(args):
     if rank != 0:
         return
     cfg = wl.CONFIGS[args.workload]
-    sample = OracleSample(cfg, 4)
+    sample = OracleSample(cfg, ORACLE_SAMPLE_SEQS)
     for _ in range(args.warmup):
         sample.run()
     t0 = time.perf_counter()
@@ -602,7 +605,7 @@ def run_cuda(args):
         extra["4"] = measure_mixed(wl.CONFIGS[4], sub, device, weights=weights)
         for k in ("metric", "unit", "n_gpus", "higher_is_better", "scaling", "vs_baseline", "dtype", "data", "value", "steps", "warmup"):
             extra["4"].pop(k, None)
-    cpu = OracleSample(cfg, 8).run()
+    cpu = OracleSample(cfg, ORACLE_SAMPLE_SEQS).run()
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic",
