@@ -77,6 +77,44 @@ def test_top_p_one_and_training_temperature():
     assert torch.allclose(gpu["nucleus_mass"], torch.ones(2), atol=1e-6)
 
 
+@pytest.mark.parametrize("vocab", [1021, 1022, 130])
+def test_vocabulary_sizes_off_every_tile_and_vector_width(vocab):
+    """Odd and tiny vocabularies: the lm_head's last weight tile is ragged, a row of logits does not
+    start on a 16-byte boundary, and the sampler takes its element-wise loads."""
+    model = dict(wl.MODEL_TINY, n_layers=1, vocab=vocab)
+    ctx = [9, 40, 17]
+    case = Case(model, 16, ctx, seed=21, headroom=3)
+    tokens = wl.make_tokens(len(ctx), vocab, seed=4)
+    run_and_compare(case, tokens, label=f"vocab {vocab} greedy")
+    for step, smp in enumerate((dict(greedy=0, temperature=0.85, top_p=0.95), dict(greedy=0, temperature=1.7, top_p=1.0)), 1):
+        gpu, _, _ = run_and_compare(case, tokens, sampling=smp, label=f"vocab {vocab} {smp}", step=step, seed=77)
+        tokens = gpu["tokens"]
+        assert ((gpu["tokens"] >= 0) & (gpu["tokens"] < vocab)).all()
+
+
+def test_nucleus_of_one_token_and_very_low_temperature():
+    """top_p so small that the nucleus is the most probable token alone, and a temperature that makes
+    the distribution nearly one-hot (most weights underflow): both must return the argmax."""
+    model = dict(wl.MODEL_TINY, n_layers=1)
+    ctx = [33, 70]
+    case = Case(model, 16, ctx, seed=22, headroom=3)
+    tokens = wl.make_tokens(len(ctx), model["vocab"], seed=6)
+    greedy, orc, _ = run_and_compare(case, tokens, label="reference greedy")
+
+    def rewind():                              # the same state again, on both sides
+        for b, c in enumerate(ctx):
+            case.kv.seq_set_len(b, c)
+            case.cur[b] = c
+
+    rewind()
+    for step, smp in enumerate((dict(greedy=0, temperature=1.0, top_p=1e-6), dict(greedy=0, temperature=0.01, top_p=0.9)), 1):
+        gpu, _, _ = run_and_compare(case, tokens, sampling=smp, label=f"{smp}", step=step, seed=5)
+        gap = torch.topk(orc["logits"].double(), 2, dim=-1).values
+        sure = (gap[:, 0] - gap[:, 1]) >= 1e-2
+        assert (gpu["tokens"][sure] == greedy["tokens"][sure]).all()
+        rewind()
+
+
 def test_sampling_distribution_matches_oracle_probabilities():
     """Many draws from one fixed state (the context length is reset between steps): token-id bins
     are hit in proportion to the oracle's nucleus probabilities."""
