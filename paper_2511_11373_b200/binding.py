@@ -18,6 +18,10 @@ MARS_OK = 0
 STATUS_NAMES = {0: "MARS_OK", 1: "MARS_ERR_INVALID_ARG", 2: "MARS_ERR_UNSUPPORTED", 3: "MARS_ERR_CUDA",
                 4: "MARS_ERR_KV_FULL", 5: "MARS_ERR_TIMEOUT", 6: "MARS_ERR_BAD_HANDLE", 7: "MARS_ERR_BAD_TOKEN",
                 8: "MARS_ERR_TOO_LARGE"}
+MARS_ERR_INVALID_ARG = 1
+# bits of mars_set_prefill_lo_planes
+MARS_LO_QKV, MARS_LO_OPROJ, MARS_LO_ROUTER, MARS_LO_GATE_UP, MARS_LO_DOWN = 1, 2, 4, 8, 16
+MARS_LO_ALL, MARS_LO_DEFAULT = 31, 7
 LAYER_FIELDS = ("attn_norm", "wqkv", "q_norm", "k_norm", "wo", "mlp_norm", "router", "w_gate_up", "w_down")
 
 

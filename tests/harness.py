@@ -274,13 +274,16 @@ def compare_sampled(gpu: dict, orc: dict, temperature: float, top_p: float, seed
     return stats
 
 
-def prefill_and_compare(model, ps, ctx, lens, seed, label, check_rows="all"):
+def prefill_and_compare(model, ps, ctx, lens, seed, label, check_rows="all", lo_planes=None):
     """One mars_prefill_chunk call over several requests (request r continues ctx[r] cached tokens
     with lens[r] new ones) against the oracle with the GPU's routing forced: every tap, the
     permutation's integer outputs and the appended cache rows (all of them, or the first and last
-    of every request).  Returns the case (positions advanced) and the sampled tokens."""
+    of every request).  lo_planes: mask for mars_set_prefill_lo_planes, or None for the library's default.
+    Returns the case (positions advanced; the comparison's figures in case.stats) and the sampled tokens."""
     n = sum(lens)
     case = Case(model, ps, ctx, seed=seed, headroom=max(lens) + 4, max_prefill_tokens=n, poison=True)
+    if lo_planes is not None:
+        case.model.set_prefill_lo_planes(lo_planes)
     dev = case.device
     L, H, k, V, E = model["n_layers"], model["hidden"], model["top_k"], model["vocab"], model["n_experts"]
     toks = wl.make_tokens(n, V, seed=seed + 100)
@@ -314,6 +317,7 @@ def prefill_and_compare(model, ps, ctx, lens, seed, label, check_rows="all"):
     stats["cache_excess"] = check_cache_rows(case.k_pool.cpu(), case.v_pool.cpu(), case.k_cpu, case.v_cpu, rows, label,
                                              floor_deep=CACHE_FLOOR_LARGE if n > 256 else None)
     print(label, stats)
+    case.stats = stats
     case.cur = [c + l for c, l in zip(ctx, lens)]
     case.last_gpu = gpu
     return case, out_t.cpu()

@@ -345,6 +345,23 @@ def test_prefill_tensor_core_path_at_the_full_layer_shape():
     prefill_and_compare(wl.MODEL_LAYER, 64, [0, 64], [400, 240], seed=62, label="prefill-full-shape-640")
 
 
+def test_activation_planes_of_large_calls_can_be_switched():
+    """mars_set_prefill_lo_planes: the default and the all-planes setting (and one in between) stay inside
+    the tolerances on a tensor-core-sized call, all planes give a smaller hidden-state error than the
+    default (experts on the hi plane), and a mask outside the defined bits is refused.  (With no lo
+    plane at all the router weights leave their tolerance, which is why the default keeps three.)"""
+    model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=1, hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=64)
+    err = {}
+    for mask in (binding.MARS_LO_ALL, binding.MARS_LO_DEFAULT | binding.MARS_LO_DOWN, binding.MARS_LO_DEFAULT):
+        case, _ = prefill_and_compare(model, 16, [0, 21], [200, 130], seed=41, label=f"lo planes {mask}", check_rows="ends",
+                                      lo_planes=mask)
+        err[mask] = case.stats["hidden_rel_max"]
+    assert err[binding.MARS_LO_ALL] < err[binding.MARS_LO_DEFAULT]
+    lib = binding.lib()
+    assert lib.mars_set_prefill_lo_planes(case.model.handle, 32) == binding.MARS_ERR_INVALID_ARG
+    assert lib.mars_set_prefill_lo_planes(case.model.handle, -1) == binding.MARS_ERR_INVALID_ARG
+
+
 def test_prefill_in_two_calls_equals_one_call():
     model = dict(wl.MODEL_TINY, n_layers=2, qk_norm=0)
     V = model["vocab"]
