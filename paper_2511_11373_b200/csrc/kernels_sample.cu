@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(Shape s, Buffers
 
     if (greedy) {
         if (tid == 0 && rank == 0) {
-            out_tokens[row] = am;
+            out_tokens[row] = am < V ? am : 0;   // (no logit compared greater than -inf: a row of NaN)
             out_logprobs[row] = -log_z;     // (l_max - max) / 1 - log Z
             if (nucleus_mass) nucleus_mass[row] = 1.f;
         }
@@ -435,6 +435,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(Shape s, Buffers
         int tok = xc.sel_token;
         if (C > 1 && tok < 0) tok = (int)ld_peer_u32(peer_smem(&xc.sel_token, 1u));
         if (tok < 0) tok = am;   // cannot happen while mass_s > 0; keeps the output defined
+        if (tok < 0 || tok >= V) tok = 0;   // a row of NaN has no maximum either: stay inside the row
         out_tokens[row] = tok;
         out_logprobs[row] = (l[tok] - mx) * inv_t - log_z;
         if (nucleus_mass) nucleus_mass[row] = (float)((double)mass_s / (double)z_fix);
