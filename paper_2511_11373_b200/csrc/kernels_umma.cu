@@ -453,9 +453,15 @@ struct SwCfg {
     static constexpr int kPlaneBytes = NB * kSwBoxBytes;
     static constexpr int kStageBytes = kSwABytes + 2 * kPlaneBytes;
     static constexpr int kStages = NB == 4 ? 2 : 3;                  // 96 / 144 / 192 / 160 KB of ring
-    static constexpr int kTmemCols = NB == 3 ? 256 : kTok;           // allocations are powers of two
+    // A tcgen05.mma of M 128, K 16 occupies the tensor pipe for ~108 clk whatever N <= 128 is (160 clk at N = 256;
+    // measured), so with up to 128 tokens the hi and the lo plane, which lie next to each other in a stage, are ONE
+    // operand of 2 x kTok columns: half as many instructions per stage, and the stream of 16 KB weight stages is no
+    // longer held to 8 x 108 clk each.  The two halves of the accumulator are added in the epilogue.
+    static constexpr bool kFusePlanes = NB <= 2;
+    static constexpr int kAccCols = kFusePlanes ? 2 * kTok : kTok;
+    static constexpr int kTmemCols = NB == 3 ? 256 : kAccCols;       // allocations are powers of two
     static constexpr int kCtasPerSm = NB == 1 ? 2 : 1;
-    static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAccCols >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     static constexpr size_t smem_bytes() { return (size_t)kStages * kStageBytes + 1024; }
 };
 
@@ -547,8 +553,8 @@ umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
                                d_lo = um_smem_desc(a + kSwABytes + kSwBBytes);
 #pragma unroll
                 for (int kk = 0; kk < kUmStageK / 16; ++kk) {
-                    um_mma_idesc(tmem_d, d_w + 2 * kk, d_hi + 2 * kk, kSwIdesc, (ks | kk) != 0);
-                    um_mma_idesc(tmem_d, d_w + 2 * kk, d_lo + 2 * kk, kSwIdesc, 1u);
+                    um_mma_idesc(tmem_d, d_w + 2 * kk, d_hi + 2 * kk, kSwIdesc, (ks | kk) != 0);   // fused: hi and lo rows in one operand
+                    if (!SwCfg<NB>::kFusePlanes) um_mma_idesc(tmem_d, d_w + 2 * kk, d_lo + 2 * kk, kSwIdesc, 1u);
                 }
                 um_commit(&empty_bar[s]);
             }
@@ -568,6 +574,12 @@ umma_swap_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
             for (int c = 0; c < kSwTok && c < p.n_tok; c += 32) {
                 uint32_t v[32];
                 um_ld32(lane_base + c, v);
+                if (SwCfg<NB>::kFusePlanes) {                        // columns kSwTok.. hold the lo plane's share
+                    uint32_t w[32];
+                    um_ld32(lane_base + kSwTok + c, w);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
+                }
                 if (row < p.rows) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
