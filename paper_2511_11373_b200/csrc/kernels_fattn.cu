@@ -7,21 +7,28 @@
 // causal mask is only 16 tokens wide.  A persistent CTA per SM walks units; per unit
 //   warp 8 (one lane)   TMA producer: the Q tile (hi and lo planes, two 64-wide halves of head_dim,
 //                       through a 4-D tensor map (d, head, plane, token)), then the K and V page
-//                       tiles of 64 cached tokens each through a 3-stage ring;
-//   warp 9 (one lane)   MMA issuer: S = Q K^T (M 128, N 64, K 128; hi and lo planes of Q accumulate
-//                       into the same fp32 tile in TMEM, two S buffers), and, once the softmax warps
-//                       have written P, O_tile = P V (M 128, N 128, K 64; hi and lo planes of P), with V
-//                       read as an MN-major operand straight from the [token][d] page tile;
+//                       tiles of 128 cached tokens each through two-stage rings;
+//   warp 10 (one lane)  S issuer: S = Q K^T (M 128, N 128, K 128; hi and lo planes of Q accumulate
+//                       into the same fp32 tile in TMEM, two S buffers);
+//   warp 9 (one lane)   P V issuer: once the softmax warps have written P, O_tile = P V (M 128, N 128,
+//                       K 128; hi and lo planes of P), with P read as the A operand from TENSOR MEMORY and
+//                       V as an MN-major operand straight from the [token][d] page tile.  (One lane can
+//                       issue a tcgen05.mma only every ~108 clk, whatever N <= 128 is: hence tiles as wide
+//                       as tensor memory allows and two issuing lanes.)
 //   warps 0..7          softmax: two threads share row r (TMEM lane r; warp w reads lanes 32 (w % 4) ..,
 //                       warps 0..3 the first half of the columns, warps 4..7 the second): each reads
-//                       its 32 scores with tcgen05.ld, masks by the row's causal length, the two
+//                       its 64 scores with tcgen05.ld, masks by the row's causal length, the two
 //                       exchange their maxima through shared memory, each writes its part of
-//                       P = exp2(s - m) as (hi, lo) bf16 pairs into a swizzled K-major shared tile and
-//                       adds its 64 columns of O_tile into fp32 output registers after rescaling them
-//                       (the output accumulator lives in registers, so no TMEM round trip is needed
-//                       when the running max moves).  Eight warps, two per scheduler, hide each
-//                       other's instruction latencies; with four the kernel ran at half the speed.
-// While the softmax warps work on tile j the tensor pipe already computes S of tile j + 1.
+//                       P = exp2(s - m) as (hi, lo) bf16 pairs back into tensor memory with tcgen05.st,
+//                       over the scores it came from (two tokens per column: hi plane in the first half
+//                       of the S buffer's columns, lo plane in the second), and adds its 64 columns of
+//                       O_tile into fp32 output registers after rescaling them (the output accumulator
+//                       lives in registers, so no TMEM round trip is needed when the running max moves).
+//                       Eight warps, two per scheduler, hide each other's instruction latencies; four
+//                       ran at half the speed, sixteen were slower again.
+// While the softmax warps work on tile j the tensor pipe already computes S of tile j + 1; S of tile
+// j + 2 waits for P V of tile j, whose P operand occupies the same columns.
+// Tensor memory: S / P buffers at columns 0 and 128, O_tile buffers at 256 and 384.
 //
 // SHARED mode (decode): the 16 "tokens" of a block are decode rows of DIFFERENT sequences that list the
 // same pages for a span of cached tokens (members of a rollout group forked from one prompt).  An
@@ -39,19 +46,23 @@ constexpr int kFaQ = 16;                   // query tokens per block
 constexpr int kFaHeads = 8;                // query heads per KV head
 constexpr int kFaRows = kFaQ * kFaHeads;   // 128 rows of the MMA tile
 constexpr int kFaD = 128;
-constexpr int kFaKv = 64;                  // cached tokens per tile
+constexpr int kFaKv = 128;                 // cached tokens per tile.  A tcgen05.mma of M 128, K 16 occupies the tensor pipe for
+                                            // ~108 clk whatever N <= 128 is (measured), so the tile is as wide as tensor memory
+                                            // allows: half as many S instructions per key as with 64
 constexpr int kFaKStages = 2;               // K tiles in flight (free as soon as S is computed)
-constexpr int kFaVStages = 3;               // V tiles in flight (free after P V)
+constexpr int kFaVStages = 2;               // V tiles in flight (free after P V)
 constexpr int kFaQTile = kFaRows * 128;    // one (plane, half) tile of Q: 128 rows x 128 B = 16 KB
 constexpr int kFaQBytes = 4 * kFaQTile;    // hi/lo x two halves of head_dim
-constexpr int kFaPTile = kFaRows * 128;    // one plane of P: 128 rows x 64 tokens bf16
-constexpr int kFaHalf = kFaKv * 128;       // one 64-wide half of a K or V tile: 64 tokens x 128 B = 8 KB
+constexpr int kFaHalf = kFaKv * 128;       // one 64-wide half (of head_dim) of a K or V tile: 128 tokens x 128 B = 16 KB
 constexpr int kFaTile = 2 * kFaHalf;        // a K or a V tile: two halves
-constexpr int kFaPBuf = 2 * kFaPTile;       // hi and lo planes of P
-constexpr int kFaSmem = kFaQBytes + 2 * kFaPBuf + (kFaKStages + kFaVStages) * kFaTile;
-constexpr int kFaThreads = 320;             // 8 softmax warps, producer warp, MMA warp
-constexpr int kFaSoftmaxThreads = 256;
-constexpr int kFaTmemCols = 512;           // S buffers at columns 0 and 64, O_tile buffers at 128 and 256
+constexpr int kFaSmem = kFaQBytes + (kFaKStages + kFaVStages) * kFaTile;
+constexpr int kFaParts = 2;                 // threads per row of the tile (each a quarter of the score / output columns)
+constexpr int kFaSoftmaxWarps = 4 * kFaParts;
+constexpr int kFaSoftmaxThreads = 32 * kFaSoftmaxWarps;
+constexpr int kFaThreads = kFaSoftmaxThreads + 96;   // softmax warps, producer warp, two MMA warps (P V and S)
+constexpr int kFaTmemCols = 512;           // S buffers (P over them) at columns 0 and 128, O_tile buffers at 256 and 384
+constexpr int kFaOCol = 2 * kFaKv;          // first O_tile column
+static_assert(kFaOCol + 2 * kFaD <= kFaTmemCols, "tensor memory layout");
 constexpr uint32_t kFaSpin = 1u << 22;
 
 constexpr int kFaShItem = 4 + 2 * kFaQ;   // words of a shared item
@@ -152,6 +163,25 @@ __device__ __forceinline__ void fa_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 16 consecutive TMEM columns of this thread's lane (the mirror image of the load above).
+__device__ __forceinline__ void fa_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+// D += A B with the A operand in tensor memory: 128 lanes (rows) x 8 columns, two bf16 per column, per K step of 16.
+__device__ __forceinline__ void fa_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
+
 __device__ __forceinline__ float fa_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -185,27 +215,26 @@ fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     extern __shared__ unsigned char fa_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)fa_raw + 1023) & ~(uintptr_t)1023);
     unsigned char* q_smem = smem;                                   // [plane][half][128 rows][128 B]
-    unsigned char* p_smem = smem + kFaQBytes;                       // [buffer][plane][128 rows][128 B]
-    unsigned char* k_smem = p_smem + 2 * kFaPBuf;                   // [stage][half][64 tokens][128 B]
-    unsigned char* v_smem = k_smem + kFaKStages * kFaTile;          // [stage][half][64 tokens][128 B]
+    unsigned char* k_smem = smem + kFaQBytes;                       // [stage][half][128 tokens][128 B]
+    unsigned char* v_smem = k_smem + kFaKStages * kFaTile;          // [stage][half][128 tokens][128 B]
     __shared__ __align__(8) uint64_t q_full, q_free, k_full[kFaKStages], k_empty[kFaKStages], v_full[kFaVStages],
-        v_empty[kFaVStages], s_ready[2], p_ready[2], o_ready[2];
+        v_empty[kFaVStages], s_ready[2], p_ready[2], o_ready[2], pv_done[2];
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int dead;
-    __shared__ float xmax[2][2][kFaRows];                            // [tile parity][column half][row]
-    __shared__ float xsum[2][kFaRows];
+    __shared__ float xmax[2][kFaParts][kFaRows];                     // [tile parity][column part][row]
+    __shared__ float xsum[kFaParts][kFaRows];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
         fa_mbar_init(&q_full, 1); fa_mbar_init(&q_free, 1);
         for (int i = 0; i < kFaKStages; ++i) { fa_mbar_init(&k_full[i], 1); fa_mbar_init(&k_empty[i], 1); }
         for (int i = 0; i < kFaVStages; ++i) { fa_mbar_init(&v_full[i], 1); fa_mbar_init(&v_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { fa_mbar_init(&s_ready[i], 1); fa_mbar_init(&p_ready[i], 8); fa_mbar_init(&o_ready[i], 1); }
+        for (int i = 0; i < 2; ++i) { fa_mbar_init(&s_ready[i], 1); fa_mbar_init(&p_ready[i], kFaSoftmaxWarps); fa_mbar_init(&o_ready[i], 1); fa_mbar_init(&pv_done[i], 1); }
         dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 8) {
+    if (warp == kFaSoftmaxWarps) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
                      "r"(kFaTmemCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
@@ -218,7 +247,7 @@ fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 
     const int n_units = p.step[SHARED ? H_SH_ITEMS : H_PF_ITEMS] * p.nkv;
 
-    if (warp == 8) {
+    if (warp == kFaSoftmaxWarps) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t g = 0;                                          // tiles requested so far (ring positions)
@@ -277,56 +306,63 @@ fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 if (!ok) { dead = 1; atomicOr(p.err, kErrTimeout); }
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == kFaSoftmaxWarps + 1) {
         // ------------------------------------------------------------------ MMA issuer
-        // Order on the tensor pipe: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...: S runs one tile ahead of
-        // the softmax, so that the softmax warps never wait for scores, and P V of tile g overlaps the
-        // softmax of tile g + 1 (P and O_tile are double-buffered).
+        // P V issuer: O_tile(g) = P(g) V(g) as soon as the softmax warps have written P(g) (into tensor memory, over S(g))
         if (lane == 0) {
             uint32_t g = 0;                                          // tiles consumed so far
-            int local = 0;
-            const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem);
-            auto issue_s = [&](uint32_t gi) -> bool {                // S(gi) = Q K^T into S buffer gi & 1
-                const int ks = gi % kFaKStages;
-                if (!fa_wait(&k_full[ks], (gi / kFaKStages) & 1)) return false;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t k_addr = smem_u32(k_smem + (size_t)ks * kFaTile);
-                const uint32_t acc = tmem + (gi & 1) * kFaKv;
-#pragma unroll
-                for (int pl = 0; pl < 2; ++pl)
-#pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {
-                        const uint64_t da = fa_desc_kmajor(q_addr + (pl * 2 + hf) * kFaQTile);
-                        const uint64_t db = fa_desc_kmajor(k_addr + hf * kFaHalf);
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) fa_mma(acc, da + 2 * kk, db + 2 * kk, kFaIdescS, (pl | hf | kk) != 0);
-                    }
-                fa_commit(&s_ready[gi & 1]);
-                fa_commit(&k_empty[ks]);                             // the K tile is free once these MMAs retire
-                return true;
-            };
-            for (int u = blockIdx.x; u < n_units && !dead; u += gridDim.x, ++local) {
+            for (int u = blockIdx.x; u < n_units && !dead; u += gridDim.x) {
                 const FaUnit c = fa_unit<SHARED>(p, u);
-                bool ok = fa_wait(&q_full, local & 1);
-                if (ok) ok = issue_s(g);
-                if (ok && c.n_tiles > 1) ok = issue_s(g + 1);
+                bool ok = true;
                 for (int j = 0; j < c.n_tiles && ok; ++j, ++g) {
                     const int vs = g % kFaVStages;
                     ok = fa_wait(&p_ready[g & 1], (g >> 1) & 1) && fa_wait(&v_full[vs], (g / kFaVStages) & 1);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t dv = fa_desc_mnmajor(smem_u32(v_smem + (size_t)vs * kFaTile), kFaHalf);
-                    const uint32_t acc = tmem + 128 + (g & 1) * kFaD;
+                    const uint32_t acc = tmem + kFaOCol + (g & 1) * kFaD;
+                    const uint32_t pt = tmem + (g & 1) * kFaKv;
 #pragma unroll
-                    for (int pl = 0; pl < 2; ++pl) {
-                        const uint64_t dp = fa_desc_kmajor(p_addr + (g & 1) * kFaPBuf + pl * kFaPTile);
+                    for (int pl = 0; pl < 2; ++pl)
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)     // 16 tokens per step: 32 B along a P row, 2048 B down the V tile
-                            fa_mma(acc, dp + 2 * kk, dv + 128 * kk, kFaIdescO, (pl | kk) != 0);
-                    }
+                        for (int kk = 0; kk < kFaKv / 16; ++kk)
+                            fa_mma_ts(acc, pt + pl * (kFaKv / 2) + kk * 8, dv + 128 * kk, kFaIdescO, (pl | kk) != 0);
                     fa_commit(&o_ready[g & 1]);
                     fa_commit(&v_empty[vs]);
-                    if (j + 2 < c.n_tiles) ok = issue_s(g + 2);
+                    fa_commit(&pv_done[g & 1]);                      // P(g) has been consumed: its columns may take S(g + 2)
+                }
+                if (!ok) { dead = 1; atomicOr(p.err, kErrTimeout); break; }
+            }
+        }
+    } else if (warp == kFaSoftmaxWarps + 2) {
+        // S issuer, a lane of its own (one lane issues a tcgen05.mma only every ~108 clk): S(g) = Q K(g)^T into S
+        // buffer g & 1 once P V(g - 2), which reads P(g - 2) out of the same columns, has retired.
+        if (lane == 0) {
+            uint32_t g = 0;
+            int local = 0;
+            const uint32_t q_addr = smem_u32(q_smem);
+            for (int u = blockIdx.x; u < n_units && !dead; u += gridDim.x, ++local) {
+                const FaUnit c = fa_unit<SHARED>(p, u);
+                bool ok = fa_wait(&q_full, local & 1);
+                for (int j = 0; j < c.n_tiles && ok; ++j, ++g) {
+                    const int ks = g % kFaKStages;
+                    if (g >= 2) ok = fa_wait(&pv_done[g & 1], ((g - 2) >> 1) & 1);
+                    if (ok) ok = fa_wait(&k_full[ks], (g / kFaKStages) & 1);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t k_addr = smem_u32(k_smem + (size_t)ks * kFaTile);
+                    const uint32_t acc = tmem + (g & 1) * kFaKv;
+#pragma unroll
+                    for (int pl = 0; pl < 2; ++pl)
+#pragma unroll
+                        for (int hf = 0; hf < 2; ++hf) {
+                            const uint64_t da = fa_desc_kmajor(q_addr + (pl * 2 + hf) * kFaQTile);
+                            const uint64_t db = fa_desc_kmajor(k_addr + hf * kFaHalf);
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) fa_mma(acc, da + 2 * kk, db + 2 * kk, kFaIdescS, (pl | hf | kk) != 0);
+                        }
+                    fa_commit(&s_ready[g & 1]);
+                    fa_commit(&k_empty[ks]);                         // the K tile is free once these MMAs retire
                 }
                 if (!ok) { dead = 1; atomicOr(p.err, kErrTimeout); break; }
                 fa_commit(&q_free);                                  // every MMA that reads this unit's Q has been issued
@@ -334,11 +370,11 @@ fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------------ softmax warps
-        const int quarter = warp & 3, half = warp >> 2;
+        const int quarter = warp & 3, half = warp >> 2;           // half: which part of the columns (0 .. kFaParts - 1)
         const int r = quarter * 32 + lane;                           // row of the tile = TMEM lane
         const int q_tok = r >> 3, head = r & 7;
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
-        constexpr int SC = kFaKv / 2, OC = kFaD / 2;                 // score and output columns of this thread
+        constexpr int SC = kFaKv / kFaParts, OC = kFaD / kFaParts;   // score and output columns of this thread
         uint32_t g = 0;
         for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
             const FaUnit c = fa_unit<SHARED>(p, u);
@@ -357,7 +393,7 @@ fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 #pragma unroll
                 for (int cb = 0; cb < OC; cb += 32) {
                     uint32_t v[32];
-                    fa_ld32(lane_base + 128 + (gt & 1) * kFaD + half * OC + cb, v);
+                    fa_ld32(lane_base + kFaOCol + (gt & 1) * kFaD + half * OC + cb, v);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) o[cb + i] = fmaf(o[cb + i], alpha, __uint_as_float(v[i]));
                 }
@@ -371,42 +407,46 @@ fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 if (lane == 0 && !dead && !fa_wait(&s_ready[g & 1], (g >> 1) & 1)) { dead = 1; atomicOr(p.err, kErrTimeout); }
                 __syncwarp();
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                // this thread's 32 scores of the row
+                // this thread's 64 scores of the row
                 const int kv0 = j * kFaKv + half * SC;
                 float sv[SC];
                 float mx = -INFINITY;
-                {
-                    uint32_t v[32];
-                    fa_ld32(lane_base + (g & 1) * kFaKv + half * SC, v);
 #pragma unroll
-                    for (int i = 0; i < SC; ++i) {
-                        sv[i] = kv0 + i < my_len ? __uint_as_float(v[i]) * p.scale_log2 : -INFINITY;
-                        mx = fmaxf(mx, sv[i]);
+                for (int cb = 0; cb < SC; cb += 32) {
+                    uint32_t v[32];
+                    fa_ld32(lane_base + (g & 1) * kFaKv + half * SC + cb, v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        sv[cb + i] = kv0 + cb + i < my_len ? __uint_as_float(v[i]) * p.scale_log2 : -INFINITY;
+                        mx = fmaxf(mx, sv[cb + i]);
                     }
                 }
                 xmax[g & 1][half][r] = mx;
                 asm volatile("bar.sync 1, %0;" ::"n"(kFaSoftmaxThreads) : "memory");
-                const float m_new = fmaxf(m_run, fmaxf(mx, xmax[g & 1][half ^ 1][r]));
+                float mo = mx;
+#pragma unroll
+                for (int q = 0; q < kFaParts; ++q) mo = fmaxf(mo, xmax[g & 1][q][r]);
+                const float m_new = fmaxf(m_run, mo);
                 const float m_use = m_new == -INFINITY ? 0.f : m_new;
                 const float alpha = fa_exp2(m_run - m_use);
                 float sum = 0.f;
-                // P as (hi, lo) bf16 planes, K-major with the 128-byte swizzle: 16-byte chunk c of row r
-                // sits at r * 128 + ((c ^ (r & 7)) << 4).  Buffer g & 1: P V of tile g - 2, which read it
-                // last, was waited for before tile g - 1's softmax.
-                unsigned char* prow = p_smem + (g & 1) * kFaPBuf + r * 128;
+                // P as (hi, lo) bf16 planes goes back into tensor memory, over this tile's scores (every thread of
+                // the row has read them: the barrier above): the A operand of P V is row = lane, two tokens per
+                // column, so this thread's 64 tokens are 32 columns of the hi plane (first half of the S buffer's
+                // columns) and 32 of the lo plane (second half).  No shared-memory round trip, no proxy fence.
 #pragma unroll
-                for (int ch = 0; ch < SC / 8; ++ch) {
-                    uint32_t hi[4], lo[4];
+                for (int cb = 0; cb < SC; cb += 32) {
+                    uint32_t hi[16], lo[16];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float a = fa_exp2(sv[ch * 8 + 2 * q] - m_use), b2 = fa_exp2(sv[ch * 8 + 2 * q + 1] - m_use);
+                    for (int q = 0; q < 16; ++q) {
+                        const float a = fa_exp2(sv[cb + 2 * q] - m_use), b2 = fa_exp2(sv[cb + 2 * q + 1] - m_use);
                         sum += a + b2;
                         hi[q] = pack_bf16(a, b2);
                         lo[q] = pack_bf16(a - bf16_lo(hi[q]), b2 - bf16_hi(hi[q]));
                     }
-                    const int sw = ((half * (SC / 8) + ch) ^ (r & 7)) << 4;
-                    *reinterpret_cast<uint4*>(prow + sw) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<uint4*>(prow + kFaPTile + sw) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    const uint32_t pt = lane_base + (g & 1) * kFaKv + (half * SC + cb) / 2;
+                    fa_st16(pt, hi);
+                    fa_st16(pt + kFaKv / 2, lo);
                 }
                 l_run = l_run * alpha + sum;
                 m_run = m_new;
@@ -423,9 +463,10 @@ fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                         *reinterpret_cast<uint4*>(vt + (piece >> 3) * kFaHalf + row * 128 + (piece & 7) * 16) = make_uint4(0, 0, 0, 0);
                     }
                 }
-                // P (and the cleared rows) must be visible to the tensor core's reads; the S buffer has
-                // been read: hand over to the MMA lane
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                // P must have landed in tensor memory, and cleared value rows must be visible to the tensor core's
+                // reads: hand over to the MMA lane
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                if (n_valid < kFaKv) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) fa_arrive(&p_ready[g & 1]);
@@ -437,7 +478,9 @@ fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             // the row's sum: both threads of the row saw the same sequence of maxima, so their sums add
             xsum[half][r] = l_run;
             asm volatile("bar.sync 1, %0;" ::"n"(kFaSoftmaxThreads) : "memory");
-            const float l_row = l_run + xsum[half ^ 1][r];
+            float l_row = 0.f;                                       // the same order in every thread of the row
+#pragma unroll
+            for (int q = 0; q < kFaParts; ++q) l_row += xsum[q][r];
             if (SHARED) {
                 if (q_tok < c.nq_blk) {
                     const size_t ph = (size_t)c.it[4 + kFaQ + q_tok] * p.nq + c.hk * kFaHeads + head;
@@ -467,7 +510,7 @@ fattn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
     __syncthreads();
-    if (warp == 8) {
+    if (warp == kFaSoftmaxWarps) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kFaTmemCols));
     }
@@ -481,7 +524,7 @@ static FaParams fa_params(const Shape& s, const Buffers& b, const StepLayout& la
     p.step = b.step; p.lay = lay; p.block_table = kv.block_table; p.o_out = b.o; p.part_o = b.part_o; p.part_ml = b.part_ml;
     p.err = b.err;
     p.max_pages_per_seq = kv.max_pages_per_seq; p.n_pages = kv.n_pages; p.page_size = kv.page_size;
-    p.box_rows = kv.page_size < kFaKv ? kv.page_size : kFaKv;
+    p.box_rows = kv.page_size < 64 ? kv.page_size : 64;   // rows of a box of the cache pools' tensor maps
     p.nkv = s.nkv; p.nq = s.nq; p.layer = layer;
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s.D));
     return p;
