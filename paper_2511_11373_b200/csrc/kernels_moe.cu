@@ -43,12 +43,13 @@ __device__ void route_select(float* z, const Shape& s, const Buffers& b, const D
                 const float v = z[e];
                 if (v > best) { best = v; bi = e; }   // ascending e: the lower index wins ties
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, best, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
-            }
+            // across the lanes with two warp reductions instead of ten shuffles: probabilities are non-negative floats,
+            // whose bit patterns order like the values (+1 keeps 0 for "nothing left in this lane"); among the lanes
+            // that hold the maximum the lowest expert index wins
+            const unsigned int key = best >= 0.f ? __float_as_uint(best) + 1u : 0u;
+            const unsigned int top = __reduce_max_sync(0xffffffffu, key);
+            bi = __reduce_min_sync(0xffffffffu, key == top ? bi : 0x7fffffff);
+            best = __uint_as_float(top - 1u);
             if (lane == j) { my_idx = bi; my_p = best; }
             if (lane == 0) z[bi] = -1.f;               // taken
             __syncwarp();
